@@ -1,0 +1,152 @@
+/*
+ * pac.h - C ABI of the adapter-over-cache trainer (one GPU, sm_100a).
+ *
+ * The library trains the Parallel Adapters side network of PAC+ (arXiv
+ * 2408.10746) from an activation cache: the frozen backbone's per-layer hidden
+ * states b_1..b_L of every training sample, stored once, so that later epochs
+ * never run the backbone (Section IV-B, "Activation Cache for Parallel
+ * Adapters"; Section V-B, data-parallel fine-tuning of the adapters alone).
+ *
+ * Model (Section IV-A, "Parallel Adapters Architecture"), per token row, with
+ * h_l the cached state of layer l (l = 1..L), adapter width r, a_0 = 0:
+ *     u_l = h_l W_down^l                       down-projection, W_down^l in R^{d x r}
+ *     z_l = lambda_l u_l + (1 - lambda_l) a_{l-1}     learnable scalar mix, lambda init 0.5
+ *     a_l = phi(z_l)                           adapter body (ReLU or identity)
+ *     y   = h_L + a_L W_up                     up-projection, summed with the backbone output
+ * Heads: PAC_HEAD_MEANPOOL_CLS  logits = mean_s(y) W_head + b_head, loss = mean softmax
+ * cross-entropy over the batch (head is trainable); PAC_HEAD_FROZEN_LM  logits = y W_lm^T
+ * with a borrowed, frozen W_lm, loss = mean cross-entropy over all B*S positions.
+ * Gradients reach the adapter parameters only; nothing is ever written toward the cache.
+ *
+ * Conventions
+ *  - Every pointer argument says "host" or "device".  Device pointers are plain
+ *    CUDA device addresses on the context's device.
+ *  - Borrowed memory (cache, labels, LM head) must outlive the context and is never
+ *    written.  Parameters, gradients, optimizer moments and scratch are owned by the
+ *    context (allocated in pac_adapter_init, freed in pac_destroy).
+ *  - Flat parameter layout (fp32), used by every get/set call:
+ *        W_down[L][d][r] | lambda[L] | W_up[r][d] | W_head[d][C] | b_head[C]
+ *    (the last two only with PAC_HEAD_MEANPOOL_CLS).
+ *  - Every call returns a pac_status and never throws or aborts.  Arguments are
+ *    checked on the host before any launch; on error no device state changes.
+ *    pac_last_error() gives a message for the most recent failure on a context.
+ *  - A context is not thread-safe.  All work is enqueued on the context's stream.
+ *  - There is no CPU fallback: without a usable CUDA device pac_create fails.
+ */
+#ifndef PAC_H
+#define PAC_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pac_ctx pac_ctx;
+
+typedef enum {
+    PAC_OK = 0,
+    PAC_ERR_INVALID_ARG = 1,      /* null pointer, non-positive size, bad enum */
+    PAC_ERR_BAD_STATE = 2,        /* call order: create -> cache_register -> adapter_init -> ... */
+    PAC_ERR_SAMPLE_ID_RANGE = 3,  /* a sample id outside [0, N) */
+    PAC_ERR_UNSUPPORTED = 4,      /* shape/dtype combination the kernels do not cover */
+    PAC_ERR_NOMEM = 5,            /* device or pinned-host allocation failed */
+    PAC_ERR_CUDA = 6,             /* a CUDA runtime/driver call failed */
+    PAC_ERR_TIMEOUT = 7           /* a bounded device-side wait ran out */
+} pac_status;
+
+typedef enum { PAC_F32 = 0, PAC_BF16 = 1 } pac_dtype;
+typedef enum { PAC_ACT_RELU = 0, PAC_ACT_IDENTITY = 1 } pac_act;
+typedef enum { PAC_HEAD_MEANPOOL_CLS = 0, PAC_HEAD_FROZEN_LM = 1 } pac_head;
+
+typedef struct {
+    int r;               /* adapter width (the paper's d / reduction factor) */
+    int act;             /* pac_act */
+    int head;            /* pac_head */
+    int n_out;           /* classes C, or vocabulary size V for the LM head */
+    float lambda_init;   /* 0.5 in the paper */
+    int max_batch;       /* largest B any later call will pass */
+    const void* lm_head; /* device, [V][d] bf16, borrowed, frozen; NULL for the classifier head */
+} pac_adapter_cfg;
+
+typedef struct { float lr, beta1, beta2, eps, weight_decay; } pac_adamw;
+
+/* Options for pac_set_option. */
+typedef enum {
+    PAC_OPT_KERNEL_PATH = 0   /* 0 = automatic (tensor-core path when the shape allows),
+                                 1 = force the plain fp32-FMA kernels */
+} pac_option;
+
+/* Creates a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t to
+ * enqueue all work on, or NULL for a stream the context creates and owns. */
+pac_status pac_create(pac_ctx** out, int device, void* cuda_stream);
+pac_status pac_destroy(pac_ctx* ctx);
+
+/* Registers the activation cache (Section IV-B): dev_cache is a device array
+ * [N][L][S][d] of `dtype`, row-major, 16-byte aligned, borrowed and read-only.
+ * dev_labels is a device int32 array [N] (labels_per_sample = 1, classifier) or
+ * [N][S] (labels_per_sample = S, LM targets), borrowed and read-only.
+ * Re-registering is allowed before pac_adapter_init only. */
+pac_status pac_cache_register(pac_ctx* ctx, const void* dev_cache, int dtype, long long N, int L, int S, int d,
+                              const int* dev_labels, int labels_per_sample);
+
+/* Allocates parameters, gradients, AdamW moments and scratch for batches up to
+ * cfg->max_batch and fills the parameters from `seed`:
+ * W_down ~ N(0, 1/d), lambda = lambda_init, W_up = 0, W_head ~ N(0, 1/d), b_head = 0
+ * (zero up-projection so the initial model equals backbone + head, the rationale of
+ * Section IV-C).  Element i of the flat vector is a function of (seed, i) only.
+ * For the classifier head this call also reads the last cached layer of every sample
+ * once to store its token mean (a per-sample constant of the frozen backbone). */
+pac_status pac_adapter_init(pac_ctx* ctx, const pac_adapter_cfg* cfg, unsigned long long seed);
+
+/* One minibatch: gather cached states of sample_ids (host, B ints, duplicates allowed),
+ * adapter forward, loss, adapter backward.  Overwrites the gradients; does not change
+ * parameters.  If loss_out (host) is non-NULL the call waits for the stream and stores
+ * the mean loss; if NULL the call returns as soon as the work is enqueued. */
+pac_status pac_train_step(pac_ctx* ctx, const int* sample_ids, int B, float* loss_out);
+
+/* AdamW on the adapter parameters (and the classifier head) from the current gradients:
+ * decoupled decay on W_down, W_up, W_head; none on lambda and b_head; bias-corrected
+ * moments; step counter advances by one. */
+pac_status pac_adam_step(pac_ctx* ctx, const pac_adamw* hp);
+
+/* Forward only.  dev_out (device, fp32): [B][C] for the classifier head, [B][S][V] for
+ * the LM head.  sample_ids is a host array. */
+pac_status pac_eval_logits(pac_ctx* ctx, const int* sample_ids, int B, float* dev_out);
+
+/* Cache gather alone: dev_out (device, cache dtype) [L][B][S][d] with
+ * dev_out[l][b] = cache[sample_ids[b]][l], bit for bit.  sample_ids is a host array. */
+pac_status pac_gather(pac_ctx* ctx, const int* sample_ids, int B, void* dev_out);
+
+/* Runs train_step + adam_step for every consecutive B-slice of perm (host, n ids,
+ * n a multiple of B) with one wait at the end.  losses_out (host, n/B floats) may be NULL. */
+pac_status pac_train_epoch(pac_ctx* ctx, const int* perm, long long n, int B, const pac_adamw* hp,
+                           float* losses_out);
+
+/* The same with ids and losses resident on the device: dev_perm (device int32, n ids,
+ * validated on the device: an out-of-range id is clamped into range, counted, and reported
+ * as PAC_ERR_SAMPLE_ID_RANGE by the next pac_sync), dev_losses (device fp32, n/B, may be
+ * NULL).  Returns without waiting. */
+pac_status pac_train_epoch_dev(pac_ctx* ctx, const int* dev_perm, long long n, int B, const pac_adamw* hp,
+                               float* dev_losses);
+
+/* Checkpointing and inspection (host buffers of pac_param_count floats). */
+pac_status pac_param_count(pac_ctx* ctx, long long* n);
+pac_status pac_get_params(pac_ctx* ctx, float* host);
+pac_status pac_set_params(pac_ctx* ctx, const float* host);
+pac_status pac_get_grads(pac_ctx* ctx, float* host);
+pac_status pac_get_opt_state(pac_ctx* ctx, float* m, float* v, long long* step);
+pac_status pac_set_opt_state(pac_ctx* ctx, const float* m, const float* v, long long step);
+
+pac_status pac_set_option(pac_ctx* ctx, int option, int value);
+/* Number of kernels this context has launched so far. */
+pac_status pac_launch_count(pac_ctx* ctx, long long* n);
+/* Waits for the context's stream; reports device-side status words (bounded waits that
+ * ran out, ids clamped by pac_train_epoch_dev). */
+pac_status pac_sync(pac_ctx* ctx);
+const char* pac_last_error(const pac_ctx* ctx);
+/* "tensor" or "simt": which kernels the next train step will use (valid after adapter_init). */
+const char* pac_kernel_path(const pac_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PAC_H */

@@ -1,0 +1,243 @@
+"""ctypes binding of the C ABI in include/pac.h: argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  There is no CPU
+fallback: if libpac_b200.so is missing or no CUDA device is usable, loading or
+pac_create fails loudly.  torch is used only to own device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import dataclasses
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+PAC_F32, PAC_BF16 = 0, 1
+PAC_ACT_RELU, PAC_ACT_IDENTITY = 0, 1
+PAC_HEAD_MEANPOOL_CLS, PAC_HEAD_FROZEN_LM = 0, 1
+PAC_OPT_KERNEL_PATH = 0
+STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_SAMPLE_ID_RANGE",
+                "PAC_ERR_UNSUPPORTED", "PAC_ERR_NOMEM", "PAC_ERR_CUDA", "PAC_ERR_TIMEOUT"]
+
+# every symbol include/pac.h declares
+EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init", "pac_train_step",
+           "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
+           "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
+           "pac_set_opt_state", "pac_set_option", "pac_launch_count", "pac_sync", "pac_last_error",
+           "pac_kernel_path"]
+
+
+class PacError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        self.status = status
+        self.status_name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{self.status_name}: {message}")
+
+
+class _AdapterCfg(C.Structure):
+    _fields_ = [("r", C.c_int), ("act", C.c_int), ("head", C.c_int), ("n_out", C.c_int),
+                ("lambda_init", C.c_float), ("max_batch", C.c_int), ("lm_head", C.c_void_p)]
+
+
+class _AdamW(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float)]
+
+
+@dataclasses.dataclass
+class AdamW:
+    lr: float = 1e-3
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 0.01
+
+    def _c(self) -> _AdamW:
+        return _AdamW(self.lr, self.beta1, self.beta2, self.eps, self.weight_decay)
+
+
+_LIB: Optional[C.CDLL] = None
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpac_b200.so")
+
+
+def load_library() -> C.CDLL:
+    """Loads libpac_b200.so (built by `python -m paper_2408_10746_b200.build`)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with `python -m paper_2408_10746_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = C.CDLL(path)
+    P, I, LL, F = C.c_void_p, C.c_int, C.c_longlong, C.c_float
+    sig = {
+        "pac_create": [C.POINTER(P), I, P], "pac_destroy": [P],
+        "pac_cache_register": [P, P, I, LL, I, I, I, P, I],
+        "pac_adapter_init": [P, C.POINTER(_AdapterCfg), C.c_ulonglong],
+        "pac_train_step": [P, P, I, C.POINTER(F)], "pac_adam_step": [P, C.POINTER(_AdamW)],
+        "pac_eval_logits": [P, P, I, P], "pac_gather": [P, P, I, P],
+        "pac_train_epoch": [P, P, LL, I, C.POINTER(_AdamW), P],
+        "pac_train_epoch_dev": [P, P, LL, I, C.POINTER(_AdamW), P],
+        "pac_param_count": [P, C.POINTER(LL)], "pac_get_params": [P, P], "pac_set_params": [P, P],
+        "pac_get_grads": [P, P], "pac_get_opt_state": [P, P, P, C.POINTER(LL)],
+        "pac_set_opt_state": [P, P, P, LL], "pac_set_option": [P, I, I],
+        "pac_launch_count": [P, C.POINTER(LL)], "pac_sync": [P],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = I
+    lib.pac_last_error.argtypes = [P]
+    lib.pac_last_error.restype = C.c_char_p
+    lib.pac_kernel_path.argtypes = [P]
+    lib.pac_kernel_path.restype = C.c_char_p
+    _LIB = lib
+    return lib
+
+
+def _ids(ids: Sequence[int]) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(ids, dtype=np.int32).reshape(-1))
+
+
+def _ptr(t) -> int:
+    """Device (torch tensor) or host (numpy array) address."""
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+class PacContext:
+    """One trainer context on one GPU.  Methods mirror the C calls one to one."""
+
+    def __init__(self, device: int = 0, stream: Optional[int] = None):
+        self._lib = load_library()
+        h = C.c_void_p()
+        st = self._lib.pac_create(C.byref(h), device, C.c_void_p(stream) if stream else None)
+        if st != 0:
+            raise PacError(st, "pac_create failed (is a CUDA device visible? there is no CPU fallback)")
+        self._h = h
+        self._keep = []          # borrowed tensors must outlive the context
+
+    def _ck(self, st: int):
+        if st != 0:
+            raise PacError(st, self._lib.pac_last_error(self._h).decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.pac_destroy(self._h)
+            self._h = None
+            self._keep = []
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    # -- the calls -----------------------------------------------------------
+    def cache_register(self, cache, labels):
+        """cache: CUDA tensor [N][L][S][d] (float32 or bfloat16); labels: CUDA int32 [N] or [N][S]."""
+        import torch
+        assert cache.is_cuda and labels.is_cuda and cache.is_contiguous() and labels.is_contiguous()
+        assert labels.dtype == torch.int32
+        N, L, S, d = cache.shape
+        dt = {torch.float32: PAC_F32, torch.bfloat16: PAC_BF16}[cache.dtype]
+        per = 1 if labels.dim() == 1 else labels.shape[1]
+        self._ck(self._lib.pac_cache_register(self._h, cache.data_ptr(), dt, N, L, S, d, labels.data_ptr(), per))
+        self._keep += [cache, labels]
+        self.shape = (N, L, S, d)
+        self.cache_dtype = cache.dtype
+
+    def adapter_init(self, r: int, n_out: int, max_batch: int, act: int = PAC_ACT_RELU,
+                     head: int = PAC_HEAD_MEANPOOL_CLS, lambda_init: float = 0.5, lm_head=None, seed: int = 1):
+        cfg = _AdapterCfg(r, act, head, n_out, lambda_init, max_batch, lm_head.data_ptr() if lm_head is not None else None)
+        self._ck(self._lib.pac_adapter_init(self._h, C.byref(cfg), seed))
+        if lm_head is not None:
+            self._keep.append(lm_head)
+        self.r, self.n_out, self.head = r, n_out, head
+
+    def set_option(self, option: int, value: int):
+        self._ck(self._lib.pac_set_option(self._h, option, value))
+
+    def train_step(self, sample_ids, want_loss: bool = True) -> Optional[float]:
+        ids = _ids(sample_ids)
+        loss = C.c_float()
+        self._ck(self._lib.pac_train_step(self._h, ids.ctypes.data, ids.size, C.byref(loss) if want_loss else None))
+        return loss.value if want_loss else None
+
+    def adam_step(self, hp: AdamW):
+        self._ck(self._lib.pac_adam_step(self._h, C.byref(hp._c())))
+
+    def eval_logits(self, sample_ids, out):
+        ids = _ids(sample_ids)
+        self._ck(self._lib.pac_eval_logits(self._h, ids.ctypes.data, ids.size, out.data_ptr()))
+        return out
+
+    def gather(self, sample_ids, out):
+        ids = _ids(sample_ids)
+        self._ck(self._lib.pac_gather(self._h, ids.ctypes.data, ids.size, out.data_ptr()))
+        return out
+
+    def train_epoch(self, perm, B: int, hp: AdamW, want_losses: bool = True) -> Optional[np.ndarray]:
+        ids = _ids(perm)
+        losses = np.empty(max(1, ids.size // max(B, 1)), dtype=np.float32) if want_losses else None
+        self._ck(self._lib.pac_train_epoch(self._h, ids.ctypes.data, ids.size, B, C.byref(hp._c()),
+                                           losses.ctypes.data if want_losses else None))
+        return losses
+
+    def train_epoch_dev(self, dev_perm, B: int, hp: AdamW, dev_losses=None):
+        self._ck(self._lib.pac_train_epoch_dev(self._h, dev_perm.data_ptr(), dev_perm.numel(), B, C.byref(hp._c()),
+                                               dev_losses.data_ptr() if dev_losses is not None else None))
+
+    def param_count(self) -> int:
+        n = C.c_longlong()
+        self._ck(self._lib.pac_param_count(self._h, C.byref(n)))
+        return n.value
+
+    def get_params(self) -> np.ndarray:
+        out = np.empty(self.param_count(), dtype=np.float32)
+        self._ck(self._lib.pac_get_params(self._h, out.ctypes.data))
+        return out
+
+    def set_params(self, flat: np.ndarray):
+        flat = np.ascontiguousarray(flat, dtype=np.float32)
+        assert flat.size == self.param_count()
+        self._ck(self._lib.pac_set_params(self._h, flat.ctypes.data))
+
+    def get_grads(self) -> np.ndarray:
+        out = np.empty(self.param_count(), dtype=np.float32)
+        self._ck(self._lib.pac_get_grads(self._h, out.ctypes.data))
+        return out
+
+    def get_opt_state(self):
+        n = self.param_count()
+        m, v, step = np.empty(n, np.float32), np.empty(n, np.float32), C.c_longlong()
+        self._ck(self._lib.pac_get_opt_state(self._h, m.ctypes.data, v.ctypes.data, C.byref(step)))
+        return m, v, step.value
+
+    def set_opt_state(self, m: np.ndarray, v: np.ndarray, step: int):
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        v = np.ascontiguousarray(v, dtype=np.float32)
+        self._ck(self._lib.pac_set_opt_state(self._h, m.ctypes.data, v.ctypes.data, step))
+
+    def launch_count(self) -> int:
+        n = C.c_longlong()
+        self._ck(self._lib.pac_launch_count(self._h, C.byref(n)))
+        return n.value
+
+    def sync(self):
+        self._ck(self._lib.pac_sync(self._h))
+
+    def kernel_path(self) -> str:
+        return self._lib.pac_kernel_path(self._h).decode()

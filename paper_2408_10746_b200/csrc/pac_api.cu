@@ -1,0 +1,712 @@
+// Host runtime and C ABI of the adapter-over-cache trainer (declarations: include/pac.h).
+#include <cmath>
+#include <cstdarg>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "pac_common.cuh"
+#include "pac_simt.cuh"
+#include "pac_tensor.cuh"
+
+using namespace pac;
+
+namespace {
+
+constexpr int STAGE_SLOTS = 8;
+
+struct Scratch {
+    // per-step state, sized for max_batch
+    int* ids = nullptr;            // [max_batch] device copy of the current ids
+    float* u = nullptr;            // [L][M][r] down-projections
+    float* a = nullptr;            // [L][M][r] adapter states
+    float* du = nullptr;           // [L][M][r] fp32 (plain path)
+    bf16* du16 = nullptr;          // [L][M][r] bf16 (tensor path)
+    float* lam_part = nullptr;     // [L][blocks]
+    float* loss = nullptr;         // [1]
+    // classifier head
+    float* hbar = nullptr;         // [N][d] token mean of the last cached layer
+    float* pooled_a = nullptr;     // [B][r]
+    float* pooled_y = nullptr;     // [B][d]
+    float* logits = nullptr;       // [B][C]
+    float* dlogits = nullptr;      // [B][C]
+    float* loss_b = nullptr;       // [B] (classifier) or [M] (LM rows)
+    float* gvec = nullptr;         // [B][d]
+    float* daL = nullptr;          // [B][r] (classifier) or [M][r] (LM)
+    // LM head
+    float* y = nullptr;            // [M][d]
+    float* lm_logits = nullptr;    // [M][V]
+    float* dy = nullptr;           // [M][d]
+    // tensor path
+    bf16* wdT = nullptr;           // [L][r][d] bf16 shadow of W_down, transposed
+    float* dw_part = nullptr;      // split partials of dW_down
+};
+
+}  // namespace
+
+struct pac_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    bool own_stream = false;
+    // cache
+    const void* cache = nullptr;
+    int dtype = PAC_F32;
+    Dims dm{};
+    const int* labels = nullptr;
+    int labels_per_sample = 0;
+    bool registered = false;
+    // adapters
+    bool inited = false;
+    pac_adapter_cfg cfg{};
+    ParamLayout lay{};
+    float *params = nullptr, *grads = nullptr, *m = nullptr, *v = nullptr;
+    long long step = 0;
+    int max_rows = 0;              // max_batch * S
+    int chain_blocks_max = 0;
+    Scratch sc;
+    unsigned* status = nullptr;    // device status words
+    // host staging (pinned)
+    int* h_ids = nullptr;          // [STAGE_SLOTS][max_batch]
+    cudaEvent_t slot_ev[STAGE_SLOTS] = {};
+    int slot = 0;
+    float* h_loss = nullptr;
+    unsigned* h_status = nullptr;
+    // epoch buffers
+    int* d_perm = nullptr; long long perm_cap = 0;
+    float* d_losses = nullptr; long long losses_cap = 0;
+    // options / bookkeeping
+    int force_simt = 0;
+    bool tensor_ok = false;
+    long long launches = 0;
+    TensorPlan tplan{};
+    std::string err;
+};
+
+namespace {
+
+pac_status fail(pac_ctx* c, pac_status s, const char* fmt, ...) {
+    if (c) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        c->err = buf;
+    }
+    return s;
+}
+
+#define CU_OK(c, call)                                                                              \
+    do {                                                                                            \
+        cudaError_t e_ = (call);                                                                    \
+        if (e_ != cudaSuccess)                                                                      \
+            return fail(c, e_ == cudaErrorMemoryAllocation ? PAC_ERR_NOMEM : PAC_ERR_CUDA,          \
+                        "%s failed: %s", #call, cudaGetErrorString(e_));                            \
+    } while (0)
+
+#define LAUNCH_CHECK(c)                                                                             \
+    do {                                                                                            \
+        (c)->launches++;                                                                            \
+        cudaError_t e_ = cudaGetLastError();                                                        \
+        if (e_ != cudaSuccess) return fail(c, PAC_ERR_CUDA, "kernel launch failed: %s (%s:%d)",     \
+                                           cudaGetErrorString(e_), __FILE__, __LINE__);             \
+    } while (0)
+
+template <typename T>
+pac_status dmalloc(pac_ctx* c, T** p, long long n) {
+    if (n <= 0) n = 1;
+    CU_OK(c, cudaMalloc((void**)p, (size_t)n * sizeof(T)));
+    return PAC_OK;
+}
+
+bool use_tensor(const pac_ctx* c) { return c->tensor_ok && !c->force_simt; }
+
+inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
+
+// ---- counter-based initial parameters (splitmix64 output function on a keyed counter;
+// twelve 16-bit fields per element summed to a centred Irwin-Hall(12) value) ----
+const unsigned long long GOLD = 0x9E3779B97F4A7C15ull;
+unsigned long long mix64(unsigned long long x) {
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+float unit_normal(unsigned long long key, unsigned long long idx) {
+    long long total = 0;
+    for (int j = 0; j < 3; ++j) {
+        unsigned long long w = mix64((idx * 3 + j) * GOLD + key);
+        total += (long long)(w & 0xFFFF) + (long long)((w >> 16) & 0xFFFF) + (long long)((w >> 32) & 0xFFFF) +
+                 (long long)(w >> 48);
+    }
+    return (float)(total - 6 * 65535) * 0x1p-16f;
+}
+
+void fill_initial_params(const pac_ctx* c, unsigned long long seed, std::vector<float>& out) {
+    const int TAG_PARAM = 4;
+    unsigned long long key = mix64(mix64(seed) ^ ((unsigned long long)TAG_PARAM * GOLD));
+    const ParamLayout& lay = c->lay;
+    out.assign((size_t)lay.total, 0.f);
+    const float inv = (float)(1.0 / std::sqrt((double)c->dm.d));
+    for (long long i = 0; i < lay.lam; ++i) out[i] = unit_normal(key, (unsigned long long)i) * inv;
+    for (long long i = lay.lam; i < lay.w_up; ++i) out[i] = c->cfg.lambda_init;
+    for (long long i = lay.w_head; i < lay.b_head; ++i) out[i] = unit_normal(key, (unsigned long long)i) * inv;
+}
+
+// ---- staging of host ids ----
+pac_status stage_ids(pac_ctx* c, const int* ids, int B, const char* who) {
+    if (!ids) return fail(c, PAC_ERR_INVALID_ARG, "%s: sample_ids is NULL", who);
+    if (B < 1 || B > c->cfg.max_batch)
+        return fail(c, PAC_ERR_INVALID_ARG, "%s: B=%d outside [1, max_batch=%d]", who, B, c->cfg.max_batch);
+    for (int b = 0; b < B; ++b)
+        if (ids[b] < 0 || ids[b] >= c->dm.N)
+            return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "%s: sample_ids[%d]=%d outside [0, %lld)", who, b, ids[b], c->dm.N);
+    int s = c->slot;
+    c->slot = (c->slot + 1) % STAGE_SLOTS;
+    CU_OK(c, cudaEventSynchronize(c->slot_ev[s]));
+    int* h = c->h_ids + (size_t)s * c->cfg.max_batch;
+    std::memcpy(h, ids, sizeof(int) * B);
+    CU_OK(c, cudaMemcpyAsync(c->sc.ids, h, sizeof(int) * B, cudaMemcpyHostToDevice, c->stream));
+    CU_OK(c, cudaEventRecord(c->slot_ev[s], c->stream));
+    return PAC_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Forward: u_l for every layer, the chain, and the head.  ids are on the device.
+// ---------------------------------------------------------------------------
+template <typename T>
+pac_status down_projection_simt(pac_ctx* c, const int* d_ids, int B) {
+    const Dims& dm = c->dm;
+    const int M = B * dm.S;
+    CacheRows<T> A{(const T*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, 0};
+    MatB_RowMajor Bm{{c->params + c->lay.w_down, (long long)dm.d * dm.r, dm.r}};
+    StoreRowMajor E{c->sc.u, (long long)M * dm.r, dm.r};
+    dim3 grid(cdiv(dm.r, SG_BN), cdiv(M, SG_BM), dm.L);
+    gemm_simt<<<grid, 256, 0, c->stream>>>(M, dm.r, dm.d, A, Bm, E);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    const Dims& dm = c->dm;
+    const int M = B * dm.S;
+    const long long stride = (long long)M * dm.r;
+    Scratch& sc = c->sc;
+    pac_status st;
+    if (use_tensor(c)) {
+        st = tensor_down_projection(c->tplan, c->stream, d_ids, B, sc.u, c->status, &c->launches);
+        if (st != PAC_OK) return fail(c, st, "tensor-core down-projection launch failed: %s", tensor_last_error());
+    } else {
+        st = c->dtype == PAC_F32 ? down_projection_simt<float>(c, d_ids, B) : down_projection_simt<bf16>(c, d_ids, B);
+        if (st != PAC_OK) return st;
+    }
+    const float* lam = c->params + c->lay.lam;
+    if (c->cfg.act == PAC_ACT_RELU)
+        chain_fwd_kernel<PAC_ACT_RELU><<<cdiv(stride, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, stride);
+    else
+        chain_fwd_kernel<PAC_ACT_IDENTITY><<<cdiv(stride, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, stride);
+    LAUNCH_CHECK(c);
+    const float* aL = sc.a + (long long)(dm.L - 1) * stride;
+    const float* W_up = c->params + c->lay.w_up;
+    if (c->cfg.head == PAC_HEAD_MEANPOOL_CLS) {
+        pool_tokens_kernel<<<B, 128, 0, c->stream>>>(aL, sc.pooled_a, dm.S, dm.r);
+        LAUNCH_CHECK(c);
+        size_t smem = sizeof(float) * (dm.d + dm.C + 32);
+        cls_head_kernel<<<B, 256, smem, c->stream>>>(sc.hbar, d_ids, dm.N, c->labels, sc.pooled_a, W_up,
+                                                     c->params + c->lay.w_head, c->params + c->lay.b_head, B, dm.S,
+                                                     dm.d, dm.r, dm.C, train ? 1 : 0, sc.pooled_y,
+                                                     train ? sc.logits : d_logits_out, sc.loss_b, sc.dlogits,
+                                                     sc.gvec, sc.daL, c->status);
+        LAUNCH_CHECK(c);
+    } else {
+        // y = h_L + a_L W_up
+        dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
+        MatA_RowMajor Aa{{aL, 0, dm.r}};
+        MatB_RowMajor Bu{{W_up, 0, dm.d}};
+        if (c->dtype == PAC_F32) {
+            StorePlusLastLayer<float> E{sc.y, dm.d, CacheRows<float>{(const float*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, dm.L - 1}};
+            gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.r, Aa, Bu, E);
+        } else {
+            StorePlusLastLayer<bf16> E{sc.y, dm.d, CacheRows<bf16>{(const bf16*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, dm.L - 1}};
+            gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.r, Aa, Bu, E);
+        }
+        LAUNCH_CHECK(c);
+        // logits = y W_lm^T
+        float* lg = train ? sc.lm_logits : d_logits_out;
+        dim3 g2(cdiv(dm.C, SG_BN), cdiv(M, SG_BM), 1);
+        MatA_RowMajor Ay{{sc.y, 0, dm.d}};
+        MatB_Bf16Rows Bw{(const bf16*)c->cfg.lm_head, dm.d};
+        StoreRowMajor El{lg, 0, dm.C};
+        gemm_simt<<<g2, 256, 0, c->stream>>>(M, dm.C, dm.d, Ay, Bw, El);
+        LAUNCH_CHECK(c);
+        if (train) {
+            lm_ce_kernel<<<M, 256, 0, c->stream>>>(lg, d_ids, dm.N, c->labels, dm.S, dm.C, M, 1, sc.loss_b, c->status);
+            LAUNCH_CHECK(c);
+        }
+    }
+    return PAC_OK;
+}
+
+template <typename T>
+pac_status dw_down_simt(pac_ctx* c, const int* d_ids, int B) {
+    const Dims& dm = c->dm;
+    const int M = B * dm.S;
+    CacheRowsT<T> A{(const T*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d};
+    MatB_RowMajor Bm{{c->sc.du, (long long)M * dm.r, dm.r}};
+    StoreRowMajor E{c->grads + c->lay.w_down, (long long)dm.d * dm.r, dm.r};
+    dim3 grid(cdiv(dm.r, SG_BN), cdiv(dm.d, SG_BM), dm.L);
+    gemm_simt<<<grid, 256, 0, c->stream>>>(dm.d, dm.r, M, A, Bm, E);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+// Backward through the adapters only, after forward(train=true).  d_loss receives the mean loss.
+pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
+    const Dims& dm = c->dm;
+    const int M = B * dm.S;
+    const long long stride = (long long)M * dm.r;
+    Scratch& sc = c->sc;
+    const float* aL = sc.a + (long long)(dm.L - 1) * stride;
+    const float* W_up = c->params + c->lay.w_up;
+    int per_sample;
+    if (c->cfg.head == PAC_HEAD_MEANPOOL_CLS) {
+        long long n = (long long)dm.r * dm.d + (long long)dm.d * dm.C + dm.C + 1;
+        cls_grads_kernel<<<cdiv(n, 256), 256, 0, c->stream>>>(sc.pooled_a, sc.gvec, sc.pooled_y, sc.dlogits, sc.loss_b,
+                                                              B, dm.d, dm.r, dm.C, c->grads + c->lay.w_up,
+                                                              c->grads + c->lay.w_head, c->grads + c->lay.b_head, d_loss);
+        LAUNCH_CHECK(c);
+        per_sample = 1;
+    } else {
+        mean_kernel<<<1, 1024, 0, c->stream>>>(sc.loss_b, M, d_loss);
+        LAUNCH_CHECK(c);
+        // dy = dlogits W_lm   (the head is frozen: it receives no gradient)
+        dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
+        MatA_RowMajor Ad{{sc.lm_logits, 0, dm.C}};
+        MatB_Bf16Cols Bw{(const bf16*)c->cfg.lm_head, dm.d};
+        StoreRowMajor Ed{sc.dy, 0, dm.d};
+        gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.C, Ad, Bw, Ed);
+        LAUNCH_CHECK(c);
+        // dW_up = a_L^T dy
+        dim3 g2(cdiv(dm.d, SG_BN), cdiv(dm.r, SG_BM), 1);
+        MatA_ColMajor At{{aL, 0, dm.r}};
+        MatB_RowMajor Bd{{sc.dy, 0, dm.d}};
+        StoreRowMajor Eu{c->grads + c->lay.w_up, 0, dm.d};
+        gemm_simt<<<g2, 256, 0, c->stream>>>(dm.r, dm.d, M, At, Bd, Eu);
+        LAUNCH_CHECK(c);
+        // da_L = dy W_up^T
+        dim3 g3(cdiv(dm.r, SG_BN), cdiv(M, SG_BM), 1);
+        MatA_RowMajor Ady{{sc.dy, 0, dm.d}};
+        MatB_ColMajor But{{W_up, 0, dm.d}};
+        StoreRowMajor Ea{sc.daL, 0, dm.r};
+        gemm_simt<<<g3, 256, 0, c->stream>>>(M, dm.r, dm.d, Ady, But, Ea);
+        LAUNCH_CHECK(c);
+        per_sample = 0;
+    }
+    const float* lam = c->params + c->lay.lam;
+    const unsigned blocks = cdiv(stride, 256);
+    const bool tens = use_tensor(c);
+#define CHAIN_BWD(ACT, DUT, DUP)                                                                              \
+    chain_bwd_kernel<ACT, DUT><<<blocks, 256, 0, c->stream>>>(sc.u, sc.a, lam, sc.daL, per_sample, dm.S, dm.r, \
+                                                              dm.L, stride, DUP, sc.lam_part)
+    if (c->cfg.act == PAC_ACT_RELU) {
+        if (tens) CHAIN_BWD(PAC_ACT_RELU, bf16, sc.du16); else CHAIN_BWD(PAC_ACT_RELU, float, sc.du);
+    } else {
+        if (tens) CHAIN_BWD(PAC_ACT_IDENTITY, bf16, sc.du16); else CHAIN_BWD(PAC_ACT_IDENTITY, float, sc.du);
+    }
+#undef CHAIN_BWD
+    LAUNCH_CHECK(c);
+    reduce_rows_kernel<<<dm.L, 256, 0, c->stream>>>(sc.lam_part, (int)blocks, c->grads + c->lay.lam);
+    LAUNCH_CHECK(c);
+    if (tens) {
+        pac_status st = tensor_dw_down(c->tplan, c->stream, d_ids, B, sc.du16, c->grads + c->lay.w_down, sc.dw_part,
+                                       c->status, &c->launches);
+        if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
+        return PAC_OK;
+    }
+    return c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
+}
+
+pac_status adam_enqueue(pac_ctx* c, const pac_adamw* hp) {
+    c->step += 1;
+    const float inv_bc1 = (float)(1.0 / (1.0 - std::pow((double)hp->beta1, (double)c->step)));
+    const float inv_bc2 = (float)(1.0 / (1.0 - std::pow((double)hp->beta2, (double)c->step)));
+    adamw_kernel<<<cdiv(c->lay.total, 256), 256, 0, c->stream>>>(c->params, c->grads, c->m, c->v, c->lay.total, c->lay,
+                                                                 *hp, inv_bc1, inv_bc2, c->sc.wdT, c->dm.d, c->dm.r);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+pac_status check_hp(pac_ctx* c, const pac_adamw* hp) {
+    if (!hp) return fail(c, PAC_ERR_INVALID_ARG, "AdamW hyper-parameters are NULL");
+    if (!(hp->lr >= 0.f) || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f) ||
+        !(hp->eps > 0.f) || !(hp->weight_decay >= 0.f))
+        return fail(c, PAC_ERR_INVALID_ARG, "AdamW hyper-parameters out of range");
+    return PAC_OK;
+}
+
+pac_status refresh_shadow(pac_ctx* c) {
+    if (!c->sc.wdT) return PAC_OK;
+    long long n = (long long)c->dm.L * c->dm.d * c->dm.r;
+    shadow_wdown_kernel<<<cdiv(n, 256), 256, 0, c->stream>>>(c->params, c->sc.wdT, c->dm.L, c->dm.d, c->dm.r);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+void free_all(pac_ctx* c) {
+    Scratch& s = c->sc;
+    void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.wdT, s.dw_part, c->params, c->grads,
+                    c->m, c->v, c->status, c->d_perm, c->d_losses};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    if (c->h_ids) cudaFreeHost(c->h_ids);
+    if (c->h_loss) cudaFreeHost(c->h_loss);
+    if (c->h_status) cudaFreeHost(c->h_status);
+    for (auto& e : c->slot_ev)
+        if (e) cudaEventDestroy(e);
+    if (c->own_stream && c->stream) cudaStreamDestroy(c->stream);
+}
+
+#define NEED_CTX(c) do { if (!(c)) return PAC_ERR_INVALID_ARG; } while (0)
+#define NEED_INIT(c, who)                                                                          \
+    do {                                                                                           \
+        NEED_CTX(c);                                                                               \
+        if (!(c)->inited) return fail(c, PAC_ERR_BAD_STATE, "%s: call pac_adapter_init first", who); \
+        cudaError_t e_ = cudaSetDevice((c)->device);                                               \
+        if (e_ != cudaSuccess) return fail(c, PAC_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(e_)); \
+    } while (0)
+
+}  // namespace
+
+extern "C" {
+
+pac_status pac_create(pac_ctx** out, int device, void* cuda_stream) {
+    if (!out) return PAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) return PAC_ERR_CUDA;   // no CPU fallback
+    if (device < 0 || device >= count) return PAC_ERR_INVALID_ARG;
+    if (cudaSetDevice(device) != cudaSuccess) return PAC_ERR_CUDA;
+    pac_ctx* c = new (std::nothrow) pac_ctx();
+    if (!c) return PAC_ERR_NOMEM;
+    c->device = device;
+    if (cuda_stream) {
+        c->stream = (cudaStream_t)cuda_stream;
+    } else {
+        if (cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking) != cudaSuccess) { delete c; return PAC_ERR_CUDA; }
+        c->own_stream = true;
+    }
+    bool ok = cudaMalloc((void**)&c->status, sizeof(unsigned) * ST_WORDS) == cudaSuccess &&
+              cudaMemsetAsync(c->status, 0, sizeof(unsigned) * ST_WORDS, c->stream) == cudaSuccess &&
+              cudaMallocHost((void**)&c->h_loss, sizeof(float)) == cudaSuccess &&
+              cudaMallocHost((void**)&c->h_status, sizeof(unsigned) * ST_WORDS) == cudaSuccess;
+    for (auto& e : c->slot_ev) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { free_all(c); delete c; return PAC_ERR_CUDA; }
+    *out = c;
+    return PAC_OK;
+}
+
+pac_status pac_destroy(pac_ctx* c) {
+    NEED_CTX(c);
+    cudaSetDevice(c->device);
+    cudaStreamSynchronize(c->stream);
+    tensor_plan_destroy(c->tplan);
+    free_all(c);
+    delete c;
+    return PAC_OK;
+}
+
+pac_status pac_cache_register(pac_ctx* c, const void* dev_cache, int dtype, long long N, int L, int S, int d,
+                              const int* dev_labels, int labels_per_sample) {
+    NEED_CTX(c);
+    if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_cache_register: adapters already initialised");
+    if (!dev_cache || !dev_labels) return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register: NULL device pointer");
+    if (dtype != PAC_F32 && dtype != PAC_BF16) return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register: bad dtype %d", dtype);
+    if (N < 1 || L < 1 || S < 1 || d < 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register: sizes must be positive");
+    if (N > 0x7fffffffLL) return fail(c, PAC_ERR_UNSUPPORTED, "pac_cache_register: N beyond int32 sample ids");
+    if ((long long)L * S > 0x7fffffffLL / 4) return fail(c, PAC_ERR_UNSUPPORTED, "pac_cache_register: L*S too large");
+    if (labels_per_sample != 1 && labels_per_sample != S)
+        return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register: labels_per_sample must be 1 or S");
+    if (((uintptr_t)dev_cache & 15) != 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register: cache not 16-byte aligned");
+    c->cache = dev_cache; c->dtype = dtype;
+    c->dm.N = N; c->dm.L = L; c->dm.S = S; c->dm.d = d;
+    c->labels = dev_labels; c->labels_per_sample = labels_per_sample;
+    c->registered = true;
+    return PAC_OK;
+}
+
+pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned long long seed) {
+    NEED_CTX(c);
+    if (!c->registered) return fail(c, PAC_ERR_BAD_STATE, "pac_adapter_init: call pac_cache_register first");
+    if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_adapter_init: already initialised");
+    if (!cfg) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: cfg is NULL");
+    if (cfg->r < 1 || cfg->n_out < 1 || cfg->max_batch < 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: sizes must be positive");
+    if (cfg->act != PAC_ACT_RELU && cfg->act != PAC_ACT_IDENTITY) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: bad activation");
+    if (cfg->head != PAC_HEAD_MEANPOOL_CLS && cfg->head != PAC_HEAD_FROZEN_LM) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: bad head");
+    const bool cls = cfg->head == PAC_HEAD_MEANPOOL_CLS;
+    if (cls && c->labels_per_sample != 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: classifier head needs one label per sample");
+    if (!cls && c->labels_per_sample != c->dm.S) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: LM head needs S targets per sample");
+    if (!cls && !cfg->lm_head) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: LM head pointer is NULL");
+    if (cls && cfg->n_out > 4096) return fail(c, PAC_ERR_UNSUPPORTED, "pac_adapter_init: classifier head supports up to 4096 classes");
+    if ((long long)cfg->max_batch * c->dm.S > 0x7fffffffLL / 8) return fail(c, PAC_ERR_UNSUPPORTED, "pac_adapter_init: max_batch*S too large");
+    CU_OK(c, cudaSetDevice(c->device));
+    c->cfg = *cfg;
+    c->dm.r = cfg->r; c->dm.C = cfg->n_out;
+    const Dims& dm = c->dm;
+    c->lay = ParamLayout::make(dm.L, dm.d, dm.r, dm.C, cls);
+    c->max_rows = cfg->max_batch * dm.S;
+    const long long Mr = (long long)c->max_rows * dm.r;
+    c->chain_blocks_max = (int)cdiv(Mr, 256);
+    Scratch& s = c->sc;
+    pac_status st = PAC_OK;
+    auto A = [&](pac_status x) { if (st == PAC_OK) st = x; };
+    A(dmalloc(c, &c->params, c->lay.total)); A(dmalloc(c, &c->grads, c->lay.total));
+    A(dmalloc(c, &c->m, c->lay.total)); A(dmalloc(c, &c->v, c->lay.total));
+    A(dmalloc(c, &s.ids, cfg->max_batch));
+    A(dmalloc(c, &s.u, Mr * dm.L)); A(dmalloc(c, &s.a, Mr * dm.L));
+    A(dmalloc(c, &s.lam_part, (long long)dm.L * c->chain_blocks_max));
+    A(dmalloc(c, &s.loss, 1));
+    if (cls) {
+        A(dmalloc(c, &s.hbar, dm.N * dm.d));
+        A(dmalloc(c, &s.pooled_a, (long long)cfg->max_batch * dm.r));
+        A(dmalloc(c, &s.pooled_y, (long long)cfg->max_batch * dm.d));
+        A(dmalloc(c, &s.logits, (long long)cfg->max_batch * dm.C));
+        A(dmalloc(c, &s.dlogits, (long long)cfg->max_batch * dm.C));
+        A(dmalloc(c, &s.loss_b, cfg->max_batch));
+        A(dmalloc(c, &s.gvec, (long long)cfg->max_batch * dm.d));
+        A(dmalloc(c, &s.daL, (long long)cfg->max_batch * dm.r));
+    } else {
+        A(dmalloc(c, &s.loss_b, c->max_rows));
+        A(dmalloc(c, &s.daL, Mr));
+        A(dmalloc(c, &s.y, (long long)c->max_rows * dm.d));
+        A(dmalloc(c, &s.lm_logits, (long long)c->max_rows * dm.C));
+        A(dmalloc(c, &s.dy, (long long)c->max_rows * dm.d));
+    }
+    if (st == PAC_OK && cudaMallocHost((void**)&c->h_ids, sizeof(int) * STAGE_SLOTS * cfg->max_batch) != cudaSuccess)
+        st = fail(c, PAC_ERR_NOMEM, "pinned id staging allocation failed");
+    // tensor-core path: bf16 cache with TMA/UMMA-compatible sizes
+    c->tensor_ok = false;
+    if (st == PAC_OK && c->dtype == PAC_BF16 && tensor_shape_supported(dm)) {
+        A(dmalloc(c, &s.wdT, (long long)dm.L * dm.r * dm.d));
+        A(dmalloc(c, &s.du16, Mr * dm.L));
+        long long part_floats = 0;
+        if (st == PAC_OK) {
+            pac_status ts = tensor_plan_create(c->tplan, c->device, (const bf16*)c->cache, dm, cfg->max_batch, s.wdT,
+                                               s.du16, &part_floats);
+            if (ts == PAC_OK) {
+                A(dmalloc(c, &s.dw_part, part_floats));
+                c->tensor_ok = (st == PAC_OK);
+            } else if (ts != PAC_ERR_UNSUPPORTED) {
+                st = fail(c, ts, "tensor path set-up failed: %s", tensor_last_error());
+            }
+        }
+    }
+    if (st == PAC_OK && !c->tensor_ok) A(dmalloc(c, &s.du, Mr * dm.L));
+    if (st != PAC_OK) return st;
+    CU_OK(c, cudaMemsetAsync(c->grads, 0, sizeof(float) * c->lay.total, c->stream));
+    CU_OK(c, cudaMemsetAsync(c->m, 0, sizeof(float) * c->lay.total, c->stream));
+    CU_OK(c, cudaMemsetAsync(c->v, 0, sizeof(float) * c->lay.total, c->stream));
+    std::vector<float> init;
+    fill_initial_params(c, seed, init);
+    CU_OK(c, cudaMemcpyAsync(c->params, init.data(), sizeof(float) * c->lay.total, cudaMemcpyHostToDevice, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    c->step = 0;
+    if ((st = refresh_shadow(c)) != PAC_OK) return st;
+    if (cls) {
+        if (c->dtype == PAC_F32)
+            pool_last_layer_kernel<float><<<(unsigned)dm.N, 256, 0, c->stream>>>((const float*)c->cache, s.hbar, dm.L, dm.S, dm.d);
+        else
+            pool_last_layer_kernel<bf16><<<(unsigned)dm.N, 256, 0, c->stream>>>((const bf16*)c->cache, s.hbar, dm.L, dm.S, dm.d);
+        LAUNCH_CHECK(c);
+    }
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    c->inited = true;
+    return PAC_OK;
+}
+
+pac_status pac_train_step(pac_ctx* c, const int* sample_ids, int B, float* loss_out) {
+    NEED_INIT(c, "pac_train_step");
+    pac_status st = stage_ids(c, sample_ids, B, "pac_train_step");
+    if (st != PAC_OK) return st;
+    if ((st = forward(c, c->sc.ids, B, true, nullptr)) != PAC_OK) return st;
+    if ((st = backward(c, c->sc.ids, B, c->sc.loss)) != PAC_OK) return st;
+    if (loss_out) {
+        CU_OK(c, cudaMemcpyAsync(c->h_loss, c->sc.loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+        CU_OK(c, cudaStreamSynchronize(c->stream));
+        *loss_out = *c->h_loss;
+    }
+    return PAC_OK;
+}
+
+pac_status pac_adam_step(pac_ctx* c, const pac_adamw* hp) {
+    NEED_INIT(c, "pac_adam_step");
+    pac_status st = check_hp(c, hp);
+    if (st != PAC_OK) return st;
+    return adam_enqueue(c, hp);
+}
+
+pac_status pac_eval_logits(pac_ctx* c, const int* sample_ids, int B, float* dev_out) {
+    NEED_INIT(c, "pac_eval_logits");
+    if (!dev_out) return fail(c, PAC_ERR_INVALID_ARG, "pac_eval_logits: dev_out is NULL");
+    pac_status st = stage_ids(c, sample_ids, B, "pac_eval_logits");
+    if (st != PAC_OK) return st;
+    return forward(c, c->sc.ids, B, false, dev_out);
+}
+
+pac_status pac_gather(pac_ctx* c, const int* sample_ids, int B, void* dev_out) {
+    NEED_INIT(c, "pac_gather");
+    if (!dev_out) return fail(c, PAC_ERR_INVALID_ARG, "pac_gather: dev_out is NULL");
+    pac_status st = stage_ids(c, sample_ids, B, "pac_gather");
+    if (st != PAC_OK) return st;
+    const Dims& dm = c->dm;
+    const long long slab = (long long)dm.S * dm.d * (c->dtype == PAC_F32 ? 4 : 2);
+    const int vec16 = (slab % 16 == 0) && (((uintptr_t)dev_out & 15) == 0);
+    unsigned chunks = (unsigned)std::min<long long>(64, std::max<long long>(1, slab / (16 * 256 * 4)));
+    dim3 grid((unsigned)(B * dm.L), chunks, 1);
+    gather_kernel<<<grid, 256, 0, c->stream>>>((const unsigned char*)c->cache, c->sc.ids, dm.N, dm.L, B, slab,
+                                               (unsigned char*)dev_out, vec16, c->status);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+static pac_status epoch_common(pac_ctx* c, const int* d_perm, long long n, int B, const pac_adamw* hp, float* d_losses) {
+    for (long long s = 0; s < n / B; ++s) {
+        const int* ids = d_perm + s * B;
+        pac_status st = forward(c, ids, B, true, nullptr);
+        if (st != PAC_OK) return st;
+        if ((st = backward(c, ids, B, d_losses ? d_losses + s : c->sc.loss)) != PAC_OK) return st;
+        if ((st = adam_enqueue(c, hp)) != PAC_OK) return st;
+    }
+    return PAC_OK;
+}
+
+pac_status pac_train_epoch(pac_ctx* c, const int* perm, long long n, int B, const pac_adamw* hp, float* losses_out) {
+    NEED_INIT(c, "pac_train_epoch");
+    pac_status st = check_hp(c, hp);
+    if (st != PAC_OK) return st;
+    if (!perm) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch: perm is NULL");
+    if (B < 1 || B > c->cfg.max_batch) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch: B=%d outside [1, max_batch]", B);
+    if (n < B || n % B != 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch: n=%lld is not a positive multiple of B=%d", n, B);
+    for (long long i = 0; i < n; ++i)
+        if (perm[i] < 0 || perm[i] >= c->dm.N)
+            return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "pac_train_epoch: perm[%lld]=%d outside [0, %lld)", i, perm[i], c->dm.N);
+    if (n > c->perm_cap) {
+        CU_OK(c, cudaStreamSynchronize(c->stream));
+        if (c->d_perm) cudaFree(c->d_perm);
+        c->d_perm = nullptr; c->perm_cap = 0;
+        if ((st = dmalloc(c, &c->d_perm, n)) != PAC_OK) return st;
+        c->perm_cap = n;
+    }
+    if (n / B > c->losses_cap) {
+        CU_OK(c, cudaStreamSynchronize(c->stream));
+        if (c->d_losses) cudaFree(c->d_losses);
+        c->d_losses = nullptr; c->losses_cap = 0;
+        if ((st = dmalloc(c, &c->d_losses, n / B)) != PAC_OK) return st;
+        c->losses_cap = n / B;
+    }
+    // perm is pageable host memory: cudaMemcpyAsync stages it before returning
+    CU_OK(c, cudaMemcpyAsync(c->d_perm, perm, sizeof(int) * n, cudaMemcpyHostToDevice, c->stream));
+    if ((st = epoch_common(c, c->d_perm, n, B, hp, c->d_losses)) != PAC_OK) return st;
+    if (losses_out)
+        CU_OK(c, cudaMemcpyAsync(losses_out, c->d_losses, sizeof(float) * (n / B), cudaMemcpyDeviceToHost, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    return PAC_OK;
+}
+
+pac_status pac_train_epoch_dev(pac_ctx* c, const int* dev_perm, long long n, int B, const pac_adamw* hp, float* dev_losses) {
+    NEED_INIT(c, "pac_train_epoch_dev");
+    pac_status st = check_hp(c, hp);
+    if (st != PAC_OK) return st;
+    if (!dev_perm) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch_dev: dev_perm is NULL");
+    if (B < 1 || B > c->cfg.max_batch) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch_dev: B=%d outside [1, max_batch]", B);
+    if (n < B || n % B != 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch_dev: n=%lld is not a positive multiple of B=%d", n, B);
+    return epoch_common(c, dev_perm, n, B, hp, dev_losses);
+}
+
+pac_status pac_param_count(pac_ctx* c, long long* n) {
+    NEED_INIT(c, "pac_param_count");
+    if (!n) return fail(c, PAC_ERR_INVALID_ARG, "pac_param_count: n is NULL");
+    *n = c->lay.total;
+    return PAC_OK;
+}
+
+pac_status pac_get_params(pac_ctx* c, float* host) {
+    NEED_INIT(c, "pac_get_params");
+    if (!host) return fail(c, PAC_ERR_INVALID_ARG, "pac_get_params: host is NULL");
+    CU_OK(c, cudaMemcpyAsync(host, c->params, sizeof(float) * c->lay.total, cudaMemcpyDeviceToHost, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    return PAC_OK;
+}
+
+pac_status pac_set_params(pac_ctx* c, const float* host) {
+    NEED_INIT(c, "pac_set_params");
+    if (!host) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_params: host is NULL");
+    CU_OK(c, cudaMemcpyAsync(c->params, host, sizeof(float) * c->lay.total, cudaMemcpyHostToDevice, c->stream));
+    pac_status st = refresh_shadow(c);
+    if (st != PAC_OK) return st;
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    return PAC_OK;
+}
+
+pac_status pac_get_grads(pac_ctx* c, float* host) {
+    NEED_INIT(c, "pac_get_grads");
+    if (!host) return fail(c, PAC_ERR_INVALID_ARG, "pac_get_grads: host is NULL");
+    CU_OK(c, cudaMemcpyAsync(host, c->grads, sizeof(float) * c->lay.total, cudaMemcpyDeviceToHost, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    return PAC_OK;
+}
+
+pac_status pac_get_opt_state(pac_ctx* c, float* m, float* v, long long* step) {
+    NEED_INIT(c, "pac_get_opt_state");
+    if (!m || !v || !step) return fail(c, PAC_ERR_INVALID_ARG, "pac_get_opt_state: NULL argument");
+    CU_OK(c, cudaMemcpyAsync(m, c->m, sizeof(float) * c->lay.total, cudaMemcpyDeviceToHost, c->stream));
+    CU_OK(c, cudaMemcpyAsync(v, c->v, sizeof(float) * c->lay.total, cudaMemcpyDeviceToHost, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    *step = c->step;
+    return PAC_OK;
+}
+
+pac_status pac_set_opt_state(pac_ctx* c, const float* m, const float* v, long long step) {
+    NEED_INIT(c, "pac_set_opt_state");
+    if (!m || !v || step < 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_opt_state: bad argument");
+    CU_OK(c, cudaMemcpyAsync(c->m, m, sizeof(float) * c->lay.total, cudaMemcpyHostToDevice, c->stream));
+    CU_OK(c, cudaMemcpyAsync(c->v, v, sizeof(float) * c->lay.total, cudaMemcpyHostToDevice, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    c->step = step;
+    return PAC_OK;
+}
+
+pac_status pac_set_option(pac_ctx* c, int option, int value) {
+    NEED_CTX(c);
+    if (option == PAC_OPT_KERNEL_PATH) {
+        if (value != 0 && value != 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0 or 1");
+        if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_set_option: set the kernel path before pac_adapter_init");
+        c->force_simt = value;
+        return PAC_OK;
+    }
+    return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: unknown option %d", option);
+}
+
+pac_status pac_launch_count(pac_ctx* c, long long* n) {
+    NEED_CTX(c);
+    if (!n) return fail(c, PAC_ERR_INVALID_ARG, "pac_launch_count: n is NULL");
+    *n = c->launches;
+    return PAC_OK;
+}
+
+pac_status pac_sync(pac_ctx* c) {
+    NEED_CTX(c);
+    CU_OK(c, cudaSetDevice(c->device));
+    CU_OK(c, cudaMemcpyAsync(c->h_status, c->status, sizeof(unsigned) * ST_WORDS, cudaMemcpyDeviceToHost, c->stream));
+    CU_OK(c, cudaMemsetAsync(c->status, 0, sizeof(unsigned) * ST_WORDS, c->stream));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    if (c->h_status[ST_TIMEOUT]) return fail(c, PAC_ERR_TIMEOUT, "a bounded device-side wait ran out (%u)", c->h_status[ST_TIMEOUT]);
+    if (c->h_status[ST_CLAMPED_IDS])
+        return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "%u device-resident sample ids were outside [0, N) and were clamped", c->h_status[ST_CLAMPED_IDS]);
+    return PAC_OK;
+}
+
+const char* pac_last_error(const pac_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+const char* pac_kernel_path(const pac_ctx* c) { return (c && c->inited && use_tensor(c)) ? "tensor" : "simt"; }
+
+}  // extern "C"

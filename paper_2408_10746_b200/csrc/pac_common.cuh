@@ -1,0 +1,55 @@
+// Shared device helpers and the context structure of the adapter-over-cache trainer.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cstdint>
+#include <cstdio>
+#include <string>
+
+#include "pac.h"
+
+namespace pac {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(bf16 x) { return __bfloat162float(x); }
+
+// Device-side status words (one small array per context).
+enum { ST_CLAMPED_IDS = 0, ST_TIMEOUT = 1, ST_WORDS = 4 };
+
+// Sample id of batch row b, clamped into [0, N) so that no kernel can read outside
+// the cache even if a device-resident id is bad; clamps are counted.
+__device__ __forceinline__ long long safe_id(const int* __restrict__ ids, int b, long long N, unsigned* status) {
+    long long id = ids[b];
+    if (id < 0 || id >= N) {
+        if (status) atomicAdd(&status[ST_CLAMPED_IDS], 1u);
+        id = id < 0 ? 0 : N - 1;
+    }
+    return id;
+}
+
+struct Dims {
+    long long N;   // samples in the cache
+    int L, S, d;   // layers, tokens, hidden width
+    int r;         // adapter width
+    int C;         // classes or vocabulary
+};
+
+// Offsets of the flat fp32 parameter vector:
+// W_down[L][d][r] | lambda[L] | W_up[r][d] | W_head[d][C] | b_head[C]
+struct ParamLayout {
+    long long w_down, lam, w_up, w_head, b_head, total;
+    __host__ __device__ static ParamLayout make(int L, int d, int r, int C, bool cls) {
+        ParamLayout p;
+        p.w_down = 0;
+        p.lam = (long long)L * d * r;
+        p.w_up = p.lam + L;
+        p.w_head = p.w_up + (long long)r * d;
+        p.b_head = p.w_head + (cls ? (long long)d * C : 0);
+        p.total = p.b_head + (cls ? C : 0);
+        return p;
+    }
+};
+
+}  // namespace pac

@@ -1,0 +1,241 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same
+seeded inputs.  Tolerances: gather bit-exact; fp32 caches 1e-4 relative on the loss and
+on every gradient block; bf16 caches 2e-2 relative on the loss and 1e-2 relative L2 on
+the parameter vector after 10 steps."""
+import numpy as np
+import pytest
+import torch
+
+import pac_inputs as pi
+from oracle import pac_oracle as po
+from tests.common import Case, block_slices, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+TINY = pi.CONFIGS["tiny_fp32"]
+# ragged everything: S not a multiple of any tile, d and r odd-ish
+RAGGED_F32 = pi.CacheSpec("ragged_f32", N=24, L=3, S=19, d=100, dtype="f32", r=12, n_out=3, B=5)
+RAGGED_BF16 = pi.CacheSpec("ragged_bf16", N=24, L=3, S=19, d=100, dtype="bf16", r=12, n_out=3, B=5)
+SMALL_LM = pi.CacheSpec("small_lm", N=12, L=3, S=24, d=128, dtype="bf16", r=16, n_out=1000, B=4, head="lm")
+SMALL_LM_F32 = pi.CacheSpec("small_lm_f32", N=12, L=2, S=10, d=72, dtype="f32", r=8, n_out=300, B=3, head="lm")
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    return Case(TINY)
+
+
+# ------------------------------------------------------------------ gather
+@pytest.mark.parametrize("spec", [TINY, RAGGED_BF16, pi.CONFIGS["t5_base"].scaled(N=64)], ids=lambda s: s.name)
+def test_gather_bit_exact(spec):
+    case = Case(spec, materialize_cpu=False)
+    ctx = case.context(max_batch=16)
+    N = spec.N
+    rng = np.random.default_rng(0)
+    for ids in ([0], [N - 1], list(range(8)), list(range(N - 1, N - 9, -1)), [3, 3, 3, 0, N - 1, 3],
+                rng.integers(0, N, 16).tolist()):
+        out = torch.full((spec.L, len(ids), spec.S, spec.d), float("nan"), dtype=spec.torch_dtype, device="cuda")
+        ctx.gather(ids, out)
+        ctx.sync()
+        ref = pi.cache_samples(spec, 0, ids, "cpu").permute(1, 0, 2, 3).contiguous()   # [L][B][S][d]
+        assert out.cpu().view(torch.uint8).flatten().equal(ref.view(torch.uint8).flatten())
+        assert po.gather(ref.permute(1, 0, 2, 3).float().numpy(), range(len(ids))).shape[0] == len(ids)
+
+
+# ------------------------------------------------------------------ loss + gradients
+def check_loss_grads(case, ids, act, loss_tol, grad_tol, force_simt=False, seed=3):
+    spec = case.spec
+    ctx = case.context(max_batch=max(len(ids), spec.B), act=act, force_simt=force_simt)
+    flat = pi.random_params(spec, seed)
+    ctx.set_params(flat)
+    loss = ctx.train_step(ids)
+    g = ctx.get_grads()
+    ref_loss, ref_g, _ = case.oracle_loss_grads(flat, ids, act)
+    assert abs(loss - ref_loss) <= loss_tol * abs(ref_loss), (loss, ref_loss)
+    ref_flat = po.flatten(ref_g)
+    for name, sl in block_slices(spec).items():
+        err = rel_l2(g[sl], ref_flat[sl])
+        assert np.linalg.norm(ref_flat[sl]) > 0, name
+        assert err < grad_tol, f"{name}: rel L2 {err}"
+    return ctx
+
+
+@pytest.mark.parametrize("act", [0, 1])
+def test_tiny_fp32_loss_and_gradients(tiny, act):
+    ids = pi.epoch_permutation(TINY.N, 2)[:TINY.B].tolist()
+    check_loss_grads(tiny, ids, act, 1e-4, 1e-4)
+
+
+@pytest.mark.parametrize("spec", [RAGGED_F32, SMALL_LM_F32], ids=lambda s: s.name)
+def test_ragged_fp32_loss_and_gradients(spec):
+    case = Case(spec)
+    check_loss_grads(case, [5, 0, spec.N - 1, 5, 7][:spec.B], 0, 1e-4, 1e-4)
+    check_loss_grads(case, [2], 1, 1e-4, 1e-4)
+
+
+@pytest.mark.parametrize("spec", [RAGGED_BF16, SMALL_LM], ids=lambda s: s.name)
+def test_bf16_cache_plain_kernels_loss_and_gradients(spec):
+    """bf16 caches widen exactly to fp32, so the plain fp32-FMA kernels still meet the fp32 bound."""
+    case = Case(spec)
+    check_loss_grads(case, list(range(spec.B)), 0, 1e-4, 1e-4, force_simt=True)
+
+
+def test_duplicate_ids_and_single_sample(tiny):
+    check_loss_grads(tiny, [7, 7, 7, 7], 0, 1e-4, 1e-4)
+    check_loss_grads(tiny, [255], 0, 1e-4, 1e-4)
+
+
+# ------------------------------------------------------------------ eval
+@pytest.mark.parametrize("spec", [TINY, RAGGED_BF16, SMALL_LM], ids=lambda s: s.name)
+def test_eval_logits(spec):
+    case = Case(spec)
+    ctx = case.context(force_simt=True)
+    flat = pi.random_params(spec, 4)
+    ctx.set_params(flat)
+    ids = list(range(spec.B))
+    shape = (spec.B, spec.n_out) if spec.head == "cls" else (spec.B, spec.S, spec.n_out)
+    out = torch.zeros(shape, dtype=torch.float32, device="cuda")
+    ctx.eval_logits(ids, out)
+    ctx.sync()
+    ref = po.eval_logits(case.oracle_params(flat), case.H(ids), 0, case.lm_np)
+    assert rel_l2(out.cpu().numpy(), ref) < 1e-4
+
+
+def test_zero_up_projection_is_head_only(tiny):
+    """Freshly initialised adapters (W_up = 0) give the head-only logits and no gradient
+    toward W_down or lambda."""
+    ctx = tiny.context()
+    flat = ctx.get_params()
+    assert np.array_equal(flat, pi.init_params(TINY, 1))          # same counter-based law on both sides
+    ids = list(range(8))
+    out = torch.zeros((8, 2), dtype=torch.float32, device="cuda")
+    ctx.eval_logits(ids, out)
+    P = tiny.oracle_params(flat)
+    head_only = tiny.H(ids)[:, -1].mean(axis=1) @ P.W_head + P.b_head
+    assert rel_l2(out.cpu().numpy(), head_only) < 1e-5
+    ctx.train_step(ids)
+    g = ctx.get_grads()
+    sl = block_slices(TINY)
+    assert not g[sl["W_down"]].any() and not g[sl["lam"]].any() and g[sl["W_up"]].any()
+
+
+# ------------------------------------------------------------------ trajectories
+def run_trajectory(case, steps, act=0, force_simt=False, hp=None):
+    import paper_2408_10746_b200 as pac
+    spec = case.spec
+    hp = hp or po.AdamW()
+    ctx = case.context(act=act, force_simt=force_simt)
+    flat0 = ctx.get_params()
+    perm = pi.epoch_permutation(spec.N, 2)
+    batches = [perm[i * spec.B:(i + 1) * spec.B].tolist() for i in range(steps)]
+    tr, remap = case.oracle_trainer(flat0, act, hp, ids_universe=[i for b in batches for i in b])
+    losses, ref_losses = [], []
+    for ids in batches:
+        losses.append(ctx.train_step(ids))
+        ctx.adam_step(pac.AdamW(hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay))
+        ref_losses.append(tr.train_step([remap[i] for i in ids] if remap else ids))
+        tr.adam_step()
+    return ctx, np.array(losses), np.array(ref_losses), ctx.get_params(), po.flatten(tr.P), flat0
+
+
+def test_tiny_fp32_ten_adamw_steps(tiny):
+    ctx, losses, ref_losses, p, ref_p, p0 = run_trajectory(tiny, 10)
+    assert np.all(np.abs(losses - ref_losses) <= 1e-4 * np.abs(ref_losses))
+    assert rel_l2(p, ref_p) < 1e-4
+    assert rel_l2(p - p0, ref_p - p0) < 1e-2            # the update itself, not just the large initial values
+    m, v, step = ctx.get_opt_state()
+    assert step == 10
+
+
+def test_bf16_ten_steps_plain_kernels():
+    case = Case(RAGGED_BF16)
+    _, losses, ref_losses, p, ref_p, _ = run_trajectory(case, 4, force_simt=True)
+    assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses))
+    assert rel_l2(p, ref_p) < 1e-2
+
+
+# ------------------------------------------------------------------ runtime behaviour
+def test_epoch_equals_step_loop_and_is_deterministic(tiny):
+    import paper_2408_10746_b200 as pac
+    hp = pac.AdamW()
+    perm = pi.epoch_permutation(TINY.N, 2)[:10 * TINY.B]
+    a = tiny.context()
+    losses_a = a.train_epoch(perm, TINY.B, hp)
+    b = tiny.context()
+    losses_b = []
+    for i in range(10):
+        losses_b.append(b.train_step(perm[i * TINY.B:(i + 1) * TINY.B]))
+        b.adam_step(hp)
+    c = tiny.context()
+    dperm = torch.from_numpy(perm).cuda()
+    dl = torch.zeros(10, dtype=torch.float32, device="cuda")
+    c.train_epoch_dev(dperm, TINY.B, hp, dl)
+    c.sync()
+    assert np.array_equal(losses_a, np.array(losses_b, dtype=np.float32))
+    assert np.array_equal(losses_a, dl.cpu().numpy())
+    assert np.array_equal(a.get_params(), b.get_params()) and np.array_equal(a.get_params(), c.get_params())
+
+
+def test_checkpoint_round_trip(tiny):
+    import paper_2408_10746_b200 as pac
+    hp = pac.AdamW()
+    perm = pi.epoch_permutation(TINY.N, 2)
+    full = tiny.context()
+    full.train_epoch(perm[:80], TINY.B, hp)
+    first = tiny.context()
+    first.train_epoch(perm[:40], TINY.B, hp)
+    params, (m, v, step) = first.get_params(), first.get_opt_state()
+    assert step == 5
+    second = tiny.context(seed=99)
+    second.set_params(params)
+    second.set_opt_state(m, v, step)
+    second.train_epoch(perm[40:80], TINY.B, hp)
+    assert np.array_equal(second.get_params(), full.get_params())
+
+
+def test_frozen_inputs_untouched_and_errors_leave_state_alone(tiny):
+    import paper_2408_10746_b200 as pac
+    ctx = tiny.context()
+    before = (tiny.cache.clone(), tiny.labels.clone())
+    p0 = ctx.get_params()
+    for bad in ([TINY.N], [-1], [0, 1, 2, 10 ** 6]):
+        with pytest.raises(pac.PacError) as e:
+            ctx.train_step(bad)
+        assert e.value.status_name == "PAC_ERR_SAMPLE_ID_RANGE"
+    with pytest.raises(pac.PacError) as e:
+        ctx.train_step(list(range(TINY.B + 1)))
+    assert e.value.status_name == "PAC_ERR_INVALID_ARG"
+    with pytest.raises(pac.PacError):
+        ctx.train_epoch(np.arange(12, dtype=np.int32), 8, pac.AdamW())
+    with pytest.raises(pac.PacError):
+        ctx.adam_step(pac.AdamW(beta1=1.5))
+    assert np.array_equal(ctx.get_params(), p0)
+    ctx.train_epoch(np.arange(64, dtype=np.int32), 8, pac.AdamW())
+    out = torch.zeros((8, 2), device="cuda")
+    ctx.eval_logits(list(range(8)), out)
+    ctx.sync()
+    assert torch.equal(before[0], tiny.cache) and torch.equal(before[1], tiny.labels)
+    assert ctx.launch_count() > 0
+
+
+def test_call_order_is_enforced():
+    import paper_2408_10746_b200 as pac
+    ctx = pac.PacContext(0)
+    with pytest.raises(pac.PacError) as e:
+        ctx.adapter_init(r=4, n_out=2, max_batch=2)
+    assert e.value.status_name == "PAC_ERR_BAD_STATE"
+    with pytest.raises(pac.PacError) as e:
+        ctx.train_step([0])
+    assert e.value.status_name == "PAC_ERR_BAD_STATE"
+
+
+def test_device_resident_bad_id_is_clamped_and_reported(tiny):
+    import paper_2408_10746_b200 as pac
+    ctx = tiny.context()
+    dperm = torch.tensor([0, 1, 2, 3, 4, 5, 6, 10 ** 6], dtype=torch.int32, device="cuda")
+    ctx.train_epoch_dev(dperm, 8, pac.AdamW())
+    with pytest.raises(pac.PacError) as e:
+        ctx.sync()
+    assert e.value.status_name == "PAC_ERR_SAMPLE_ID_RANGE"
+    ctx.sync()                                              # the report is one-shot
+    assert np.isfinite(ctx.get_params()).all()
