@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of adapter-over-cache training (PAC+ phase 2) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one minibatch: gather of the cached
+states, adapter forward, head and loss, adapter-only backward, AdamW.  `value` is
+samples/s with the cache, the shuffled ids and the losses resident in HBM (one
+pac_train_epoch_dev call over K*B ids); `e2e` is the same metric through
+pac_train_step/pac_adam_step with host ids in and the host loss out every step.
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import pac_inputs as pi  # noqa: E402
+
+METRIC = "adapter_epoch_samples_per_sec"
+UNIT = "samples/s"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
+# capture summarised under profiles/ (None until a capture of the current kernel exists).
+NCU_TRAFFIC_BYTES = {"t5_base": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def workload_name(spec: pi.CacheSpec) -> str:
+    return (f"{spec.name}: cache N={spec.N} L={spec.L} S={spec.S} d={spec.d} {spec.dtype}, r={spec.r}, "
+            f"{'C' if spec.head == 'cls' else 'V'}={spec.n_out}, B={spec.B}, shuffled epochs")
+
+
+def epoch_ids(spec: pi.CacheSpec, steps: int) -> np.ndarray:
+    """K*B ids: consecutive seeded permutations of 0..N-1 (one per epoch), cut at K steps."""
+    out, e = [], 0
+    while sum(len(x) for x in out) < steps * spec.B:
+        perm = pi.epoch_permutation(spec.N, 2, epoch=e)
+        out.append(perm[:(spec.N // spec.B) * spec.B])
+        e += 1
+    return np.concatenate(out)[:steps * spec.B].astype(np.int32)
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int, period_s: float = 0.005):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.max_mhz = period_s, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception as e:  # NVML missing: report that clocks were not sampled
+            self.err = repr(e)
+
+    def run(self):
+        while self.ok and not self._stop_evt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def finish(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=1.0)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "note": "clocks not sampled"}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": float(self.max_mhz),
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_baseline(spec: pi.CacheSpec, budget_s: float, max_steps: int):
+    """Times the CPU oracle as it stands on a bounded sample: whole train steps (B samples each)
+    on freshly generated slabs until about budget_s of oracle time is spent."""
+    from oracle import pac_oracle as po
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    perm = pi.epoch_permutation(spec.N, 2)
+    P = po.unflatten(pi.random_params(spec, 3), spec.L, spec.d, spec.r, spec.n_out if spec.head == "cls" else None)
+    labels_all = pi.labels(spec, 0).numpy().astype(np.int64)
+    W_lm = pi.lm_head(spec, 0).float().numpy() if spec.head == "lm" else None
+    spent, steps = 0.0, 0
+    while steps < max_steps and (steps == 0 or spent < budget_s):
+        ids = perm[steps * spec.B:(steps + 1) * spec.B].tolist()
+        cache = pi.cache_samples(spec, 0, ids).float().numpy()
+        tr = po.Trainer(cache, labels_all[ids], P, W_lm=W_lm) if steps == 0 else tr
+        tr.cache, tr.labels = cache, labels_all[ids]
+        t0 = time.perf_counter()
+        tr.train_step(list(range(spec.B)))
+        tr.adam_step()
+        spent += time.perf_counter() - t0
+        steps += 1
+    return {"value": steps * spec.B / spent, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"{steps} whole train steps (B={spec.B}) of {spec.name} in fp32, {spent:.1f} s of oracle time; "
+                      "slab generation not timed"}
+
+
+def run_reference(args, spec):
+    """The reference arm: the CPU oracle as it stands, K timed steps after W warm-up steps,
+    each step a bounded sample (B' <= B samples) so the run ends within a few minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import pac_oracle as po
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    P = po.unflatten(pi.random_params(spec, 3), spec.L, spec.d, spec.r, spec.n_out if spec.head == "cls" else None)
+    labels_all = pi.labels(spec, 0).numpy().astype(np.int64)
+    W_lm = pi.lm_head(spec, 0).float().numpy() if spec.head == "lm" else None
+    perm = pi.epoch_permutation(spec.N, 2)
+    pool_ids = perm[:spec.B].tolist()
+    cache = pi.cache_samples(spec, 0, pool_ids).float().numpy()
+    tr = po.Trainer(cache, labels_all[pool_ids], P, W_lm=W_lm)
+    t0 = time.perf_counter()
+    tr.train_step(list(range(spec.B)))
+    tr.adam_step()
+    t_full = time.perf_counter() - t0
+    total = args.steps + args.warmup
+    Bp = spec.B if t_full * total <= 150 else max(1, int(spec.B * 150 / (t_full * total)))
+    sub = list(range(Bp))
+    for _ in range(args.warmup):
+        tr.train_step(sub); tr.adam_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        tr.train_step(sub); tr.adam_step()
+    dt = time.perf_counter() - t0
+    value = args.steps * Bp / dt
+    sample = (f"{args.steps} oracle train steps of {Bp} samples each (of B={spec.B}) drawn from one generated "
+              f"minibatch of {spec.name}, fp32")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(spec), "note": "CPU oracle on host cores"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2560)
+    ap.add_argument("--warmup", type=int, default=128)
+    ap.add_argument("--config", default="t5_base", choices=sorted(pi.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--force-simt", action="store_true", help="use the plain fp32-FMA kernels")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    spec = pi.CONFIGS[args.config]
+    if args.impl == "reference":
+        return run_reference(args, spec)
+
+    import torch
+    import paper_2408_10746_b200 as pac
+    from paper_2408_10746_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # the cache must fit: keep 8 GB of headroom, halve N otherwise (and say so)
+    note = []
+    free, _ = torch.cuda.mem_get_info()
+    while spec.cache_bytes + (8 << 30) > free and spec.N > spec.B:
+        spec = spec.scaled(N=spec.N // 2)
+        note.append(f"N halved to {spec.N} to fit device memory")
+
+    dev = torch.device("cuda", local)
+    seed = rank                                   # each rank trains its own replica on its own cache
+    cache = pi.cache_full(spec, seed, dev)
+    labels = pi.labels(spec, seed, dev)
+    lm = pi.lm_head(spec, seed, dev) if spec.head == "lm" else None
+    stream = torch.cuda.Stream(device=dev)
+    ctx = pac.PacContext(local, stream.cuda_stream)
+    if args.force_simt:
+        ctx.set_option(binding.PAC_OPT_KERNEL_PATH, 1)
+    ctx.cache_register(cache, labels)
+    ctx.adapter_init(r=spec.r, n_out=spec.n_out, max_batch=spec.B,
+                     head=pac.PAC_HEAD_FROZEN_LM if spec.head == "lm" else pac.PAC_HEAD_MEANPOOL_CLS, lm_head=lm)
+    hp = pac.AdamW()
+    K, W, B = args.steps, args.warmup, spec.B
+    ids_host = epoch_ids(spec, K)
+    d_ids = torch.from_numpy(ids_host).to(dev)
+    d_warm = torch.from_numpy(epoch_ids(spec, W)).to(dev)
+    d_losses = torch.zeros(K, dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- device-resident timing (value) ----------------
+    ctx.train_epoch_dev(d_warm, B, hp, None)
+    ctx.sync()
+    sampler = ClockSampler(local)
+    launches0 = ctx.launch_count()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    with torch.cuda.stream(stream):
+        start.record(stream)
+        ctx.train_epoch_dev(d_ids, B, hp, d_losses)
+        end.record(stream)
+    barrier()
+    clocks = sampler.finish()
+    ms = start.elapsed_time(end)
+    launches = ctx.launch_count() - launches0
+    ctx.sync()
+    losses = d_losses.cpu().numpy()
+    if not np.isfinite(losses).all():
+        raise SystemExit("non-finite loss in the timed region")
+
+    # ---------------- end to end through the public per-step calls ----------------
+    for i in range(3):
+        ctx.train_step(ids_host[i * B:(i + 1) * B]); ctx.adam_step(hp)
+    Ke = min(K, 512)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for i in range(Ke):
+            ctx.train_step(ids_host[i * B:(i + 1) * B], want_loss=True)
+            ctx.adam_step(hp)
+        e1.record(stream)
+    barrier()
+    wall_ms = 1e3 * (time.perf_counter() - t0)
+    e2e_ms = max(e0.elapsed_time(e1), wall_ms)
+
+    # ---------------- per-kernel times of the two cache-stream kernels ----------------
+    ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 1)
+    ctx.kernel_times()
+    Kt = min(K, 256)
+    ctx.train_epoch_dev(d_ids[:Kt * B], B, hp, None)
+    kt = ctx.kernel_times()
+    ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 0)
+
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = t.tolist()
+
+    peaks = load_peaks()
+    pass_bytes = B * spec.L * spec.S * spec.d * spec.elem_bytes          # one read of the minibatch's slabs
+    kern = {}
+    for name, (tot_ms, cnt) in kt.items():
+        if cnt:
+            avg = tot_ms / cnt
+            kern[name] = {"avg_ms": avg, "launches": cnt, "gbs": pass_bytes / (avg * 1e-3) / 1e9}
+    dominant = max(kern, key=lambda k: kern[k]["avg_ms"]) if kern else None
+    roofline = None
+    if dominant:
+        a = kern[dominant]["gbs"]
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name), "algorithmic_bytes_per_launch": pass_bytes,
+                    "kernels": kern}
+    step_s = ms * 1e-3 / K
+    stream_gbs = 2 * pass_bytes / step_s / 1e9
+
+    out = {
+        "metric": METRIC, "value": world * K * B / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if spec.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": workload_name(spec), "kernel_path": ctx.kernel_path(),
+                   "l2": "each step gathers a different minibatch from a cache far larger than L2 "
+                         f"({spec.cache_bytes / 1e9:.2f} GB)", "parallelism": "replicas" if world > 1 else "1 GPU",
+                   "notes": note},
+        "clocks": clocks,
+        "e2e": {"value": world * Ke * B / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * B,
+                "d2h_bytes_per_step": 4, "steps": Ke},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cache_stream": {"gbs_two_reads": stream_gbs, "frac_of_peak": stream_gbs / peaks["hbm_gbs"],
+                         "gbs_one_read": stream_gbs / 2, "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+                         "frac_of_8000_nominal": stream_gbs / 8000.0},
+        "final_loss": float(losses[-1]),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = oracle_baseline(spec, args.cpu_budget, 16)
+    elif rank == 0:
+        out["cpu_baseline"] = None
+    ctx.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -71,8 +71,9 @@ typedef struct { float lr, beta1, beta2, eps, weight_decay; } pac_adamw;
 
 /* Options for pac_set_option. */
 typedef enum {
-    PAC_OPT_KERNEL_PATH = 0   /* 0 = automatic (tensor-core path when the shape allows),
-                                 1 = force the plain fp32-FMA kernels */
+    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic (tensor-core path when the shape allows),
+                                 1 = force the plain fp32-FMA kernels; set before adapter_init */
+    PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events */
 } pac_option;
 
 /* Creates a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t to
@@ -137,6 +138,13 @@ pac_status pac_get_opt_state(pac_ctx* ctx, float* m, float* v, long long* step);
 pac_status pac_set_opt_state(pac_ctx* ctx, const float* m, const float* v, long long step);
 
 pac_status pac_set_option(pac_ctx* ctx, int option, int value);
+/* Per-kernel device times.  With PAC_OPT_KERNEL_TIMING = 1 the two cache-stream kernels of
+ * every later train step (down-projection u_l = h_l W_down^l over all layers; dW_down =
+ * h_l^T du_l over all layers) are bracketed by CUDA events on the context's stream.  This
+ * call waits for the stream, then stores the summed milliseconds and launch counts since the
+ * last call: out_ms[0], out_count[0] for the down-projection, [1] for dW_down (host arrays of 2).
+ * At most 4096 bracketed launches per kernel are kept between two calls. */
+pac_status pac_kernel_times(pac_ctx* ctx, double* out_ms, long long* out_count);
 /* Number of kernels this context has launched so far. */
 pac_status pac_launch_count(pac_ctx* ctx, long long* n);
 /* Waits for the context's stream; reports device-side status words (bounded waits that

@@ -17,6 +17,7 @@ PAC_F32, PAC_BF16 = 0, 1
 PAC_ACT_RELU, PAC_ACT_IDENTITY = 0, 1
 PAC_HEAD_MEANPOOL_CLS, PAC_HEAD_FROZEN_LM = 0, 1
 PAC_OPT_KERNEL_PATH = 0
+PAC_OPT_KERNEL_TIMING = 1
 STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_SAMPLE_ID_RANGE",
                 "PAC_ERR_UNSUPPORTED", "PAC_ERR_NOMEM", "PAC_ERR_CUDA", "PAC_ERR_TIMEOUT"]
 
@@ -24,7 +25,7 @@ STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_S
 EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init", "pac_train_step",
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
-           "pac_set_opt_state", "pac_set_option", "pac_launch_count", "pac_sync", "pac_last_error",
+           "pac_set_opt_state", "pac_set_option", "pac_kernel_times", "pac_launch_count", "pac_sync", "pac_last_error",
            "pac_kernel_path"]
 
 
@@ -87,6 +88,7 @@ def load_library() -> C.CDLL:
         "pac_get_grads": [P, P], "pac_get_opt_state": [P, P, P, C.POINTER(LL)],
         "pac_set_opt_state": [P, P, P, LL], "pac_set_option": [P, I, I],
         "pac_launch_count": [P, C.POINTER(LL)], "pac_sync": [P],
+        "pac_kernel_times": [P, C.POINTER(C.c_double), C.POINTER(LL)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -230,6 +232,13 @@ class PacContext:
         m = np.ascontiguousarray(m, dtype=np.float32)
         v = np.ascontiguousarray(v, dtype=np.float32)
         self._ck(self._lib.pac_set_opt_state(self._h, m.ctypes.data, v.ctypes.data, step))
+
+    def kernel_times(self):
+        """(ms_total, launches) for the down-projection and for dW_down since the last call."""
+        ms = (C.c_double * 2)()
+        cnt = (C.c_longlong * 2)()
+        self._ck(self._lib.pac_kernel_times(self._h, ms, cnt))
+        return {"down_projection": (ms[0], cnt[0]), "dw_down": (ms[1], cnt[1])}
 
     def launch_count(self) -> int:
         n = C.c_longlong()

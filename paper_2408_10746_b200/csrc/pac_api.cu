@@ -76,6 +76,9 @@ struct pac_ctx {
     float* d_losses = nullptr; long long losses_cap = 0;
     // options / bookkeeping
     int force_simt = 0;
+    int timing = 0;
+    std::vector<cudaEvent_t> tev[2];   // start/stop pairs per bracketed kernel
+    size_t tev_used[2] = {0, 0};
     bool tensor_ok = false;
     long long launches = 0;
     TensorPlan tplan{};
@@ -152,6 +155,23 @@ void fill_initial_params(const pac_ctx* c, unsigned long long seed, std::vector<
     for (long long i = lay.w_head; i < lay.b_head; ++i) out[i] = unit_normal(key, (unsigned long long)i) * inv;
 }
 
+// ---- optional event brackets around the two cache-stream kernels ----
+constexpr size_t MAX_TIMED = 4096;
+void time_mark(pac_ctx* c, int which, bool stop) {
+    if (!c->timing) return;
+    size_t pair = c->tev_used[which] / 2;
+    if (pair >= MAX_TIMED) return;
+    if (c->tev[which].size() < 2 * (pair + 1)) {
+        cudaEvent_t a, b;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+        c->tev[which].push_back(a);
+        c->tev[which].push_back(b);
+    }
+    cudaEventRecord(c->tev[which][c->tev_used[which]], c->stream);
+    c->tev_used[which] += 1;
+    (void)stop;
+}
+
 // ---- staging of host ids ----
 pac_status stage_ids(pac_ctx* c, const int* ids, int B, const char* who) {
     if (!ids) return fail(c, PAC_ERR_INVALID_ARG, "%s: sample_ids is NULL", who);
@@ -192,6 +212,7 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
     const long long stride = (long long)M * dm.r;
     Scratch& sc = c->sc;
     pac_status st;
+    time_mark(c, 0, false);
     if (use_tensor(c)) {
         st = tensor_down_projection(c->tplan, c->stream, d_ids, B, sc.u, c->status, &c->launches);
         if (st != PAC_OK) return fail(c, st, "tensor-core down-projection launch failed: %s", tensor_last_error());
@@ -199,6 +220,7 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
         st = c->dtype == PAC_F32 ? down_projection_simt<float>(c, d_ids, B) : down_projection_simt<bf16>(c, d_ids, B);
         if (st != PAC_OK) return st;
     }
+    time_mark(c, 0, true);
     const float* lam = c->params + c->lay.lam;
     if (c->cfg.act == PAC_ACT_RELU)
         chain_fwd_kernel<PAC_ACT_RELU><<<cdiv(stride, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, stride);
@@ -316,13 +338,18 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
     LAUNCH_CHECK(c);
     reduce_rows_kernel<<<dm.L, 256, 0, c->stream>>>(sc.lam_part, (int)blocks, c->grads + c->lay.lam);
     LAUNCH_CHECK(c);
+    pac_status st;
+    time_mark(c, 1, false);
     if (tens) {
-        pac_status st = tensor_dw_down(c->tplan, c->stream, d_ids, B, sc.du16, c->grads + c->lay.w_down, sc.dw_part,
-                                       c->status, &c->launches);
+        st = tensor_dw_down(c->tplan, c->stream, d_ids, B, sc.du16, c->grads + c->lay.w_down, sc.dw_part,
+                            c->status, &c->launches);
         if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
-        return PAC_OK;
+    } else {
+        st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
+        if (st != PAC_OK) return st;
     }
-    return c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
+    time_mark(c, 1, true);
+    return PAC_OK;
 }
 
 pac_status adam_enqueue(pac_ctx* c, const pac_adamw* hp) {
@@ -363,6 +390,8 @@ void free_all(pac_ctx* c) {
     if (c->h_status) cudaFreeHost(c->h_status);
     for (auto& e : c->slot_ev)
         if (e) cudaEventDestroy(e);
+    for (auto& vec : c->tev)
+        for (auto& e : vec) cudaEventDestroy(e);
     if (c->own_stream && c->stream) cudaStreamDestroy(c->stream);
 }
 
@@ -683,7 +712,31 @@ pac_status pac_set_option(pac_ctx* c, int option, int value) {
         c->force_simt = value;
         return PAC_OK;
     }
+    if (option == PAC_OPT_KERNEL_TIMING) {
+        if (value != 0 && value != 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: timing must be 0 or 1");
+        c->timing = value;
+        return PAC_OK;
+    }
     return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: unknown option %d", option);
+}
+
+pac_status pac_kernel_times(pac_ctx* c, double* out_ms, long long* out_count) {
+    NEED_CTX(c);
+    if (!out_ms || !out_count) return fail(c, PAC_ERR_INVALID_ARG, "pac_kernel_times: NULL argument");
+    CU_OK(c, cudaSetDevice(c->device));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    for (int w = 0; w < 2; ++w) {
+        double tot = 0.0;
+        long long cnt = 0;
+        for (size_t i = 0; i + 1 < c->tev_used[w]; i += 2) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, c->tev[w][i], c->tev[w][i + 1]) == cudaSuccess) { tot += ms; cnt++; }
+        }
+        out_ms[w] = tot;
+        out_count[w] = cnt;
+        c->tev_used[w] = 0;
+    }
+    return PAC_OK;
 }
 
 pac_status pac_launch_count(pac_ctx* c, long long* n) {
