@@ -191,10 +191,15 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--force-simt", action="store_true", help="use the plain fp32-FMA kernels")
+    ap.add_argument("--n-samples", type=int, default=0,
+                    help="profiling aid: shrink the cache to this many samples (same per-step shapes); "
+                         "the JSON line then names the reduced workload")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     spec = pi.CONFIGS[args.config]
+    if args.n_samples:
+        spec = spec.scaled(N=args.n_samples, name=f"{spec.name}[N={args.n_samples}]")
     if args.impl == "reference":
         return run_reference(args, spec)
 
@@ -309,7 +314,7 @@ def main():
         a = kern[dominant]["gbs"]
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name), "algorithmic_bytes_per_launch": pass_bytes,
+                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]), "algorithmic_bytes_per_launch": pass_bytes,
                     "kernels": kern}
     step_s = ms * 1e-3 / K
     stream_gbs = 2 * pass_bytes / step_s / 1e9

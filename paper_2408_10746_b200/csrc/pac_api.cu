@@ -8,6 +8,7 @@
 #include "pac_common.cuh"
 #include "pac_simt.cuh"
 #include "pac_tensor.cuh"
+#include "pac_mid.cuh"
 
 using namespace pac;
 
@@ -38,7 +39,7 @@ struct Scratch {
     float* lm_logits = nullptr;    // [M][V]
     float* dy = nullptr;           // [M][d]
     // tensor path
-    bf16* wdT = nullptr;           // [L][r][d] bf16 shadow of W_down, transposed
+    bf16* wdT = nullptr;           // [L][2][r][d] bf16 hi/lo shadow of W_down, transposed
     float* dw_part = nullptr;      // split partials of dW_down
 };
 
@@ -82,6 +83,7 @@ struct pac_ctx {
     bool tensor_ok = false;
     long long launches = 0;
     TensorPlan tplan{};
+    MidPlan mplan{};               // fused classifier-head kernel (when the shape allows)
     std::string err;
 };
 
@@ -123,6 +125,9 @@ pac_status dmalloc(pac_ctx* c, T** p, long long n) {
 }
 
 bool use_tensor(const pac_ctx* c) { return c->tensor_ok && !c->force_simt; }
+pac_status adam_enqueue(pac_ctx* c, const pac_adamw* hp);
+pac_status down_projection(pac_ctx* c, const int* d_ids, int B);
+pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits);
 
 inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
 
@@ -199,7 +204,7 @@ pac_status down_projection_simt(pac_ctx* c, const int* d_ids, int B) {
     const int M = B * dm.S;
     CacheRows<T> A{(const T*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, 0};
     MatB_RowMajor Bm{{c->params + c->lay.w_down, (long long)dm.d * dm.r, dm.r}};
-    StoreRowMajor E{c->sc.u, (long long)M * dm.r, dm.r};
+    StoreRowMajor E{c->sc.u, (long long)c->max_rows * dm.r, dm.r};
     dim3 grid(cdiv(dm.r, SG_BN), cdiv(M, SG_BM), dm.L);
     gemm_simt<<<grid, 256, 0, c->stream>>>(M, dm.r, dm.d, A, Bm, E);
     LAUNCH_CHECK(c);
@@ -209,23 +214,15 @@ pac_status down_projection_simt(pac_ctx* c, const int* d_ids, int B) {
 pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
     const Dims& dm = c->dm;
     const int M = B * dm.S;
-    const long long stride = (long long)M * dm.r;
+    const long long n = (long long)M * dm.r, stride = (long long)c->max_rows * dm.r;
     Scratch& sc = c->sc;
-    pac_status st;
-    time_mark(c, 0, false);
-    if (use_tensor(c)) {
-        st = tensor_down_projection(c->tplan, c->stream, d_ids, B, sc.u, c->status, &c->launches);
-        if (st != PAC_OK) return fail(c, st, "tensor-core down-projection launch failed: %s", tensor_last_error());
-    } else {
-        st = c->dtype == PAC_F32 ? down_projection_simt<float>(c, d_ids, B) : down_projection_simt<bf16>(c, d_ids, B);
-        if (st != PAC_OK) return st;
-    }
-    time_mark(c, 0, true);
+    pac_status st = down_projection(c, d_ids, B);
+    if (st != PAC_OK) return st;
     const float* lam = c->params + c->lay.lam;
     if (c->cfg.act == PAC_ACT_RELU)
-        chain_fwd_kernel<PAC_ACT_RELU><<<cdiv(stride, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, stride);
+        chain_fwd_kernel<PAC_ACT_RELU><<<cdiv(n, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, n, stride);
     else
-        chain_fwd_kernel<PAC_ACT_IDENTITY><<<cdiv(stride, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, stride);
+        chain_fwd_kernel<PAC_ACT_IDENTITY><<<cdiv(n, 256), 256, 0, c->stream>>>(sc.u, sc.a, lam, dm.L, n, stride);
     LAUNCH_CHECK(c);
     const float* aL = sc.a + (long long)(dm.L - 1) * stride;
     const float* W_up = c->params + c->lay.w_up;
@@ -273,7 +270,7 @@ pac_status dw_down_simt(pac_ctx* c, const int* d_ids, int B) {
     const Dims& dm = c->dm;
     const int M = B * dm.S;
     CacheRowsT<T> A{(const T*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d};
-    MatB_RowMajor Bm{{c->sc.du, (long long)M * dm.r, dm.r}};
+    MatB_RowMajor Bm{{c->sc.du, (long long)c->max_rows * dm.r, dm.r}};
     StoreRowMajor E{c->grads + c->lay.w_down, (long long)dm.d * dm.r, dm.r};
     dim3 grid(cdiv(dm.r, SG_BN), cdiv(dm.d, SG_BM), dm.L);
     gemm_simt<<<grid, 256, 0, c->stream>>>(dm.d, dm.r, M, A, Bm, E);
@@ -285,7 +282,7 @@ pac_status dw_down_simt(pac_ctx* c, const int* d_ids, int B) {
 pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
     const Dims& dm = c->dm;
     const int M = B * dm.S;
-    const long long stride = (long long)M * dm.r;
+    const long long n = (long long)M * dm.r, stride = (long long)c->max_rows * dm.r;
     Scratch& sc = c->sc;
     const float* aL = sc.a + (long long)(dm.L - 1) * stride;
     const float* W_up = c->params + c->lay.w_up;
@@ -324,11 +321,11 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
         per_sample = 0;
     }
     const float* lam = c->params + c->lay.lam;
-    const unsigned blocks = cdiv(stride, 256);
+    const unsigned blocks = cdiv(n, 256);
     const bool tens = use_tensor(c);
 #define CHAIN_BWD(ACT, DUT, DUP)                                                                              \
     chain_bwd_kernel<ACT, DUT><<<blocks, 256, 0, c->stream>>>(sc.u, sc.a, lam, sc.daL, per_sample, dm.S, dm.r, \
-                                                              dm.L, stride, DUP, sc.lam_part)
+                                                              dm.L, n, stride, DUP, sc.lam_part)
     if (c->cfg.act == PAC_ACT_RELU) {
         if (tens) CHAIN_BWD(PAC_ACT_RELU, bf16, sc.du16); else CHAIN_BWD(PAC_ACT_RELU, float, sc.du);
     } else {
@@ -338,11 +335,31 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
     LAUNCH_CHECK(c);
     reduce_rows_kernel<<<dm.L, 256, 0, c->stream>>>(sc.lam_part, (int)blocks, c->grads + c->lay.lam);
     LAUNCH_CHECK(c);
+    return dw_down(c, d_ids, B, true);
+}
+
+bool use_fused_cls(const pac_ctx* c) { return c->cfg.head == PAC_HEAD_MEANPOOL_CLS && c->mplan.ok; }
+
+pac_status down_projection(pac_ctx* c, const int* d_ids, int B) {
+    pac_status st;
+    time_mark(c, 0, false);
+    if (use_tensor(c)) {
+        st = tensor_down_projection(c->tplan, c->stream, d_ids, B, c->sc.u, c->status, &c->launches);
+        if (st != PAC_OK) return fail(c, st, "tensor-core down-projection launch failed: %s", tensor_last_error());
+    } else {
+        st = c->dtype == PAC_F32 ? down_projection_simt<float>(c, d_ids, B) : down_projection_simt<bf16>(c, d_ids, B);
+        if (st != PAC_OK) return st;
+    }
+    time_mark(c, 0, true);
+    return PAC_OK;
+}
+
+pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     pac_status st;
     time_mark(c, 1, false);
-    if (tens) {
-        st = tensor_dw_down(c->tplan, c->stream, d_ids, B, sc.du16, c->grads + c->lay.w_down, sc.dw_part,
-                            c->status, &c->launches);
+    if (use_tensor(c)) {
+        st = tensor_dw_down(c->tplan, c->stream, d_ids, B, c->sc.du16, c->grads + c->lay.w_down, c->sc.dw_part,
+                            reduce_splits, c->status, &c->launches);
         if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
     } else {
         st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
@@ -352,12 +369,76 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
     return PAC_OK;
 }
 
+pac_status mid_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    const Dims& dm = c->dm;
+    Scratch& sc = c->sc;
+    MidParams p{};
+    p.ids = d_ids; p.N = dm.N; p.labels = c->labels;
+    p.L = dm.L; p.S = dm.S; p.d = dm.d; p.r = dm.r; p.C = dm.C; p.B = B;
+    p.G = c->mplan.G; p.Sg = c->mplan.Sg; p.dg = c->mplan.dg; p.train = train ? 1 : 0;
+    p.u = sc.u; p.lstride = (long long)c->max_rows * dm.r;
+    p.lam = c->params + c->lay.lam; p.W_up = c->params + c->lay.w_up;
+    p.W_head = c->params + c->lay.w_head; p.b_head = c->params + c->lay.b_head; p.hbar = sc.hbar;
+    const bool tens = use_tensor(c);
+    p.du = tens ? (void*)sc.du16 : (void*)sc.du;
+    p.pooled_a = sc.pooled_a; p.pooled_y = sc.pooled_y; p.gvec = sc.gvec; p.dlogits = sc.dlogits;
+    p.loss_b = sc.loss_b; p.lam_part = sc.lam_part; p.logits_out = train ? sc.logits : d_logits_out;
+    p.status = c->status;
+    cudaError_t e = mid_launch(c->mplan, p, c->cfg.act, tens, c->stream);
+    c->launches++;
+    if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "fused head kernel launch failed: %s", cudaGetErrorString(e));
+    return PAC_OK;
+}
+
+void bias_corrections(const pac_adamw* hp, long long step, float* bc1, float* bc2) {
+    *bc1 = (float)(1.0 - std::pow((double)hp->beta1, (double)step));
+    *bc2 = (float)(1.0 - std::pow((double)hp->beta2, (double)step));
+}
+
+pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* hp) {
+    const Dims& dm = c->dm;
+    Scratch& sc = c->sc;
+    FinalizeParams f{};
+    f.lay = c->lay; f.B = B; f.d = dm.d; f.r = dm.r; f.C = dm.C; f.L = dm.L;
+    f.dw_part = sc.dw_part;
+    f.splits = use_tensor(c) ? tensor_splits(c->tplan, B) : 1;
+    f.dw_elems = (long long)dm.L * dm.d * dm.r;
+    f.lam_part = sc.lam_part; f.lam_blocks = B * c->mplan.G;
+    f.pooled_a = sc.pooled_a; f.gvec = sc.gvec; f.pooled_y = sc.pooled_y; f.dlogits = sc.dlogits; f.loss_b = sc.loss_b;
+    f.grads = c->grads; f.loss_out = d_loss;
+    f.adam = hp ? 1 : 0;
+    if (hp) {
+        c->step += 1;
+        f.params = c->params; f.m = c->m; f.v = c->v; f.hp = *hp;
+        bias_corrections(hp, c->step, &f.bc1, &f.bc2);
+        f.wdT = sc.wdT;
+    }
+    finalize_cls_kernel<<<cdiv(c->lay.total, 256), 256, 0, c->stream>>>(f);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+// One whole train step; with hp != NULL the AdamW update is fused into the last kernel.
+pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, const pac_adamw* hp) {
+    pac_status st;
+    if (use_fused_cls(c)) {
+        if ((st = down_projection(c, d_ids, B)) != PAC_OK) return st;
+        if ((st = mid_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
+        if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
+        return finalize_enqueue(c, B, d_loss, hp);
+    }
+    if ((st = forward(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
+    if ((st = backward(c, d_ids, B, d_loss)) != PAC_OK) return st;
+    if (hp) return adam_enqueue(c, hp);
+    return PAC_OK;
+}
+
 pac_status adam_enqueue(pac_ctx* c, const pac_adamw* hp) {
     c->step += 1;
-    const float inv_bc1 = (float)(1.0 / (1.0 - std::pow((double)hp->beta1, (double)c->step)));
-    const float inv_bc2 = (float)(1.0 / (1.0 - std::pow((double)hp->beta2, (double)c->step)));
+    float bc1, bc2;
+    bias_corrections(hp, c->step, &bc1, &bc2);
     adamw_kernel<<<cdiv(c->lay.total, 256), 256, 0, c->stream>>>(c->params, c->grads, c->m, c->v, c->lay.total, c->lay,
-                                                                 *hp, inv_bc1, inv_bc2, c->sc.wdT, c->dm.d, c->dm.r);
+                                                                 *hp, bc1, bc2, c->sc.wdT, c->dm.d, c->dm.r);
     LAUNCH_CHECK(c);
     return PAC_OK;
 }
@@ -485,6 +566,8 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     c->max_rows = cfg->max_batch * dm.S;
     const long long Mr = (long long)c->max_rows * dm.r;
     c->chain_blocks_max = (int)cdiv(Mr, 256);
+    c->mplan = cls ? mid_plan(dm) : MidPlan{};
+    if (c->mplan.ok && cfg->max_batch * c->mplan.G > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * c->mplan.G;
     Scratch& s = c->sc;
     pac_status st = PAC_OK;
     auto A = [&](pac_status x) { if (st == PAC_OK) st = x; };
@@ -515,7 +598,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     // tensor-core path: bf16 cache with TMA/UMMA-compatible sizes
     c->tensor_ok = false;
     if (st == PAC_OK && c->dtype == PAC_BF16 && tensor_shape_supported(dm)) {
-        A(dmalloc(c, &s.wdT, (long long)dm.L * dm.r * dm.d));
+        A(dmalloc(c, &s.wdT, (long long)dm.L * 2 * dm.r * dm.d));
         A(dmalloc(c, &s.du16, Mr * dm.L));
         long long part_floats = 0;
         if (st == PAC_OK) {
@@ -529,8 +612,12 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             }
         }
     }
-    if (st == PAC_OK && !c->tensor_ok) A(dmalloc(c, &s.du, Mr * dm.L));
+    if (st == PAC_OK && !use_tensor(c)) A(dmalloc(c, &s.du, Mr * dm.L));    // the plain path keeps du in fp32
     if (st != PAC_OK) return st;
+    CU_OK(c, cudaMemsetAsync(s.u, 0, sizeof(float) * Mr * dm.L, c->stream));
+    CU_OK(c, cudaMemsetAsync(s.a, 0, sizeof(float) * Mr * dm.L, c->stream));
+    if (s.du) CU_OK(c, cudaMemsetAsync(s.du, 0, sizeof(float) * Mr * dm.L, c->stream));
+    if (s.du16) CU_OK(c, cudaMemsetAsync(s.du16, 0, sizeof(bf16) * Mr * dm.L, c->stream));
     CU_OK(c, cudaMemsetAsync(c->grads, 0, sizeof(float) * c->lay.total, c->stream));
     CU_OK(c, cudaMemsetAsync(c->m, 0, sizeof(float) * c->lay.total, c->stream));
     CU_OK(c, cudaMemsetAsync(c->v, 0, sizeof(float) * c->lay.total, c->stream));
@@ -556,8 +643,7 @@ pac_status pac_train_step(pac_ctx* c, const int* sample_ids, int B, float* loss_
     NEED_INIT(c, "pac_train_step");
     pac_status st = stage_ids(c, sample_ids, B, "pac_train_step");
     if (st != PAC_OK) return st;
-    if ((st = forward(c, c->sc.ids, B, true, nullptr)) != PAC_OK) return st;
-    if ((st = backward(c, c->sc.ids, B, c->sc.loss)) != PAC_OK) return st;
+    if ((st = train_enqueue(c, c->sc.ids, B, c->sc.loss, nullptr)) != PAC_OK) return st;
     if (loss_out) {
         CU_OK(c, cudaMemcpyAsync(c->h_loss, c->sc.loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
         CU_OK(c, cudaStreamSynchronize(c->stream));
@@ -578,6 +664,10 @@ pac_status pac_eval_logits(pac_ctx* c, const int* sample_ids, int B, float* dev_
     if (!dev_out) return fail(c, PAC_ERR_INVALID_ARG, "pac_eval_logits: dev_out is NULL");
     pac_status st = stage_ids(c, sample_ids, B, "pac_eval_logits");
     if (st != PAC_OK) return st;
+    if (use_fused_cls(c)) {
+        if ((st = down_projection(c, c->sc.ids, B)) != PAC_OK) return st;
+        return mid_enqueue(c, c->sc.ids, B, false, dev_out);
+    }
     return forward(c, c->sc.ids, B, false, dev_out);
 }
 
@@ -600,10 +690,8 @@ pac_status pac_gather(pac_ctx* c, const int* sample_ids, int B, void* dev_out) {
 static pac_status epoch_common(pac_ctx* c, const int* d_perm, long long n, int B, const pac_adamw* hp, float* d_losses) {
     for (long long s = 0; s < n / B; ++s) {
         const int* ids = d_perm + s * B;
-        pac_status st = forward(c, ids, B, true, nullptr);
+        pac_status st = train_enqueue(c, ids, B, d_losses ? d_losses + s : c->sc.loss, hp);
         if (st != PAC_OK) return st;
-        if ((st = backward(c, ids, B, d_losses ? d_losses + s : c->sc.loss)) != PAC_OK) return st;
-        if ((st = adam_enqueue(c, hp)) != PAC_OK) return st;
     }
     return PAC_OK;
 }

@@ -1,0 +1,348 @@
+// The part of a classifier-head train step that sits between the two passes over the
+// cache, fused into one kernel, and the gradient finalisation (+ AdamW) fused into another.
+//
+// mid_cls_kernel: one thread-block cluster per batch sample.  From the down-projections
+// u_l it runs the lambda-merge / adapter-body chain (Section IV-A) for all layers keeping
+// what the reverse pass needs (u_l - a_{l-1} and the ReLU mask) in registers, pools a_L over
+// the sample's tokens through distributed shared memory, evaluates head, loss and their
+// gradients for the sample, and walks the chain backwards to emit du_l (bf16 or fp32) and
+// per-block partial sums of dlambda_l.  Nothing but u is read and nothing but du and a few
+// per-sample vectors is written.
+//
+// All cross-thread sums use a fixed order, so results are bit-reproducible.
+#pragma once
+#include <cooperative_groups.h>
+
+#include "pac_common.cuh"
+#include "pac_simt.cuh"
+
+namespace pac {
+
+namespace cg = cooperative_groups;
+
+struct MidParams {
+    const int* ids; long long N; const int* labels;
+    int L, S, d, r, C, B;
+    int G;                      // cluster size: CTAs per sample
+    int Sg;                     // tokens per CTA = ceil(S / G)
+    int dg;                     // head columns per CTA = ceil(d / G)
+    int train;
+    const float* u; long long lstride;
+    const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
+    void* du;                   // [L][max_rows][r] bf16 or fp32
+    float* pooled_a;            // [B][r]
+    float* pooled_y;            // [B][d]
+    float* gvec;                // [B][d]
+    float* dlogits;             // [B][C]
+    float* loss_b;              // [B]
+    float* lam_part;            // [L][B*G]
+    float* logits_out;          // [B][C] (train: scratch copy; eval: caller's buffer)
+    unsigned* status;
+};
+
+constexpr int MID_MAX_C = 32;
+
+template <int ACT, int LT, typename DU>
+__global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int q = (int)cluster.block_rank();
+    const int b = blockIdx.x / p.G;
+    const int t = threadIdx.x, nt = blockDim.x;
+    const int r = p.r, L = p.L, C = p.C;
+    const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
+
+    extern __shared__ float sm[];
+    float* aL = sm;                              // [Sg][r]   a_L of this CTA's tokens
+    float* colsum = aL + (size_t)p.Sg * r;       // [r]       exchanged through DSMEM
+    float* lpart = colsum + r;                   // [MID_MAX_C] exchanged
+    float* dpart = lpart + MID_MAX_C;            // [r]       exchanged
+    float* pooled = dpart + r;                   // [r]
+    float* daL = pooled + r;                     // [r]
+    float* py = daL + r;                         // [dg]
+    float* gk = py + p.dg;                       // [dg]
+    float* lg = gk + p.dg;                       // [MID_MAX_C] logits, then dlogits
+    float* lam_s = lg + MID_MAX_C;               // [LT]
+    float* red = lam_s + LT;                     // [32]
+    float* lred = red + 32;                      // [nwarps][LT]
+
+    const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
+    if (t < LT) lam_s[t] = t < L ? p.lam[t] : 0.f;
+    __syncthreads();
+
+    // ---- forward chain: thread owns 4 consecutive adapter columns of one token ----
+    const int groups_per_tok = r >> 2;
+    const int s_local = t / groups_per_tok, j4 = (t - s_local * groups_per_tok) << 2;
+    const int s = q * p.Sg + s_local;
+    const bool live = s_local < p.Sg && s < p.S;
+    const long long base = ((long long)b * p.S + s) * r + j4;
+    float w[LT][4];
+    unsigned mask[4] = {0u, 0u, 0u, 0u};
+    float ap[4] = {0.f, 0.f, 0.f, 0.f};                 // a_0 = 0
+#pragma unroll
+    for (int l = 0; l < LT; ++l) {
+        if (l < L) {
+            float4 uu = live ? *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base) : make_float4(0, 0, 0, 0);
+            const float uv[4] = {uu.x, uu.y, uu.z, uu.w};
+            const float lm = lam_s[l];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float z = lm * uv[e] + (1.f - lm) * ap[e];
+                w[l][e] = uv[e] - ap[e];                     // d z_l / d lambda_l
+                if (ACT == PAC_ACT_RELU) {
+                    const bool on = z > 0.f;
+                    mask[e] |= (on ? 1u : 0u) << l;
+                    ap[e] = on ? z : 0.f;
+                } else {
+                    ap[e] = z;
+                }
+            }
+        }
+    }
+    if (s_local < p.Sg) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) aL[(size_t)s_local * r + j4 + e] = live ? ap[e] : 0.f;
+    }
+    __syncthreads();
+    // column sums over this CTA's tokens, in token order
+    for (int j = t; j < r; j += nt) {
+        float acc = 0.f;
+        for (int sl = 0; sl < p.Sg; ++sl) acc += aL[(size_t)sl * r + j];
+        colsum[j] = acc;
+    }
+    cluster.sync();
+    for (int j = t; j < r; j += nt) {
+        float acc = 0.f;
+        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(colsum, g)[j];
+        pooled[j] = acc / (float)p.S;                     // mean_s a_L
+    }
+    __syncthreads();
+
+    // ---- head on this CTA's slice of the hidden width ----
+    const int k0 = q * p.dg, kn = min(p.dg, p.d - k0);     // kn may be <= 0 for the last ranks
+    for (int kk = t; kk < kn; kk += nt) {
+        const int k = k0 + kk;
+        float acc = 0.f;
+        for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], p.W_up[(long long)j * p.d + k], acc);
+        py[kk] = p.hbar[id * p.d + k] + acc;              // mean_s y = mean_s h_L + (mean_s a_L) W_up
+    }
+    __syncthreads();
+    for (int c = 0; c < C; ++c) {
+        float part = 0.f;
+        for (int kk = t; kk < kn; kk += nt) part = fmaf(py[kk], p.W_head[(long long)(k0 + kk) * C + c], part);
+        const float tot = block_sum(part, red);
+        if (t == 0) lpart[c] = tot;
+    }
+    cluster.sync();
+    if (t < C) {
+        float acc = p.b_head[t];
+        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(lpart, g)[t];
+        lg[t] = acc;
+        if (q == 0) p.logits_out[(long long)b * C + t] = acc;
+    }
+    __syncthreads();
+    if (!p.train) {
+        cluster.sync();                                   // peers may still be reading this CTA's shared memory
+        return;
+    }
+    {
+        float mx = -INFINITY;
+        for (int c = 0; c < C; ++c) mx = fmaxf(mx, lg[c]);
+        float se = 0.f;
+        for (int c = 0; c < C; ++c) se += expf(lg[c] - mx);
+        const int label = p.labels[id];
+        const float my = (t < C) ? (expf(lg[t] - mx) / se - (t == label ? 1.f : 0.f)) / (float)p.B : 0.f;
+        if (t == 0 && q == 0) p.loss_b[b] = mx + logf(se) - lg[label];
+        __syncthreads();
+        if (t < C) {
+            lg[t] = my;                                   // dlogits
+            if (q == 0) p.dlogits[(long long)b * C + t] = my;
+        }
+        __syncthreads();
+    }
+    for (int kk = t; kk < kn; kk += nt) {
+        const int k = k0 + kk;
+        float acc = 0.f;
+        for (int c = 0; c < C; ++c) acc = fmaf(p.W_head[(long long)k * C + c], lg[c], acc);
+        gk[kk] = acc;                                     // d loss / d mean_s y
+        p.gvec[(long long)b * p.d + k] = acc;
+        p.pooled_y[(long long)b * p.d + k] = py[kk];
+    }
+    if (q == 0)
+        for (int j = t; j < r; j += nt) p.pooled_a[(long long)b * r + j] = pooled[j];
+    __syncthreads();
+    for (int j = warp; j < r; j += nwarps) {
+        float part = 0.f;
+        for (int kk = lane; kk < kn; kk += 32) part = fmaf(p.W_up[(long long)j * p.d + k0 + kk], gk[kk], part);
+        part = warp_sum(part);
+        if (lane == 0) dpart[j] = part;
+    }
+    cluster.sync();
+    for (int j = t; j < r; j += nt) {
+        float acc = 0.f;
+        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(dpart, g)[j];
+        daL[j] = acc / (float)p.S;                         // da_L, the same for every token of the sample
+    }
+    __syncthreads();
+
+    // ---- reverse chain from registers ----
+    float da[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) da[e] = live ? daL[j4 + e] : 0.f;
+    DU* du = reinterpret_cast<DU*>(p.du);
+#pragma unroll
+    for (int l = LT - 1; l >= 0; --l) {
+        if (l < L) {
+            const float lm = lam_s[l];
+            float part = 0.f, dv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float dz = (ACT == PAC_ACT_RELU) ? (((mask[e] >> l) & 1u) ? da[e] : 0.f) : da[e];
+                part = fmaf(dz, w[l][e], part);
+                dv[e] = lm * dz;                           // du_l
+                da[e] = (1.f - lm) * dz;                   // da_{l-1}
+            }
+            if (live) {
+                DU* dst = du + (long long)l * p.lstride + base;
+                if constexpr (sizeof(DU) == 2) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<unsigned*>(&lo);
+                    pk.y = *reinterpret_cast<unsigned*>(&hi);
+                    *reinterpret_cast<uint2*>(dst) = pk;
+                } else {
+                    *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+                }
+            }
+            part = warp_sum(part);
+            if (lane == 0) lred[warp * LT + l] = part;
+        }
+    }
+    __syncthreads();
+    if (t < L) {
+        float acc = 0.f;
+        for (int wv = 0; wv < nwarps; ++wv) acc += lred[wv * LT + t];
+        p.lam_part[(long long)t * (p.B * p.G) + blockIdx.x] = acc;
+    }
+    cluster.sync();                                       // keep shared memory alive until every peer has read it
+}
+
+// ---------------------------------------------------------------------------
+// Gradient finalisation for the classifier head, one thread per flat parameter index:
+//   W_down : sum of the row-split partials of h^T du (split order), or already final
+//   lambda : sum of per-block partials (block order)
+//   W_up   : pooled_a^T g        W_head : pooled_y^T dlogits        b_head : sum_b dlogits
+// plus the mean loss.  With adam != 0 the AdamW update of the same element follows at once.
+// ---------------------------------------------------------------------------
+struct FinalizeParams {
+    ParamLayout lay;
+    int B, d, r, C, L;
+    const float* dw_part; int splits; long long dw_elems;     // splits <= 1: W_down gradient already in grads
+    const float* lam_part; int lam_blocks;
+    const float *pooled_a, *gvec, *pooled_y, *dlogits, *loss_b;
+    float* grads; float* loss_out;
+    // AdamW
+    int adam;
+    float *params, *m, *v;
+    pac_adamw hp; float bc1, bc2;
+    bf16* wdT;                                               // [L][2][r][d] bf16 hi/lo shadow of W_down (may be null)
+};
+
+__global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const ParamLayout& lay = f.lay;
+    if (i == 0) {
+        float acc = 0.f;
+        for (int b = 0; b < f.B; ++b) acc += f.loss_b[b];
+        *f.loss_out = acc / (float)f.B;
+    }
+    if (i >= lay.total) return;
+    float g;
+    if (i < lay.lam) {
+        if (f.splits > 1) {
+            g = f.dw_part[i];
+            for (int j = 1; j < f.splits; ++j) g += f.dw_part[(long long)j * f.dw_elems + i];
+        } else {
+            g = f.grads[i];
+        }
+    } else if (i < lay.w_up) {
+        const int l = (int)(i - lay.lam);
+        g = 0.f;
+        for (int k = 0; k < f.lam_blocks; ++k) g += f.lam_part[(long long)l * f.lam_blocks + k];
+    } else if (i < lay.w_head) {
+        const long long e = i - lay.w_up;
+        const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
+        g = 0.f;
+        for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], f.gvec[(long long)b * f.d + k], g);
+    } else if (i < lay.b_head) {
+        const long long e = i - lay.w_head;
+        const int k = (int)(e / f.C), c = (int)(e - (long long)k * f.C);
+        g = 0.f;
+        for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_y[(long long)b * f.d + k], f.dlogits[(long long)b * f.C + c], g);
+    } else {
+        const int c = (int)(i - lay.b_head);
+        g = 0.f;
+        for (int b = 0; b < f.B; ++b) g += f.dlogits[(long long)b * f.C + c];
+    }
+    f.grads[i] = g;
+    if (f.adam) adamw_element(f.params, f.m, f.v, i, g, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+}
+
+// Shape test and launch geometry of the fused kernel: G CTAs per sample, one 4-column
+// group per thread, chain state in registers.
+struct MidPlan {
+    bool ok = false;
+    int G = 1, Sg = 0, dg = 0, threads = 0, LT = 0;
+    size_t smem = 0;
+};
+
+inline MidPlan mid_plan(const Dims& dm) {
+    MidPlan mp;
+    if (dm.r % 4 != 0 || dm.C > MID_MAX_C || dm.L > 32) return mp;
+    mp.LT = dm.L <= 8 ? 8 : dm.L <= 16 ? 16 : dm.L <= 24 ? 24 : 32;
+    const int max_threads = mp.LT <= 16 ? 512 : 256;          // register budget: 4*LT state values per thread
+    for (int G = 1; G <= 8; G *= 2) {
+        const int Sg = (dm.S + G - 1) / G;
+        const long long need = (long long)Sg * (dm.r / 4);
+        if (need <= max_threads) {
+            mp.G = G; mp.Sg = Sg; mp.dg = (dm.d + G - 1) / G;
+            int th = (int)((need + 31) / 32 * 32);
+            if (th < 128) th = 128;
+            mp.threads = th;
+            mp.smem = sizeof(float) * ((size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)mp.dg + 2 * MID_MAX_C + mp.LT + 32 +
+                                       (size_t)(th / 32) * mp.LT);
+            mp.ok = true;
+            return mp;
+        }
+    }
+    return mp;
+}
+
+template <int ACT, typename DU>
+inline cudaError_t mid_launch_lt(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.B * mp.G), 1, 1);
+    cfg.blockDim = dim3((unsigned)mp.threads, 1, 1);
+    cfg.dynamicSmemBytes = mp.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)mp.G;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    switch (mp.LT) {
+        case 8: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 8, DU>, p);
+        case 16: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 16, DU>, p);
+        case 24: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 24, DU>, p);
+        default: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 32, DU>, p);
+    }
+}
+
+inline cudaError_t mid_launch(const MidPlan& mp, const MidParams& p, int act, bool du_bf16, cudaStream_t stream) {
+    if (act == PAC_ACT_RELU)
+        return du_bf16 ? mid_launch_lt<PAC_ACT_RELU, bf16>(mp, p, stream) : mid_launch_lt<PAC_ACT_RELU, float>(mp, p, stream);
+    return du_bf16 ? mid_launch_lt<PAC_ACT_IDENTITY, bf16>(mp, p, stream) : mid_launch_lt<PAC_ACT_IDENTITY, float>(mp, p, stream);
+}
+
+}  // namespace pac

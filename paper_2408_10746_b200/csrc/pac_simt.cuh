@@ -144,19 +144,20 @@ struct StorePlusLastLayer {            // y = h_L + a_L W_up
 
 // ---------------------------------------------------------------------------
 // The lambda-merge / adapter-body chain over saved u (forward) and its reverse.
-// One thread per (row, column) element e of the [M][r] state; stride = M*r.
+// One thread per (row, column) element e < n = M*r of the [M][r] state; layer l of a
+// saved stack starts at l * lstride (lstride = max_rows * r, fixed per context).
 // ---------------------------------------------------------------------------
 template <int ACT>
 __global__ void chain_fwd_kernel(const float* __restrict__ u, float* __restrict__ a, const float* __restrict__ lam,
-                                 int L, long long stride) {
+                                 int L, long long n, long long lstride) {
     long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= stride) return;
+    if (e >= n) return;
     float prev = 0.f;                                   // a_0 = 0
     for (int l = 0; l < L; ++l) {
         float lm = lam[l];
-        float z = lm * u[l * stride + e] + (1.f - lm) * prev;
+        float z = lm * u[l * lstride + e] + (1.f - lm) * prev;
         prev = (ACT == PAC_ACT_RELU) ? (z > 0.f ? z : 0.f) : z;
-        a[l * stride + e] = prev;
+        a[l * lstride + e] = prev;
     }
 }
 
@@ -333,11 +334,11 @@ template <int ACT, typename DU>
 __global__ void __launch_bounds__(256) chain_bwd_kernel(const float* __restrict__ u, const float* __restrict__ a,
                                                         const float* __restrict__ lam,
                                                         const float* __restrict__ daL, int per_sample, int S,
-                                                        int r, int L, long long stride, DU* __restrict__ du,
-                                                        float* __restrict__ lam_part) {
+                                                        int r, int L, long long n, long long stride,
+                                                        DU* __restrict__ du, float* __restrict__ lam_part) {
     __shared__ float red[32];
     long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool live = e < stride;
+    const bool live = e < n;
     float da = 0.f;
     if (live) {
         if (per_sample) {
@@ -413,38 +414,53 @@ __global__ void mean_kernel(const float* __restrict__ x, int n, float* __restric
 
 // ---------------------------------------------------------------------------
 // Fused AdamW over the flat parameter vector (decoupled decay on the weight matrices
-// only).  inv_bc1 = 1/(1-beta1^t), inv_bc2 = 1/(1-beta2^t).  Also refreshes the bf16
-// transposed shadow of W_down ([L][r][d]) that the tensor-core path multiplies with.
+// only).  bc1 = 1-beta1^t, bc2 = 1-beta2^t (bias corrections, computed on the host in double).  Also refreshes the bf16
+// transposed hi/lo shadow of W_down ([L][2][r][d]) that the tensor-core path multiplies with.
 // ---------------------------------------------------------------------------
-__global__ void adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
-                             float* __restrict__ v, long long n, ParamLayout lay, pac_adamw hp, float inv_bc1,
-                             float inv_bc2, bf16* __restrict__ wdT, int d, int r) {
-    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
+// One element of the update, shared by every kernel that applies AdamW so that fused and
+// separate updates are bit-identical.
+__device__ __forceinline__ void adamw_element(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
+                                              long long i, float gi, const ParamLayout& lay, const pac_adamw& hp,
+                                              float bc1, float bc2, bf16* __restrict__ wdT, int d, int r) {
     const bool decays = (i < lay.lam) || (i >= lay.w_up && i < lay.b_head);
-    float gi = g[i], th = p[i];
-    float mi = hp.beta1 * m[i] + (1.f - hp.beta1) * gi;
-    float vi = hp.beta2 * v[i] + (1.f - hp.beta2) * gi * gi;
+    float th = p[i];
+    // every rounding is spelled out (no contraction into FMAs), in the order the update is written:
+    // m = b1 m + (1-b1) g;  v = b2 v + ((1-b2) g) g;  theta = (theta - lr wd theta) - (lr mhat)/(sqrt(vhat)+eps)
+    const float mi = __fadd_rn(__fmul_rn(hp.beta1, m[i]), __fmul_rn(__fsub_rn(1.f, hp.beta1), gi));
+    const float vi = __fadd_rn(__fmul_rn(hp.beta2, v[i]), __fmul_rn(__fmul_rn(__fsub_rn(1.f, hp.beta2), gi), gi));
     m[i] = mi;
     v[i] = vi;
-    float mhat = mi * inv_bc1, vhat = vi * inv_bc2;
-    float decay = decays ? hp.lr * hp.weight_decay * th : 0.f;
-    th = th - decay - hp.lr * mhat / (sqrtf(vhat) + hp.eps);
+    const float mhat = __fdiv_rn(mi, bc1), vhat = __fdiv_rn(vi, bc2);
+    const float decay = decays ? __fmul_rn(__fmul_rn(hp.lr, hp.weight_decay), th) : 0.f;
+    th = __fsub_rn(__fsub_rn(th, decay), __fdiv_rn(__fmul_rn(hp.lr, mhat), __fadd_rn(__fsqrt_rn(vhat), hp.eps)));
     p[i] = th;
     if (wdT && i < lay.lam) {
-        long long l = i / ((long long)d * r), rem = i - l * (long long)d * r;
-        int k = rem / r, j = rem - (long long)k * r;
-        wdT[(l * r + j) * (long long)d + k] = __float2bfloat16(th);
+        const long long dr = (long long)d * r, l = i / dr, rem = i - l * dr;
+        const int k = (int)(rem / r), j = (int)(rem - (long long)k * r);
+        const bf16 hi = __float2bfloat16(th);
+        wdT[((l * 2 + 0) * r + j) * (long long)d + k] = hi;
+        wdT[((l * 2 + 1) * r + j) * (long long)d + k] = __float2bfloat16(th - __bfloat162float(hi));
     }
 }
 
-// bf16 transposed shadow of W_down from the fp32 master: wdT[l][j][k] = W_down[l][k][j].
+__global__ void adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
+                             float* __restrict__ v, long long n, ParamLayout lay, pac_adamw hp, float bc1,
+                             float bc2, bf16* __restrict__ wdT, int d, int r) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    adamw_element(p, m, v, i, g[i], lay, hp, bc1, bc2, wdT, d, r);
+}
+
+// bf16 transposed hi/lo shadow of W_down from the fp32 master:
+// wdT[l][0][j][k] = bf16(W_down[l][k][j]), wdT[l][1][j][k] = bf16(W_down[l][k][j] - hi).
 __global__ void shadow_wdown_kernel(const float* __restrict__ w, bf16* __restrict__ wdT, int L, int d, int r) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)L * d * r) return;
     long long l = i / ((long long)d * r), rem = i - l * (long long)d * r;
     int k = rem / r, j = rem - (long long)k * r;
-    wdT[(l * r + j) * (long long)d + k] = __float2bfloat16(w[i]);
+    const bf16 hi = __float2bfloat16(w[i]);
+    wdT[((l * 2 + 0) * r + j) * (long long)d + k] = hi;
+    wdT[((l * 2 + 1) * r + j) * (long long)d + k] = __float2bfloat16(w[i] - __bfloat162float(hi));
 }
 
 }  // namespace pac

@@ -239,3 +239,112 @@ def test_device_resident_bad_id_is_clamped_and_reported(tiny):
     assert e.value.status_name == "PAC_ERR_SAMPLE_ID_RANGE"
     ctx.sync()                                              # the report is one-shot
     assert np.isfinite(ctx.get_params()).all()
+
+
+# ------------------------------------------------------------------ tensor-core path (bf16 caches)
+TC_BASE = pi.CacheSpec("tc_full_tiles", N=16, L=3, S=128, d=256, dtype="bf16", r=64, n_out=3, B=4)
+TC_SPECS = [
+    (TC_BASE, 4, 0),
+    (TC_BASE.scaled(name="tc_ragged", S=150, d=200, r=48, B=3), 5, 0),      # ragged S and d, B < max_batch
+    (TC_BASE.scaled(name="tc_small_S", S=19, d=72, r=16), 4, 0),            # one tile larger than a sample
+    (TC_BASE.scaled(name="tc_r128", S=256, d=1024, r=128, L=2), 4, 0),      # two 64-column blocks of du
+    (TC_BASE.scaled(name="tc_r256", S=64, d=320, r=256, L=2, B=2), 2, 0),   # widest adapter the path takes
+    (TC_BASE.scaled(name="tc_identity", S=64, d=512, r=32, L=4, B=2), 2, 1),
+    (TC_BASE.scaled(name="tc_deep", S=32, d=128, r=32, L=30, B=3, N=8), 3, 0),
+]
+
+
+def tc_check(spec, max_batch, act, ids=None, loss_tol=2e-2, chain_tol=1e-2, head_tol=2e-3, case=None):
+    case = case or Case(spec)
+    ids = ids or [spec.N - 1, 0, 5, 5][:spec.B]
+    ctx = case.context(max_batch=max_batch, act=act)
+    assert ctx.kernel_path() == "tensor"
+    flat = pi.random_params(spec, 3)
+    ctx.set_params(flat)
+    loss = ctx.train_step(ids)
+    ctx.sync()
+    g = ctx.get_grads()
+    ref_loss, ref_g, _ = case.oracle_loss_grads(flat, ids, act)
+    assert abs(loss - ref_loss) <= loss_tol * abs(ref_loss)
+    ref = po.flatten(ref_g)
+    for name, sl in block_slices(spec).items():
+        tol = chain_tol if name in ("W_down", "lam") else head_tol
+        assert np.linalg.norm(ref[sl]) > 0
+        assert rel_l2(g[sl], ref[sl]) < tol, (name, rel_l2(g[sl], ref[sl]))
+    return ctx, case
+
+
+@pytest.mark.parametrize("spec,max_batch,act", TC_SPECS, ids=[s[0].name for s in TC_SPECS])
+def test_tensor_path_loss_and_gradients(spec, max_batch, act):
+    """bf16 cache through TMA + tcgen05: loss within 2e-2; the gradients that pass through the
+    ReLU masks (W_down, lambda) within 1e-2 relative L2 (du is rounded to bf16 and a few masks
+    flip), the head-side blocks within 2e-3."""
+    tc_check(spec, max_batch, act)
+
+
+def test_tensor_path_eval_and_determinism():
+    case = Case(TC_BASE)
+    flat = pi.random_params(TC_BASE, 4)
+    outs, grads = [], []
+    for _ in range(2):
+        ctx = case.context()
+        ctx.set_params(flat)
+        out = torch.zeros((4, 3), dtype=torch.float32, device="cuda")
+        ctx.eval_logits([1, 2, 3, 4], out)
+        ctx.train_step([1, 2, 3, 4])
+        grads.append(ctx.get_grads())
+        outs.append(out.cpu().numpy())
+    ref = po.eval_logits(case.oracle_params(flat), case.H([1, 2, 3, 4]), 0)
+    assert rel_l2(outs[0], ref) < 1e-3
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(grads[0], grads[1])    # fixed summation orders
+
+
+def test_tensor_path_ten_steps_t5_base_shape():
+    """T5-Base layer shape (L=12, S=128, d=768, r=64) on a short cache: 10 AdamW steps from the
+    seeded initial state; loss within 2e-2, parameter vector within 1e-2 relative L2."""
+    spec = pi.CONFIGS["t5_base"].scaled(N=96, B=8, name="t5_base_short")
+    case = Case(spec, materialize_cpu=False)
+    ctx, losses, ref_losses, p, ref_p, p0 = run_trajectory(case, 10)
+    assert ctx.kernel_path() == "tensor"
+    assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses))
+    assert rel_l2(p, ref_p) < 1e-2
+    assert rel_l2(p - p0, ref_p - p0) < 0.1          # the update itself is reproduced, not only the initial values
+
+
+# ------------------------------------------------------------------ full-size launch configurations
+class SparseCase(Case):
+    """A cache of the full size and strides whose slabs are filled only for the sample ids a
+    test touches (the rest stays zero), so full-size launch geometry costs seconds, not minutes."""
+
+    def __init__(self, spec, ids, seed=0):
+        self.spec, self.seed = spec, seed
+        self.cache = torch.zeros((spec.N, spec.L, spec.S, spec.d), dtype=spec.torch_dtype, device="cuda")
+        uniq = sorted(set(ids))
+        for i in range(0, len(uniq), 8):
+            chunk = uniq[i:i + 8]
+            self.cache[chunk] = pi.cache_samples(spec, seed, chunk, "cuda")
+        self.labels = pi.labels(spec, seed, "cuda")
+        self.lm = pi.lm_head(spec, seed, "cuda") if spec.head == "lm" else None
+        self.labels_np = pi.labels(spec, seed, "cpu").numpy().astype(np.int64)
+        self.lm_np = pi.lm_head(spec, seed, "cpu").float().numpy() if spec.head == "lm" else None
+        self.cache_np = None
+
+
+@pytest.mark.parametrize("name", ["t5_base", "bart_large", "t5_large"])
+def test_full_size_step_matches_oracle(name):
+    """One train step in the benchmark's launch configuration (full N, L, S, d, r, B) on a
+    shuffled minibatch that includes the first and the last sample of the cache."""
+    spec = pi.CONFIGS[name]
+    free, _ = torch.cuda.mem_get_info()
+    if spec.cache_bytes + (6 << 30) > free:
+        pytest.skip("cache does not fit this device")
+    ids = pi.epoch_permutation(spec.N, 2)[:spec.B].tolist()
+    ids[0], ids[-1] = 0, spec.N - 1
+    case = SparseCase(spec, ids)
+    ctx, _ = tc_check(spec, spec.B, 0, ids=ids, case=case)
+    # gather of the same ids, bit-exact, from the full-size cache
+    out = torch.empty((spec.L, 4, spec.S, spec.d), dtype=spec.torch_dtype, device="cuda")
+    ctx.gather(ids[:4], out)
+    ctx.sync()
+    ref = pi.cache_samples(spec, 0, ids[:4], "cpu").permute(1, 0, 2, 3).contiguous()
+    assert out.cpu().view(torch.uint8).flatten().equal(ref.view(torch.uint8).flatten())
