@@ -39,7 +39,7 @@ struct Scratch {
     float* lm_logits = nullptr;    // [M][V]
     float* dy = nullptr;           // [M][d]
     // tensor path
-    bf16* wdT = nullptr;           // [L][2][r][d] bf16 hi/lo shadow of W_down, transposed
+    bf16* wdT = nullptr;           // [L][2][d][r] bf16 hi/lo shadow of W_down
     float* dw_part = nullptr;      // split partials of dW_down
 };
 
@@ -376,6 +376,7 @@ pac_status mid_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d
     p.ids = d_ids; p.N = dm.N; p.labels = c->labels;
     p.L = dm.L; p.S = dm.S; p.d = dm.d; p.r = dm.r; p.C = dm.C; p.B = B;
     p.G = c->mplan.G; p.Sg = c->mplan.Sg; p.dg = c->mplan.dg; p.train = train ? 1 : 0;
+    p.scratch = c->mplan.scratch; p.wup_smem = c->mplan.wup_smem; p.u_smem = c->mplan.u_smem;
     p.u = sc.u; p.lstride = (long long)c->max_rows * dm.r;
     p.lam = c->params + c->lay.lam; p.W_up = c->params + c->lay.w_up;
     p.W_head = c->params + c->lay.w_head; p.b_head = c->params + c->lay.b_head; p.hbar = sc.hbar;
@@ -413,7 +414,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         bias_corrections(hp, c->step, &f.bc1, &f.bc2);
         f.wdT = sc.wdT;
     }
-    finalize_cls_kernel<<<cdiv(c->lay.total, 256), 256, 0, c->stream>>>(f);
+    finalize_cls_kernel<<<cdiv(c->lay.total, 256) + 1, 256, 0, c->stream>>>(f);    // + one block for lambda and the loss
     LAUNCH_CHECK(c);
     return PAC_OK;
 }

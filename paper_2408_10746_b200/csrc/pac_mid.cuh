@@ -27,6 +27,9 @@ struct MidParams {
     int Sg;                     // tokens per CTA = ceil(S / G)
     int dg;                     // head columns per CTA = ceil(d / G)
     int train;
+    int scratch;                // floats of block-local reduction scratch
+    int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
+    int u_smem;                 // 1: every thread's u values are prefetched into shared memory
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
     void* du;                   // [L][max_rows][r] bf16 or fp32
@@ -42,6 +45,16 @@ struct MidParams {
 
 constexpr int MID_MAX_C = 32;
 
+__device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 template <int ACT, int LT, typename DU>
 __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams p) {
     cg::cluster_group cluster = cg::this_cluster();
@@ -51,37 +64,54 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
     const int r = p.r, L = p.L, C = p.C;
     const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
 
-    extern __shared__ float sm[];
+    extern __shared__ float4 sm4[];
+    float4* u_s = sm4;                           // [L][nt] each thread's own u values (when p.u_smem)
+    float* sm = reinterpret_cast<float*>(sm4 + (p.u_smem ? (size_t)L * nt : 0));
     float* aL = sm;                              // [Sg][r]   a_L of this CTA's tokens
     float* colsum = aL + (size_t)p.Sg * r;       // [r]       exchanged through DSMEM
     float* lpart = colsum + r;                   // [MID_MAX_C] exchanged
     float* dpart = lpart + MID_MAX_C;            // [r]       exchanged
     float* pooled = dpart + r;                   // [r]
     float* daL = pooled + r;                     // [r]
-    float* py = daL + r;                         // [dg]
+    float* py = daL + r;                         // [dg]  hbar slice, then mean_s y
     float* gk = py + p.dg;                       // [dg]
     float* lg = gk + p.dg;                       // [MID_MAX_C] logits, then dlogits
     float* lam_s = lg + MID_MAX_C;               // [LT]
-    float* red = lam_s + LT;                     // [32]
-    float* lred = red + 32;                      // [nwarps][LT]
+    float* wh_s = lam_s + LT;                    // [dg][C] slice of W_head
+    float* lred = wh_s + (size_t)p.dg * C;       // [nwarps][LT]; also [nwarps][MID_MAX_C] and [parts][r] scratch
+    float* wup_s = lred + (size_t)p.scratch;     // [r][dg] slice of W_up (when p.wup_smem)
 
-    const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
-    if (t < LT) lam_s[t] = t < L ? p.lam[t] : 0.f;
-    __syncthreads();
-
-    // ---- forward chain: thread owns 4 consecutive adapter columns of one token ----
+    // ---- everything this CTA will read from global memory is requested up front ----
     const int groups_per_tok = r >> 2;
     const int s_local = t / groups_per_tok, j4 = (t - s_local * groups_per_tok) << 2;
     const int s = q * p.Sg + s_local;
     const bool live = s_local < p.Sg && s < p.S;
     const long long base = ((long long)b * p.S + s) * r + j4;
+    if (p.u_smem && live)
+        for (int l = 0; l < L; ++l) cp_async_16(u_s + (size_t)l * nt + t, p.u + (long long)l * p.lstride + base);
+    cp_async_commit();                                                          // group: u
+    const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
+    const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
+    for (int kk = t; kk < kn; kk += nt) cp_async_4(py + kk, p.hbar + id * p.d + k0 + kk);
+    for (int e = t; e < kn * C; e += nt) cp_async_4(wh_s + e, p.W_head + (long long)k0 * C + e);
+    if (p.wup_smem)
+        for (int j = warp; j < r; j += nwarps)
+            for (int kk = lane; kk < kn; kk += 32) cp_async_4(wup_s + (size_t)j * p.dg + kk, p.W_up + (long long)j * p.d + k0 + kk);
+    cp_async_commit();                                                          // group: head operands
+    const int label = p.train ? p.labels[id] : 0;
+    if (t < LT) lam_s[t] = t < L ? p.lam[t] : 0.f;
+    __syncthreads();
+    cp_async_wait_group<1>();                                                   // own u values have landed
+
+    // ---- forward chain: thread owns 4 consecutive adapter columns of one token ----
     float w[LT][4];
     unsigned mask[4] = {0u, 0u, 0u, 0u};
     float ap[4] = {0.f, 0.f, 0.f, 0.f};                 // a_0 = 0
 #pragma unroll
     for (int l = 0; l < LT; ++l) {
         if (l < L) {
-            float4 uu = live ? *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base) : make_float4(0, 0, 0, 0);
+            float4 uu = make_float4(0, 0, 0, 0);
+            if (live) uu = p.u_smem ? u_s[(size_t)l * nt + t] : *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base);
             const float uv[4] = {uu.x, uu.y, uu.z, uu.w};
             const float lm = lam_s[l];
 #pragma unroll
@@ -103,11 +133,23 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
         for (int e = 0; e < 4; ++e) aL[(size_t)s_local * r + j4 + e] = live ? ap[e] : 0.f;
     }
     __syncthreads();
-    // column sums over this CTA's tokens, in token order
-    for (int j = t; j < r; j += nt) {
-        float acc = 0.f;
-        for (int sl = 0; sl < p.Sg; ++sl) acc += aL[(size_t)sl * r + j];
-        colsum[j] = acc;
+    // column sums over this CTA's tokens: `parts` partial sums per column over contiguous token
+    // ranges, then added in range order
+    {
+        const int parts = max(1, min(nt / r, p.Sg));
+        const int per = (p.Sg + parts - 1) / parts;
+        if (t < parts * r) {
+            const int j = t % r, part = t / r;
+            float acc = 0.f;
+            for (int sl = part * per; sl < min(p.Sg, (part + 1) * per); ++sl) acc += aL[(size_t)sl * r + j];
+            lred[part * r + j] = acc;
+        }
+        __syncthreads();
+        if (t < r) {
+            float acc = 0.f;
+            for (int part = 0; part < parts; ++part) acc += lred[part * r + t];
+            colsum[t] = acc;
+        }
     }
     cluster.sync();
     for (int j = t; j < r; j += nt) {
@@ -115,22 +157,32 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
         for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(colsum, g)[j];
         pooled[j] = acc / (float)p.S;                     // mean_s a_L
     }
+    cp_async_wait_group<0>();
     __syncthreads();
 
     // ---- head on this CTA's slice of the hidden width ----
-    const int k0 = q * p.dg, kn = min(p.dg, p.d - k0);     // kn may be <= 0 for the last ranks
     for (int kk = t; kk < kn; kk += nt) {
-        const int k = k0 + kk;
         float acc = 0.f;
-        for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], p.W_up[(long long)j * p.d + k], acc);
-        py[kk] = p.hbar[id * p.d + k] + acc;              // mean_s y = mean_s h_L + (mean_s a_L) W_up
+        if (p.wup_smem) {
+#pragma unroll 8
+            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], wup_s[(size_t)j * p.dg + kk], acc);
+        } else {
+            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], p.W_up[(long long)j * p.d + k0 + kk], acc);
+        }
+        py[kk] += acc;                                    // mean_s y = mean_s h_L + (mean_s a_L) W_up
     }
     __syncthreads();
     for (int c = 0; c < C; ++c) {
         float part = 0.f;
-        for (int kk = t; kk < kn; kk += nt) part = fmaf(py[kk], p.W_head[(long long)(k0 + kk) * C + c], part);
-        const float tot = block_sum(part, red);
-        if (t == 0) lpart[c] = tot;
+        for (int kk = t; kk < kn; kk += nt) part = fmaf(py[kk], wh_s[kk * C + c], part);
+        part = warp_sum(part);
+        if (lane == 0) lred[warp * MID_MAX_C + c] = part;
+    }
+    __syncthreads();
+    if (t < C) {
+        float acc = 0.f;
+        for (int wv = 0; wv < nwarps; ++wv) acc += lred[wv * MID_MAX_C + t];
+        lpart[t] = acc;
     }
     cluster.sync();
     if (t < C) {
@@ -149,7 +201,6 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
         for (int c = 0; c < C; ++c) mx = fmaxf(mx, lg[c]);
         float se = 0.f;
         for (int c = 0; c < C; ++c) se += expf(lg[c] - mx);
-        const int label = p.labels[id];
         const float my = (t < C) ? (expf(lg[t] - mx) / se - (t == label ? 1.f : 0.f)) / (float)p.B : 0.f;
         if (t == 0 && q == 0) p.loss_b[b] = mx + logf(se) - lg[label];
         __syncthreads();
@@ -162,7 +213,7 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
     for (int kk = t; kk < kn; kk += nt) {
         const int k = k0 + kk;
         float acc = 0.f;
-        for (int c = 0; c < C; ++c) acc = fmaf(p.W_head[(long long)k * C + c], lg[c], acc);
+        for (int c = 0; c < C; ++c) acc = fmaf(wh_s[kk * C + c], lg[c], acc);
         gk[kk] = acc;                                     // d loss / d mean_s y
         p.gvec[(long long)b * p.d + k] = acc;
         p.pooled_y[(long long)b * p.d + k] = py[kk];
@@ -172,7 +223,11 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
     __syncthreads();
     for (int j = warp; j < r; j += nwarps) {
         float part = 0.f;
-        for (int kk = lane; kk < kn; kk += 32) part = fmaf(p.W_up[(long long)j * p.d + k0 + kk], gk[kk], part);
+        if (p.wup_smem) {
+            for (int kk = lane; kk < kn; kk += 32) part = fmaf(wup_s[(size_t)j * p.dg + kk], gk[kk], part);
+        } else {
+            for (int kk = lane; kk < kn; kk += 32) part = fmaf(p.W_up[(long long)j * p.d + k0 + kk], gk[kk], part);
+        }
         part = warp_sum(part);
         if (lane == 0) dpart[j] = part;
     }
@@ -189,8 +244,10 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
 #pragma unroll
     for (int e = 0; e < 4; ++e) da[e] = live ? daL[j4 + e] : 0.f;
     DU* du = reinterpret_cast<DU*>(p.du);
+    float lpart_l[LT];                                     // this thread's share of dlambda_l
 #pragma unroll
     for (int l = LT - 1; l >= 0; --l) {
+        lpart_l[l] = 0.f;
         if (l < L) {
             const float lm = lam_s[l];
             float part = 0.f, dv[4];
@@ -201,6 +258,7 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
                 dv[e] = lm * dz;                           // du_l
                 da[e] = (1.f - lm) * dz;                   // da_{l-1}
             }
+            lpart_l[l] = part;
             if (live) {
                 DU* dst = du + (long long)l * p.lstride + base;
                 if constexpr (sizeof(DU) == 2) {
@@ -213,9 +271,16 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
                     *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
                 }
             }
-            part = warp_sum(part);
-            if (lane == 0) lred[warp * LT + l] = part;
         }
+    }
+    // warp sums of all layers together (independent shuffle chains overlap), then across warps in order
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int l = 0; l < LT; ++l) lpart_l[l] += __shfl_xor_sync(0xffffffffu, lpart_l[l], o);
+    if (lane == 0) {
+#pragma unroll
+        for (int l = 0; l < LT; ++l) lred[warp * LT + l] = lpart_l[l];
     }
     __syncthreads();
     if (t < L) {
@@ -244,19 +309,37 @@ struct FinalizeParams {
     int adam;
     float *params, *m, *v;
     pac_adamw hp; float bc1, bc2;
-    bf16* wdT;                                               // [L][2][r][d] bf16 hi/lo shadow of W_down (may be null)
+    bf16* wdT;                                               // [L][2][d][r] bf16 hi/lo shadow of W_down (may be null)
 };
 
 __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const ParamLayout& lay = f.lay;
-    if (i == 0) {
-        float acc = 0.f;
-        for (int b = 0; b < f.B; ++b) acc += f.loss_b[b];
-        *f.loss_out = acc / (float)f.B;
+    if (blockIdx.x == gridDim.x - 1) {
+        // the last block: dlambda_l (one warp per layer, lanes over the per-block partials, fixed
+        // shuffle order) and the mean loss
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+        for (int l = warp; l < f.L; l += nw) {
+            float acc = 0.f;
+            for (int k = lane; k < f.lam_blocks; k += 32) acc += f.lam_part[(long long)l * f.lam_blocks + k];
+            acc = warp_sum(acc);
+            if (lane == 0) {
+                const long long i = lay.lam + l;
+                f.grads[i] = acc;
+                if (f.adam) adamw_element(f.params, f.m, f.v, i, acc, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+            }
+        }
+        if (warp == nw - 1) {
+            float acc = 0.f;
+            for (int b = lane; b < f.B; b += 32) acc += f.loss_b[b];
+            acc = warp_sum(acc);
+            if (lane == 0) *f.loss_out = acc / (float)f.B;
+        }
+        return;
     }
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= lay.total) return;
     float g;
+    if (i >= lay.lam && i < lay.w_up) return;            // lambda is handled by the last block
     if (i < lay.lam) {
         if (f.splits > 1) {
             g = f.dw_part[i];
@@ -264,19 +347,17 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         } else {
             g = f.grads[i];
         }
-    } else if (i < lay.w_up) {
-        const int l = (int)(i - lay.lam);
-        g = 0.f;
-        for (int k = 0; k < f.lam_blocks; ++k) g += f.lam_part[(long long)l * f.lam_blocks + k];
     } else if (i < lay.w_head) {
         const long long e = i - lay.w_up;
         const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
         g = 0.f;
+#pragma unroll 8
         for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], f.gvec[(long long)b * f.d + k], g);
     } else if (i < lay.b_head) {
         const long long e = i - lay.w_head;
         const int k = (int)(e / f.C), c = (int)(e - (long long)k * f.C);
         g = 0.f;
+#pragma unroll 8
         for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_y[(long long)b * f.d + k], f.dlogits[(long long)b * f.C + c], g);
     } else {
         const int c = (int)(i - lay.b_head);
@@ -291,7 +372,7 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
 // group per thread, chain state in registers.
 struct MidPlan {
     bool ok = false;
-    int G = 1, Sg = 0, dg = 0, threads = 0, LT = 0;
+    int G = 1, Sg = 0, dg = 0, threads = 0, LT = 0, scratch = 0, wup_smem = 0, u_smem = 0;
     size_t smem = 0;
 };
 
@@ -308,13 +389,37 @@ inline MidPlan mid_plan(const Dims& dm) {
             int th = (int)((need + 31) / 32 * 32);
             if (th < 128) th = 128;
             mp.threads = th;
-            mp.smem = sizeof(float) * ((size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)mp.dg + 2 * MID_MAX_C + mp.LT + 32 +
-                                       (size_t)(th / 32) * mp.LT);
+            const int nw = th / 32;
+            int scratch = nw * mp.LT;
+            if (nw * MID_MAX_C > scratch) scratch = nw * MID_MAX_C;
+            const int parts = th / dm.r > 0 ? th / dm.r : 1;
+            if (parts * dm.r > scratch) scratch = parts * dm.r;
+            mp.scratch = scratch;
+            size_t floats = (size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)mp.dg + 2 * MID_MAX_C + mp.LT + scratch +
+                            (size_t)mp.dg * dm.C + 4;
+            const size_t budget = 200 * 1024 / sizeof(float);
+            const size_t ufl = 4 * (size_t)dm.L * th, wup = (size_t)dm.r * mp.dg;
+            mp.u_smem = floats + ufl <= budget ? 1 : 0;
+            if (mp.u_smem) floats += ufl;
+            mp.wup_smem = floats + wup <= budget ? 1 : 0;
+            if (mp.wup_smem) floats += wup;
+            mp.smem = sizeof(float) * floats;
             mp.ok = true;
             return mp;
         }
     }
     return mp;
+}
+
+template <int ACT, int LT, typename DU>
+inline cudaError_t mid_launch_one(cudaLaunchConfig_t* cfg, const MidParams& p) {
+    static size_t allowed = 0;                       // largest dynamic shared memory size already opted in to
+    if (cfg->dynamicSmemBytes > 48 * 1024 && cfg->dynamicSmemBytes > allowed) {
+        cudaError_t e = cudaFuncSetAttribute(mid_cls_kernel<ACT, LT, DU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        allowed = 200 * 1024;
+    }
+    return cudaLaunchKernelEx(cfg, mid_cls_kernel<ACT, LT, DU>, p);
 }
 
 template <int ACT, typename DU>
@@ -332,10 +437,10 @@ inline cudaError_t mid_launch_lt(const MidPlan& mp, const MidParams& p, cudaStre
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     switch (mp.LT) {
-        case 8: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 8, DU>, p);
-        case 16: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 16, DU>, p);
-        case 24: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 24, DU>, p);
-        default: return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, 32, DU>, p);
+        case 8: return mid_launch_one<ACT, 8, DU>(&cfg, p);
+        case 16: return mid_launch_one<ACT, 16, DU>(&cfg, p);
+        case 24: return mid_launch_one<ACT, 24, DU>(&cfg, p);
+        default: return mid_launch_one<ACT, 32, DU>(&cfg, p);
     }
 }
 

@@ -415,7 +415,7 @@ __global__ void mean_kernel(const float* __restrict__ x, int n, float* __restric
 // ---------------------------------------------------------------------------
 // Fused AdamW over the flat parameter vector (decoupled decay on the weight matrices
 // only).  bc1 = 1-beta1^t, bc2 = 1-beta2^t (bias corrections, computed on the host in double).  Also refreshes the bf16
-// transposed hi/lo shadow of W_down ([L][2][r][d]) that the tensor-core path multiplies with.
+// hi/lo shadow of W_down ([L][2][d][r]) that the tensor-core path multiplies with.
 // ---------------------------------------------------------------------------
 // One element of the update, shared by every kernel that applies AdamW so that fused and
 // separate updates are bit-identical.
@@ -436,10 +436,9 @@ __device__ __forceinline__ void adamw_element(float* __restrict__ p, float* __re
     p[i] = th;
     if (wdT && i < lay.lam) {
         const long long dr = (long long)d * r, l = i / dr, rem = i - l * dr;
-        const int k = (int)(rem / r), j = (int)(rem - (long long)k * r);
         const bf16 hi = __float2bfloat16(th);
-        wdT[((l * 2 + 0) * r + j) * (long long)d + k] = hi;
-        wdT[((l * 2 + 1) * r + j) * (long long)d + k] = __float2bfloat16(th - __bfloat162float(hi));
+        wdT[(l * 2 + 0) * dr + rem] = hi;
+        wdT[(l * 2 + 1) * dr + rem] = __float2bfloat16(th - __bfloat162float(hi));
     }
 }
 
@@ -451,16 +450,15 @@ __global__ void adamw_kernel(float* __restrict__ p, const float* __restrict__ g,
     adamw_element(p, m, v, i, g[i], lay, hp, bc1, bc2, wdT, d, r);
 }
 
-// bf16 transposed hi/lo shadow of W_down from the fp32 master:
-// wdT[l][0][j][k] = bf16(W_down[l][k][j]), wdT[l][1][j][k] = bf16(W_down[l][k][j] - hi).
+// bf16 hi/lo shadow of W_down from the fp32 master, same [d][r] order:
+// wdT[l][0][k][j] = bf16(W_down[l][k][j]), wdT[l][1][k][j] = bf16(W_down[l][k][j] - hi).
 __global__ void shadow_wdown_kernel(const float* __restrict__ w, bf16* __restrict__ wdT, int L, int d, int r) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)L * d * r) return;
     long long l = i / ((long long)d * r), rem = i - l * (long long)d * r;
-    int k = rem / r, j = rem - (long long)k * r;
     const bf16 hi = __float2bfloat16(w[i]);
-    wdT[((l * 2 + 0) * r + j) * (long long)d + k] = hi;
-    wdT[((l * 2 + 1) * r + j) * (long long)d + k] = __float2bfloat16(w[i] - __bfloat162float(hi));
+    wdT[(l * 2 + 0) * (long long)d * r + rem] = hi;
+    wdT[(l * 2 + 1) * (long long)d * r + rem] = __float2bfloat16(w[i] - __bfloat162float(hi));
 }
 
 }  // namespace pac

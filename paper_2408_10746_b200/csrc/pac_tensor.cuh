@@ -178,10 +178,10 @@ struct FwdParams {
 
 // ---------------------------------------------------------------------------
 // u_l = h_l W_down^l.  A tile: 128 tokens of one (sample, layer) x 64 columns, K-major,
-// straight from the cache.  B tile: W_down^l transposed and split into two bf16 terms
-// (hi = bf16(W), lo = bf16(W - hi); shadow [L][2][r][d]), 2 x (r x 64), K-major; both
-// products accumulate into the same fp32 accumulator, so the weights enter with about 16
-// mantissa bits.  (With bf16-rounded weights alone the ReLU masks of about one element in a
+// straight from the cache.  B tile: 64 rows of W_down^l in its natural [d][r] order (an
+// MN-major operand), split into two bf16 terms (hi = bf16(W), lo = bf16(W - hi); shadow
+// [L][2][d][r]); both products accumulate into the same fp32 accumulator, so the weights
+// enter with about 16 mantissa bits.  (With bf16-rounded weights alone the ReLU masks of about one element in a
 // thousand flip, which alone costs ~3% relative error in dW_down and dlambda.)
 // Persistent CTAs walk tiles (layer, sample, token chunk); accumulators are double-buffered
 // in TMEM so the epilogue of one tile overlaps the loads and MMAs of the next.
@@ -191,8 +191,10 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int r_pad = (p.r + 7) & ~7;
-    const uint32_t a_bytes = FWD_ROWS * KC * 2, b_half = (uint32_t)r_pad * KC * 2, b_bytes = 2 * b_half;
-    const uint32_t b_off = a_bytes, stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
+    const int r_blocks = (p.r + 63) >> 6;
+    const uint32_t a_bytes = FWD_ROWS * KC * 2, b_box = KC * 128;            // one [64 k][64 columns of r] box
+    const uint32_t b_bytes = (uint32_t)r_blocks * 2 * b_box;                 // [r block][hi|lo][64 k][128 B]
+    const uint32_t b_off = a_bytes, stage_bytes = a_bytes + b_bytes;
     __shared__ __align__(8) unsigned long long bars[2 * 16 + 4];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
@@ -229,13 +231,14 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
                     mbar_expect_tx(full0 + 8 * s, a_bytes + b_bytes);
                     tma_load_4d(dst, &map_cache, full0 + 8 * s, kc * KC, sc * FWD_ROWS, l, id);
-                    tma_load_4d(dst + b_off, &map_w, full0 + 8 * s, kc * KC, 0, 0, l);
+                    for (int rb = 0; rb < r_blocks; ++rb)
+                        tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full0 + 8 * s, rb * 64, kc * KC, 0, l);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(FWD_ROWS, r_pad, 0, 0);
+            const uint32_t idesc = instr_desc_bf16(FWD_ROWS, r_pad, 0, 1);
             uint32_t it = 0, tile_n = 0;
             for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++tile_n) {
                 const int buf = tile_n & 1;
@@ -250,11 +253,14 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + b_off;
+                    // descriptors of the first 16-wide K step; later steps only move the start address
+                    // (field in 16-byte units): +32 B per step in the K-major A tile, +2048 B (16 rows) in B
+                    const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
+                    const uint64_t bh0 = smem_desc_sw128(b0, 2 * b_box, 1024), bl0 = smem_desc_sw128(b0 + b_box, 2 * b_box, 1024);
 #pragma unroll
                     for (int k = 0; k < KC / 16; ++k) {
-                        const uint64_t ad = smem_desc_sw128(a0 + k * 32, 16, 1024);
-                        umma_bf16(d_tmem, ad, smem_desc_sw128(b0 + k * 32, 16, 1024), idesc, (kc | k) ? 1u : 0u);
-                        umma_bf16(d_tmem, ad, smem_desc_sw128(b0 + b_half + k * 32, 16, 1024), idesc, 1u);
+                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bh0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
+                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bl0 + (uint64_t)(k * 128), idesc, 1u);
                     }
                     umma_commit(empty0 + 8 * s);          // frees the smem slot once these MMAs are done
                 }
@@ -333,7 +339,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     int item = blockIdx.x;
     const int j = item % p.splits; item /= p.splits;
     const int g = item % p.d_groups;
-    const int l = item / p.d_groups;
+    const int l = p.L - 1 - item / p.d_groups;       // last layers first: they were read most recently by the forward pass
     const int row_tiles = p.B * p.s_chunks;
     const int rt0 = (int)((long long)row_tiles * j / p.splits), rt1 = (int)((long long)row_tiles * (j + 1) / p.splits);
     const int col0 = g * p.chunks * 128;
@@ -381,12 +387,13 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
-                for (int k = 0; k < BWD_KR / 16; ++k) {
-                    const uint64_t bd = smem_desc_sw128(b0 + k * 2048, box_bytes, 1024);
-                    for (int c = 0; c < p.chunks; ++c) {
-                        const uint64_t ad = smem_desc_sw128(a0 + c * 2 * box_bytes + k * 2048, box_bytes, 1024);
-                        umma_bf16(tmem_base + (uint32_t)(c * r_pad), ad, bd, idesc, (it | (uint32_t)k) ? 1u : 0u);
-                    }
+                const uint64_t bd0 = smem_desc_sw128(b0, box_bytes, 1024);
+                for (int c = 0; c < p.chunks; ++c) {
+                    const uint64_t ad0 = smem_desc_sw128(a0 + c * 2 * box_bytes, box_bytes, 1024);
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(c * r_pad);
+#pragma unroll
+                    for (int k = 0; k < BWD_KR / 16; ++k)      // 16 tokens = 2048 B further along K in both operands
+                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 128), bd0 + (uint64_t)(k * 128), idesc, (it | (uint32_t)k) ? 1u : 0u);
                 }
                 umma_commit(empty0 + 8 * s);
             }
@@ -500,7 +507,7 @@ inline bool make_map(CUtensorMap* map, const void* base, int rank, const cuuint6
 
 inline int pow2_at_least(int x) { int p = 32; while (p < x) p <<= 1; return p; }
 
-// wdT: [L][2][r][d] bf16 hi/lo shadow of W_down (transposed); du16: [L][max_rows][r] bf16.  *part_floats receives the
+// wdT: [L][2][d][r] bf16 hi/lo shadow of W_down; du16: [L][max_rows][r] bf16.  *part_floats receives the
 // size of the split-partial buffer dW needs (0 when no split is used).
 inline pac_status tensor_plan_create(TensorPlan& tp, int device, const bf16* cache, const Dims& dm, int max_batch,
                                      const bf16* wdT, const bf16* du16, long long* part_floats) {
@@ -524,9 +531,9 @@ inline pac_status tensor_plan_create(TensorPlan& tp, int device, const bf16* cac
         if (!make_map(&tp.map_cache_bwd, cache, 4, dims, str, box_b)) return PAC_ERR_UNSUPPORTED;
     }
     {
-        cuuint64_t dims[4] = {(cuuint64_t)dm.d, (cuuint64_t)dm.r, 2, (cuuint64_t)dm.L};
-        cuuint64_t str[3] = {(cuuint64_t)dm.d * 2, (cuuint64_t)dm.r * dm.d * 2, (cuuint64_t)2 * dm.r * dm.d * 2};
-        cuuint32_t box[4] = {KC, (cuuint32_t)dm.r, 2, 1};
+        cuuint64_t dims[4] = {(cuuint64_t)dm.r, (cuuint64_t)dm.d, 2, (cuuint64_t)dm.L};
+        cuuint64_t str[3] = {(cuuint64_t)dm.r * 2, (cuuint64_t)dm.r * dm.d * 2, (cuuint64_t)2 * dm.r * dm.d * 2};
+        cuuint32_t box[4] = {64, KC, 2, 1};
         if (!make_map(&tp.map_w, wdT, 4, dims, str, box)) return PAC_ERR_UNSUPPORTED;
     }
     {
@@ -544,7 +551,7 @@ inline pac_status tensor_plan_create(TensorPlan& tp, int device, const bf16* cac
     f.tmem_cols = pow2_at_least(2 * r_pad);
     f.acc_stride = f.tmem_cols / 2;
     {
-        const int stage = FWD_ROWS * KC * 2 + ((2 * dm.r * KC * 2 + 1023) & ~1023);
+        const int stage = FWD_ROWS * KC * 2 + ((dm.r + 63) / 64) * 2 * KC * 128;
         int st = (max_smem - 2048) / stage;
         if (st > 16) st = 16;
         if (st < 2) { tensor_err() = "not enough shared memory for the forward pipeline"; return PAC_ERR_UNSUPPORTED; }
