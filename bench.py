@@ -307,8 +307,11 @@ def main():
     for name, (tot_ms, cnt) in kt.items():
         if cnt:
             avg = tot_ms / cnt
-            kern[name] = {"avg_ms": avg, "launches": cnt, "gbs": pass_bytes / (avg * 1e-3) / 1e9}
-    dominant = max(kern, key=lambda k: kern[k]["avg_ms"]) if kern else None
+            kern[name] = {"avg_ms": avg, "launches": cnt}
+            if name in ("down_projection", "dw_down"):      # the two passes over the cached activations
+                kern[name]["gbs"] = pass_bytes / (avg * 1e-3) / 1e9
+    stream_k = [k for k in kern if "gbs" in kern[k]]
+    dominant = max(stream_k, key=lambda k: kern[k]["avg_ms"]) if stream_k else None
     roofline = None
     if dominant:
         a = kern[dominant]["gbs"]

@@ -138,12 +138,15 @@ pac_status pac_get_opt_state(pac_ctx* ctx, float* m, float* v, long long* step);
 pac_status pac_set_opt_state(pac_ctx* ctx, const float* m, const float* v, long long step);
 
 pac_status pac_set_option(pac_ctx* ctx, int option, int value);
-/* Per-kernel device times.  With PAC_OPT_KERNEL_TIMING = 1 the two cache-stream kernels of
- * every later train step (down-projection u_l = h_l W_down^l over all layers; dW_down =
- * h_l^T du_l over all layers) are bracketed by CUDA events on the context's stream.  This
- * call waits for the stream, then stores the summed milliseconds and launch counts since the
- * last call: out_ms[0], out_count[0] for the down-projection, [1] for dW_down (host arrays of 2).
- * At most 4096 bracketed launches per kernel are kept between two calls. */
+/* Per-kernel device times.  With PAC_OPT_KERNEL_TIMING = 1 the kernels of every later train
+ * step are bracketed by CUDA events on the context's stream, in four groups:
+ *   [0] down-projection u_l = h_l W_down^l over all layers (first pass over the cache)
+ *   [1] merge/activation chain, head, loss and the reverse chain
+ *   [2] dW_down = h_l^T du_l over all layers (second pass over the cache)
+ *   [3] gradient finalisation (+ AdamW when fused into the step)
+ * This call waits for the stream, then stores the summed milliseconds and the number of
+ * bracketed launches since the last call in out_ms[4] and out_count[4] (host arrays).
+ * At most 4096 brackets per group are kept between two calls. */
 pac_status pac_kernel_times(pac_ctx* ctx, double* out_ms, long long* out_count);
 /* Number of kernels this context has launched so far. */
 pac_status pac_launch_count(pac_ctx* ctx, long long* n);

@@ -234,11 +234,12 @@ class PacContext:
         self._ck(self._lib.pac_set_opt_state(self._h, m.ctypes.data, v.ctypes.data, step))
 
     def kernel_times(self):
-        """(ms_total, launches) for the down-projection and for dW_down since the last call."""
-        ms = (C.c_double * 2)()
-        cnt = (C.c_longlong * 2)()
+        """(ms_total, launches) per kernel group of the train step since the last call."""
+        ms = (C.c_double * 4)()
+        cnt = (C.c_longlong * 4)()
         self._ck(self._lib.pac_kernel_times(self._h, ms, cnt))
-        return {"down_projection": (ms[0], cnt[0]), "dw_down": (ms[1], cnt[1])}
+        names = ["down_projection", "chain_head", "dw_down", "finalize"]
+        return {n: (ms[i], cnt[i]) for i, n in enumerate(names)}
 
     def launch_count(self) -> int:
         n = C.c_longlong()

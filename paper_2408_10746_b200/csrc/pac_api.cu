@@ -78,8 +78,8 @@ struct pac_ctx {
     // options / bookkeeping
     int force_simt = 0;
     int timing = 0;
-    std::vector<cudaEvent_t> tev[2];   // start/stop pairs per bracketed kernel
-    size_t tev_used[2] = {0, 0};
+    std::vector<cudaEvent_t> tev[4];   // start/stop pairs per bracketed kernel group
+    size_t tev_used[4] = {0, 0, 0, 0};
     bool tensor_ok = false;
     long long launches = 0;
     TensorPlan tplan{};
@@ -356,7 +356,7 @@ pac_status down_projection(pac_ctx* c, const int* d_ids, int B) {
 
 pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     pac_status st;
-    time_mark(c, 1, false);
+    time_mark(c, 2, false);
     if (use_tensor(c)) {
         st = tensor_dw_down(c->tplan, c->stream, d_ids, B, c->sc.du16, c->grads + c->lay.w_down, c->sc.dw_part,
                             reduce_splits, c->status, &c->launches);
@@ -365,7 +365,7 @@ pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
         st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
         if (st != PAC_OK) return st;
     }
-    time_mark(c, 1, true);
+    time_mark(c, 2, true);
     return PAC_OK;
 }
 
@@ -376,7 +376,7 @@ pac_status mid_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d
     p.ids = d_ids; p.N = dm.N; p.labels = c->labels;
     p.L = dm.L; p.S = dm.S; p.d = dm.d; p.r = dm.r; p.C = dm.C; p.B = B;
     p.G = c->mplan.G; p.Sg = c->mplan.Sg; p.dg = c->mplan.dg; p.train = train ? 1 : 0;
-    p.scratch = c->mplan.scratch; p.wup_smem = c->mplan.wup_smem; p.u_smem = c->mplan.u_smem;
+    p.scratch = c->mplan.scratch; p.wup_smem = c->mplan.wup_smem;
     p.u = sc.u; p.lstride = (long long)c->max_rows * dm.r;
     p.lam = c->params + c->lay.lam; p.W_up = c->params + c->lay.w_up;
     p.W_head = c->params + c->lay.w_head; p.b_head = c->params + c->lay.b_head; p.hbar = sc.hbar;
@@ -424,9 +424,14 @@ pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, con
     pac_status st;
     if (use_fused_cls(c)) {
         if ((st = down_projection(c, d_ids, B)) != PAC_OK) return st;
+        time_mark(c, 1, false);
         if ((st = mid_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
+        time_mark(c, 1, true);
         if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
-        return finalize_enqueue(c, B, d_loss, hp);
+        time_mark(c, 3, false);
+        st = finalize_enqueue(c, B, d_loss, hp);
+        time_mark(c, 3, true);
+        return st;
     }
     if ((st = forward(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
     if ((st = backward(c, d_ids, B, d_loss)) != PAC_OK) return st;
@@ -814,7 +819,7 @@ pac_status pac_kernel_times(pac_ctx* c, double* out_ms, long long* out_count) {
     if (!out_ms || !out_count) return fail(c, PAC_ERR_INVALID_ARG, "pac_kernel_times: NULL argument");
     CU_OK(c, cudaSetDevice(c->device));
     CU_OK(c, cudaStreamSynchronize(c->stream));
-    for (int w = 0; w < 2; ++w) {
+    for (int w = 0; w < 4; ++w) {
         double tot = 0.0;
         long long cnt = 0;
         for (size_t i = 0; i + 1 < c->tev_used[w]; i += 2) {

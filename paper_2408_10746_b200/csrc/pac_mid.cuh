@@ -3,7 +3,7 @@
 //
 // mid_cls_kernel: one thread-block cluster per batch sample.  From the down-projections
 // u_l it runs the lambda-merge / adapter-body chain (Section IV-A) for all layers keeping
-// what the reverse pass needs (u_l - a_{l-1} and the ReLU mask) in registers, pools a_L over
+// what the reverse pass needs (u_l - a_{l-1} in shared memory, the ReLU masks in registers), pools a_L over
 // the sample's tokens through distributed shared memory, evaluates head, loss and their
 // gradients for the sample, and walks the chain backwards to emit du_l (bf16 or fp32) and
 // per-block partial sums of dlambda_l.  Nothing but u is read and nothing but du and a few
@@ -29,7 +29,6 @@ struct MidParams {
     int train;
     int scratch;                // floats of block-local reduction scratch
     int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
-    int u_smem;                 // 1: every thread's u values are prefetched into shared memory
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
     void* du;                   // [L][max_rows][r] bf16 or fp32
@@ -44,6 +43,7 @@ struct MidParams {
 };
 
 constexpr int MID_MAX_C = 32;
+constexpr int MID_MAX_L = 32;     // ReLU masks of all layers live in one 32-bit word per element
 
 __device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
@@ -55,8 +55,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int ACT, int LT, typename DU>
-__global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams p) {
+template <int ACT, typename DU>
+__global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
+    constexpr int LT = MID_MAX_L;
     cg::cluster_group cluster = cg::this_cluster();
     const int q = (int)cluster.block_rank();
     const int b = blockIdx.x / p.G;
@@ -65,8 +66,8 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
     const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
 
     extern __shared__ float4 sm4[];
-    float4* u_s = sm4;                           // [L][nt] each thread's own u values (when p.u_smem)
-    float* sm = reinterpret_cast<float*>(sm4 + (p.u_smem ? (size_t)L * nt : 0));
+    float4* u_s = sm4;                           // [L][nt] each thread's own u values, later u_l - a_{l-1}
+    float* sm = reinterpret_cast<float*>(sm4 + (size_t)L * nt);
     float* aL = sm;                              // [Sg][r]   a_L of this CTA's tokens
     float* colsum = aL + (size_t)p.Sg * r;       // [r]       exchanged through DSMEM
     float* lpart = colsum + r;                   // [MID_MAX_C] exchanged
@@ -87,7 +88,7 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
     const int s = q * p.Sg + s_local;
     const bool live = s_local < p.Sg && s < p.S;
     const long long base = ((long long)b * p.S + s) * r + j4;
-    if (p.u_smem && live)
+    if (live)
         for (int l = 0; l < L; ++l) cp_async_16(u_s + (size_t)l * nt + t, p.u + (long long)l * p.lstride + base);
     cp_async_commit();                                                          // group: u
     const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
@@ -103,21 +104,23 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
     __syncthreads();
     cp_async_wait_group<1>();                                                   // own u values have landed
 
-    // ---- forward chain: thread owns 4 consecutive adapter columns of one token ----
-    float w[LT][4];
+    // ---- forward chain: thread owns 4 consecutive adapter columns of one token.  The slot that
+    // held u_l is overwritten with u_l - a_{l-1} (= d z_l / d lambda_l) for the reverse pass; the
+    // ReLU masks stay in four registers (bit l of mask[e]).  Loops are kept rolled on purpose:
+    // every CTA runs this code once, so small code beats unrolled code.
     unsigned mask[4] = {0u, 0u, 0u, 0u};
     float ap[4] = {0.f, 0.f, 0.f, 0.f};                 // a_0 = 0
-#pragma unroll
-    for (int l = 0; l < LT; ++l) {
-        if (l < L) {
-            float4 uu = make_float4(0, 0, 0, 0);
-            if (live) uu = p.u_smem ? u_s[(size_t)l * nt + t] : *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base);
+    if (live) {
+#pragma unroll 1
+        for (int l = 0; l < L; ++l) {
+            const float4 uu = u_s[(size_t)l * nt + t];
             const float uv[4] = {uu.x, uu.y, uu.z, uu.w};
             const float lm = lam_s[l];
+            float wv[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float z = lm * uv[e] + (1.f - lm) * ap[e];
-                w[l][e] = uv[e] - ap[e];                     // d z_l / d lambda_l
+                wv[e] = uv[e] - ap[e];
                 if (ACT == PAC_ACT_RELU) {
                     const bool on = z > 0.f;
                     mask[e] |= (on ? 1u : 0u) << l;
@@ -126,6 +129,7 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
                     ap[e] = z;
                 }
             }
+            u_s[(size_t)l * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
         }
     }
     if (s_local < p.Sg) {
@@ -244,43 +248,33 @@ __global__ void __launch_bounds__(LT <= 16 ? 512 : 256) mid_cls_kernel(MidParams
 #pragma unroll
     for (int e = 0; e < 4; ++e) da[e] = live ? daL[j4 + e] : 0.f;
     DU* du = reinterpret_cast<DU*>(p.du);
-    float lpart_l[LT];                                     // this thread's share of dlambda_l
-#pragma unroll
-    for (int l = LT - 1; l >= 0; --l) {
-        lpart_l[l] = 0.f;
-        if (l < L) {
-            const float lm = lam_s[l];
-            float part = 0.f, dv[4];
+#pragma unroll 1
+    for (int l = L - 1; l >= 0; --l) {
+        const float lm = lam_s[l];
+        float part = 0.f, dv[4] = {0.f, 0.f, 0.f, 0.f};
+        if (live) {
+            const float4 w4 = u_s[(size_t)l * nt + t];
+            const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float dz = (ACT == PAC_ACT_RELU) ? (((mask[e] >> l) & 1u) ? da[e] : 0.f) : da[e];
-                part = fmaf(dz, w[l][e], part);
+                part = fmaf(dz, wv[e], part);
                 dv[e] = lm * dz;                           // du_l
                 da[e] = (1.f - lm) * dz;                   // da_{l-1}
             }
-            lpart_l[l] = part;
-            if (live) {
-                DU* dst = du + (long long)l * p.lstride + base;
-                if constexpr (sizeof(DU) == 2) {
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
-                    uint2 pk;
-                    pk.x = *reinterpret_cast<unsigned*>(&lo);
-                    pk.y = *reinterpret_cast<unsigned*>(&hi);
-                    *reinterpret_cast<uint2*>(dst) = pk;
-                } else {
-                    *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
-                }
+            DU* dst = du + (long long)l * p.lstride + base;
+            if constexpr (sizeof(DU) == 2) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
+                uint2 pk;
+                pk.x = *reinterpret_cast<unsigned*>(&lo);
+                pk.y = *reinterpret_cast<unsigned*>(&hi);
+                *reinterpret_cast<uint2*>(dst) = pk;
+            } else {
+                *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
             }
         }
-    }
-    // warp sums of all layers together (independent shuffle chains overlap), then across warps in order
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-        for (int l = 0; l < LT; ++l) lpart_l[l] += __shfl_xor_sync(0xffffffffu, lpart_l[l], o);
-    if (lane == 0) {
-#pragma unroll
-        for (int l = 0; l < LT; ++l) lred[warp * LT + l] = lpart_l[l];
+        part = warp_sum(part);                             // this warp's share of dlambda_l
+        if (lane == 0) lred[warp * LT + l] = part;
     }
     __syncthreads();
     if (t < L) {
@@ -369,61 +363,53 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
 }
 
 // Shape test and launch geometry of the fused kernel: G CTAs per sample, one 4-column
-// group per thread, chain state in registers.
+// group per thread, chain state in shared memory.
 struct MidPlan {
     bool ok = false;
-    int G = 1, Sg = 0, dg = 0, threads = 0, LT = 0, scratch = 0, wup_smem = 0, u_smem = 0;
+    int G = 1, Sg = 0, dg = 0, threads = 0, scratch = 0, wup_smem = 0;
     size_t smem = 0;
 };
 
 inline MidPlan mid_plan(const Dims& dm) {
     MidPlan mp;
-    if (dm.r % 4 != 0 || dm.C > MID_MAX_C || dm.L > 32) return mp;
-    mp.LT = dm.L <= 8 ? 8 : dm.L <= 16 ? 16 : dm.L <= 24 ? 24 : 32;
-    const int max_threads = mp.LT <= 16 ? 512 : 256;          // register budget: 4*LT state values per thread
+    if (dm.r % 4 != 0 || dm.C > MID_MAX_C || dm.L > MID_MAX_L) return mp;
+    const int max_threads = 512;
     for (int G = 1; G <= 8; G *= 2) {
         const int Sg = (dm.S + G - 1) / G;
         const long long need = (long long)Sg * (dm.r / 4);
-        if (need <= max_threads) {
-            mp.G = G; mp.Sg = Sg; mp.dg = (dm.d + G - 1) / G;
-            int th = (int)((need + 31) / 32 * 32);
-            if (th < 128) th = 128;
-            mp.threads = th;
-            const int nw = th / 32;
-            int scratch = nw * mp.LT;
-            if (nw * MID_MAX_C > scratch) scratch = nw * MID_MAX_C;
-            const int parts = th / dm.r > 0 ? th / dm.r : 1;
-            if (parts * dm.r > scratch) scratch = parts * dm.r;
-            mp.scratch = scratch;
-            size_t floats = (size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)mp.dg + 2 * MID_MAX_C + mp.LT + scratch +
-                            (size_t)mp.dg * dm.C + 4;
-            const size_t budget = 200 * 1024 / sizeof(float);
-            const size_t ufl = 4 * (size_t)dm.L * th, wup = (size_t)dm.r * mp.dg;
-            mp.u_smem = floats + ufl <= budget ? 1 : 0;
-            if (mp.u_smem) floats += ufl;
-            mp.wup_smem = floats + wup <= budget ? 1 : 0;
-            if (mp.wup_smem) floats += wup;
-            mp.smem = sizeof(float) * floats;
-            mp.ok = true;
-            return mp;
-        }
+        if (need > max_threads) continue;
+        int th = (int)((need + 31) / 32 * 32);
+        if (th < 128) th = 128;
+        const int dg = (dm.d + G - 1) / G;
+        const int nw = th / 32;
+        int scratch = nw * MID_MAX_L;
+        if (nw * MID_MAX_C > scratch) scratch = nw * MID_MAX_C;
+        const int parts = th / dm.r > 0 ? th / dm.r : 1;
+        if (parts * dm.r > scratch) scratch = parts * dm.r;
+        size_t floats = (size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)dg + 2 * MID_MAX_C + MID_MAX_L + scratch +
+                        (size_t)dg * dm.C + 4;
+        const size_t budget = 200 * 1024 / sizeof(float);
+        const size_t ufl = 4 * (size_t)dm.L * th, wup = (size_t)dm.r * dg;
+        if (floats + ufl > budget) continue;              // the chain state must fit in shared memory: try more CTAs per sample
+        floats += ufl;
+        mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch;
+        mp.wup_smem = floats + wup <= budget ? 1 : 0;
+        if (mp.wup_smem) floats += wup;
+        mp.smem = sizeof(float) * floats;
+        mp.ok = true;
+        return mp;
     }
     return mp;
 }
 
-template <int ACT, int LT, typename DU>
-inline cudaError_t mid_launch_one(cudaLaunchConfig_t* cfg, const MidParams& p) {
-    static size_t allowed = 0;                       // largest dynamic shared memory size already opted in to
-    if (cfg->dynamicSmemBytes > 48 * 1024 && cfg->dynamicSmemBytes > allowed) {
-        cudaError_t e = cudaFuncSetAttribute(mid_cls_kernel<ACT, LT, DU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        allowed = 200 * 1024;
-    }
-    return cudaLaunchKernelEx(cfg, mid_cls_kernel<ACT, LT, DU>, p);
-}
-
 template <int ACT, typename DU>
-inline cudaError_t mid_launch_lt(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
+inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
+    static bool opted_in = false;                    // dynamic shared memory above 48 KB needs an opt-in per kernel
+    if (mp.smem > 48 * 1024 && !opted_in) {
+        cudaError_t e = cudaFuncSetAttribute(mid_cls_kernel<ACT, DU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        opted_in = true;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.B * mp.G), 1, 1);
     cfg.blockDim = dim3((unsigned)mp.threads, 1, 1);
@@ -436,18 +422,13 @@ inline cudaError_t mid_launch_lt(const MidPlan& mp, const MidParams& p, cudaStre
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    switch (mp.LT) {
-        case 8: return mid_launch_one<ACT, 8, DU>(&cfg, p);
-        case 16: return mid_launch_one<ACT, 16, DU>(&cfg, p);
-        case 24: return mid_launch_one<ACT, 24, DU>(&cfg, p);
-        default: return mid_launch_one<ACT, 32, DU>(&cfg, p);
-    }
+    return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, DU>, p);
 }
 
 inline cudaError_t mid_launch(const MidPlan& mp, const MidParams& p, int act, bool du_bf16, cudaStream_t stream) {
     if (act == PAC_ACT_RELU)
-        return du_bf16 ? mid_launch_lt<PAC_ACT_RELU, bf16>(mp, p, stream) : mid_launch_lt<PAC_ACT_RELU, float>(mp, p, stream);
-    return du_bf16 ? mid_launch_lt<PAC_ACT_IDENTITY, bf16>(mp, p, stream) : mid_launch_lt<PAC_ACT_IDENTITY, float>(mp, p, stream);
+        return du_bf16 ? mid_launch_one<PAC_ACT_RELU, bf16>(mp, p, stream) : mid_launch_one<PAC_ACT_RELU, float>(mp, p, stream);
+    return du_bf16 ? mid_launch_one<PAC_ACT_IDENTITY, bf16>(mp, p, stream) : mid_launch_one<PAC_ACT_IDENTITY, float>(mp, p, stream);
 }
 
 }  // namespace pac
