@@ -157,6 +157,38 @@ const char* pac_last_error(const pac_ctx* ctx);
 /* "tensor" or "simt": which kernels the next train step will use (valid after adapter_init). */
 const char* pac_kernel_path(const pac_ctx* ctx);
 
+/* Evaluation forward that allocates nothing (the paper has no counterpart; this is a
+ * packaging variant of pac_eval_logits for the mean-pool classifier head).
+ *
+ * Who needs it: code that runs where device allocation is off limits - inside a host
+ * application that has handed all device memory to its own pool, in a latency-critical serving
+ * loop that must never hit the allocator's implicit synchronisation, or in a plugin that is only
+ * given raw buffers.  Such callers cannot create a pac_ctx (pac_adapter_init allocates).
+ *
+ * The forward's intermediates (u_l and a_l for every layer, pooled vectors, a token mean of the
+ * last cached layer for the B samples) live in one fixed array of PAC_STATIC_SCRATCH_BYTES
+ * (8 MiB) that is part of the library image: every GPU that loads the library holds it until the
+ * process exits.  A call is rejected with PAC_ERR_UNSUPPORTED when
+ *     4 * (2*L*B*S*r + B*r + B*d + B) bytes (each block rounded up to 256) exceed that size.
+ * The first call on a device looks up the array's device address; make that first call outside
+ * any stream capture.  No call allocates or frees device or pinned memory.
+ *
+ * All calls on a device share the array.  Every part of it is rewritten before it is read, so a
+ * call never sees the previous call's contents, but two calls whose kernels overlap on the GPU
+ * (different streams, no ordering) race on it: order them.
+ *
+ * Arguments: device, cuda_stream (cudaStream_t or NULL for the default stream); dev_cache, dtype,
+ * N, L, S, d as in pac_cache_register (device, read-only); dev_params: device, flat fp32 vector
+ * in the layout W_down[L][d][r] | lambda[L] | W_up[r][d] | W_head[d][C] | b_head[C]; r, act
+ * (pac_act), n_out = C; dev_sample_ids: device, B int32 ids (an id outside [0, N) is clamped
+ * into range, not reported); dev_out: device, fp32 [B][C]; err / err_len: optional host buffer
+ * that receives a message when the status is not PAC_OK.  The work is enqueued on the stream;
+ * dev_out is valid once the stream has reached that point. */
+#define PAC_STATIC_SCRATCH_BYTES (8u << 20)
+pac_status pac_eval_logits_static(int device, void* cuda_stream, const void* dev_cache, int dtype, long long N, int L,
+                                  int S, int d, const float* dev_params, int r, int act, int n_out,
+                                  const int* dev_sample_ids, int B, float* dev_out, char* err, int err_len);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,7 @@ EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init"
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
            "pac_set_opt_state", "pac_set_option", "pac_kernel_times", "pac_launch_count", "pac_sync", "pac_last_error",
-           "pac_kernel_path"]
+           "pac_kernel_path", "pac_eval_logits_static"]
 
 
 class PacError(RuntimeError):
@@ -94,6 +94,8 @@ def load_library() -> C.CDLL:
         fn = getattr(lib, name)
         fn.argtypes = args
         fn.restype = I
+    lib.pac_eval_logits_static.argtypes = [I, P, P, I, LL, I, I, I, P, I, I, I, P, I, P, C.c_char_p, I]
+    lib.pac_eval_logits_static.restype = I
     lib.pac_last_error.argtypes = [P]
     lib.pac_last_error.restype = C.c_char_p
     lib.pac_kernel_path.argtypes = [P]
@@ -251,3 +253,30 @@ class PacContext:
 
     def kernel_path(self) -> str:
         return self._lib.pac_kernel_path(self._h).decode()
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def eval_logits_static(cache, dev_params, r: int, n_out: int, dev_sample_ids, out, act: int = PAC_ACT_RELU,
+                       device: int = 0, stream: Optional[int] = None):
+    """Classifier-head logits [B][C] without a context and without any allocation inside the
+    library (pac_eval_logits_static): for callers that may not allocate device memory - an
+    application that owns all of it through its own pool, a serving loop that must stay clear of the
+    allocator, a plugin that only ever receives raw buffers.  Intermediates live in a fixed 8 MiB
+    array inside the library, so sizes are limited (PacError PAC_ERR_UNSUPPORTED beyond that) and
+    calls that overlap on the GPU must be ordered by the caller.  All tensors are CUDA tensors the
+    caller owns: cache [N][L][S][d], dev_params flat fp32, dev_sample_ids int32 [B], out fp32 [B][C].
+    The work is enqueued on `stream` (default stream if None)."""
+    import torch
+    lib = load_library()
+    N, L, S, d = cache.shape
+    dt = {torch.float32: PAC_F32, torch.bfloat16: PAC_BF16}[cache.dtype]
+    assert dev_params.dtype == torch.float32 and dev_sample_ids.dtype == torch.int32 and out.dtype == torch.float32
+    err = C.create_string_buffer(512)
+    st = lib.pac_eval_logits_static(device, C.c_void_p(stream) if stream else None, cache.data_ptr(), dt, N, L, S, d,
+                                    dev_params.data_ptr(), r, act, n_out, dev_sample_ids.data_ptr(),
+                                    dev_sample_ids.numel(), out.data_ptr(), err, 512)
+    if st != 0:
+        raise PacError(st, err.value.decode())
+    return out

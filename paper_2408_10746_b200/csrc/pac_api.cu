@@ -2,6 +2,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -857,3 +858,115 @@ const char* pac_last_error(const pac_ctx* c) { return c ? c->err.c_str() : "null
 const char* pac_kernel_path(const pac_ctx* c) { return (c && c->inited && use_tensor(c)) ? "tensor" : "simt"; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// pac_eval_logits_static: the classifier-head evaluation forward with its scratch in a
+// fixed device array instead of context-owned allocations.
+// ---------------------------------------------------------------------------
+namespace {
+
+// The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; the
+// device address is looked up once per device below and that pointer is what kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[PAC_STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[MAX_DEVICES] = {};
+
+// Token mean of the last cached layer for the batch's samples, plus the identity index the
+// head kernel uses to address it: hbar_b[b][k] = mean_s cache[ids[b]][L-1][s][k], iota[b] = b.
+template <typename T>
+__global__ void pool_last_layer_batch_kernel(const T* __restrict__ cache, const int* __restrict__ ids, long long N, int L,
+                                             int S, int d, float* __restrict__ hbar_b, int* __restrict__ iota) {
+    const int b = blockIdx.x;
+    const long long id = safe_id(ids, b, N, nullptr);
+    const T* base = cache + ((id * L) + (L - 1)) * (long long)S * d;
+    for (int k = threadIdx.x; k < d; k += blockDim.x) {
+        float acc = 0.f;
+        for (int s = 0; s < S; ++s) acc += to_f32(base[(long long)s * d + k]);
+        hbar_b[(long long)b * d + k] = acc / (float)S;
+    }
+    if (threadIdx.x == 0) iota[b] = b;
+}
+
+pac_status static_fail(char* err, int err_len, pac_status st, const char* fmt, ...) {
+    if (err && err_len > 0) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(err, (size_t)err_len, fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+template <typename T>
+cudaError_t static_forward(cudaStream_t st, const T* cache, long long N, int L, int S, int d, const float* params,
+                           const ParamLayout& lay, int r, int act, int C, const int* ids, int B, float* out,
+                           float* u, float* a, float* pooled_a, float* hbar_b, int* iota) {
+    const int M = B * S;
+    const long long n = (long long)M * r;
+    CacheRows<T> A{cache, ids, N, L, S, d, 0};
+    MatB_RowMajor Bm{{params + lay.w_down, (long long)d * r, r}};
+    StoreRowMajor E{u, n, r};
+    dim3 grid(cdiv(r, SG_BN), cdiv(M, SG_BM), (unsigned)L);
+    gemm_simt<<<grid, 256, 0, st>>>(M, r, d, A, Bm, E);                                  // u_l = h_l W_down^l
+    if (act == PAC_ACT_RELU) chain_fwd_kernel<PAC_ACT_RELU><<<cdiv(n, 256), 256, 0, st>>>(u, a, params + lay.lam, L, n, n);
+    else chain_fwd_kernel<PAC_ACT_IDENTITY><<<cdiv(n, 256), 256, 0, st>>>(u, a, params + lay.lam, L, n, n);
+    pool_tokens_kernel<<<B, 128, 0, st>>>(a + (long long)(L - 1) * n, pooled_a, S, r);     // mean_s a_L
+    pool_last_layer_batch_kernel<T><<<B, 256, 0, st>>>(cache, ids, N, L, S, d, hbar_b, iota);
+    cls_head_kernel<<<B, 256, sizeof(float) * (d + C + 32), st>>>(hbar_b, iota, B, nullptr, pooled_a, params + lay.w_up,
+                                                                 params + lay.w_head, params + lay.b_head, B, S, d, r, C, 0,
+                                                                 nullptr, out, nullptr, nullptr, nullptr, nullptr, nullptr);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" pac_status pac_eval_logits_static(int device, void* cuda_stream, const void* dev_cache, int dtype, long long N,
+                                             int L, int S, int d, const float* dev_params, int r, int act, int n_out,
+                                             const int* dev_sample_ids, int B, float* dev_out, char* err, int err_len) {
+    if (!dev_cache || !dev_params || !dev_sample_ids || !dev_out)
+        return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: NULL device pointer");
+    if (dtype != PAC_F32 && dtype != PAC_BF16) return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: bad dtype %d", dtype);
+    if (act != PAC_ACT_RELU && act != PAC_ACT_IDENTITY) return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: bad activation %d", act);
+    if (N < 1 || L < 1 || S < 1 || d < 1 || r < 1 || n_out < 1 || B < 1)
+        return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: sizes must be positive");
+    if (device < 0 || device >= MAX_DEVICES) return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: bad device %d", device);
+    if ((size_t)(d + n_out + 32) * sizeof(float) > 48 * 1024)
+        return static_fail(err, err_len, PAC_ERR_UNSUPPORTED, "pac_eval_logits_static: d + C = %d is beyond the head kernel's shared memory", d + n_out);
+    // scratch layout: u | a | pooled_a | hbar_b | iota, each block rounded up to 256 bytes
+    const size_t Mr = (size_t)B * S * r;
+    const size_t o_u = 0, o_a = o_u + up256(sizeof(float) * Mr * L), o_p = o_a + up256(sizeof(float) * Mr * L);
+    const size_t o_h = o_p + up256(sizeof(float) * (size_t)B * r), o_i = o_h + up256(sizeof(float) * (size_t)B * d);
+    const size_t need = o_i + up256(sizeof(int) * (size_t)B);
+    if (need > (size_t)PAC_STATIC_SCRATCH_BYTES)
+        return static_fail(err, err_len, PAC_ERR_UNSUPPORTED,
+                           "pac_eval_logits_static: L=%d B=%d S=%d r=%d d=%d needs %zu bytes of scratch, the fixed array holds %u",
+                           L, B, S, r, d, need, (unsigned)PAC_STATIC_SCRATCH_BYTES);
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return static_fail(err, err_len, PAC_ERR_CUDA, "pac_eval_logits_static: cudaSetDevice: %s", cudaGetErrorString(e));
+    unsigned char* base;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[device]) {
+            // once per device, with that device current: the device address of the array
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_static_scratch);
+            if (e != cudaSuccess || !p)
+                return static_fail(err, err_len, PAC_ERR_CUDA, "pac_eval_logits_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+            g_static_ptr[device] = (unsigned char*)p;
+        }
+        base = g_static_ptr[device];
+    }
+    float *u = (float*)(base + o_u), *a = (float*)(base + o_a), *pooled_a = (float*)(base + o_p), *hbar_b = (float*)(base + o_h);
+    int* iota = (int*)(base + o_i);
+    const ParamLayout lay = ParamLayout::make(L, d, r, n_out, true);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    e = dtype == PAC_F32
+            ? static_forward<float>(st, (const float*)dev_cache, N, L, S, d, dev_params, lay, r, act, n_out, dev_sample_ids, B, dev_out, u, a, pooled_a, hbar_b, iota)
+            : static_forward<bf16>(st, (const bf16*)dev_cache, N, L, S, d, dev_params, lay, r, act, n_out, dev_sample_ids, B, dev_out, u, a, pooled_a, hbar_b, iota);
+    if (e != cudaSuccess) return static_fail(err, err_len, PAC_ERR_CUDA, "pac_eval_logits_static: kernel launch failed: %s", cudaGetErrorString(e));
+    return PAC_OK;
+}
