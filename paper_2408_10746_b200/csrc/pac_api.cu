@@ -415,8 +415,12 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         bias_corrections(hp, c->step, &f.bc1, &f.bc2);
         f.wdT = sc.wdT;
     }
-    finalize_cls_kernel<<<cdiv(c->lay.total, 256) + 1, 256, 0, c->stream>>>(f);    // + one block for lambda and the loss
-    LAUNCH_CHECK(c);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_launch_config(&cfg, attr, dim3(cdiv(c->lay.total, 256) + 1), dim3(256), 0, c->stream);   // + one block for lambda and the loss
+    cudaError_t le = cudaLaunchKernelEx(&cfg, finalize_cls_kernel, f);
+    c->launches++;
+    if (le != cudaSuccess) return fail(c, PAC_ERR_CUDA, "finalize kernel launch failed: %s", cudaGetErrorString(le));
     return PAC_OK;
 }
 

@@ -15,6 +15,7 @@
 
 #include "pac_common.cuh"
 #include "pac_simt.cuh"
+#include "pac_tensor.cuh"
 
 namespace pac {
 
@@ -82,6 +83,8 @@ __global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
     float* lred = wh_s + (size_t)p.dg * C;       // [nwarps][LT]; also [nwarps][MID_MAX_C] and [parts][r] scratch
     float* wup_s = lred + (size_t)p.scratch;     // [r][dg] slice of W_up (when p.wup_smem)
 
+    pdl_trigger();
+    pdl_wait();             // u comes from the kernel before this one
     // ---- everything this CTA will read from global memory is requested up front ----
     const int groups_per_tok = r >> 2;
     const int s_local = t / groups_per_tok, j4 = (t - s_local * groups_per_tok) << 2;
@@ -307,6 +310,8 @@ struct FinalizeParams {
 };
 
 __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
+    pdl_trigger();
+    pdl_wait();
     const ParamLayout& lay = f.lay;
     if (blockIdx.x == gridDim.x - 1) {
         // the last block: dlambda_l (one warp per layer, lanes over the per-block partials, fixed
@@ -415,13 +420,15 @@ inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStr
     cfg.blockDim = dim3((unsigned)mp.threads, 1, 1);
     cfg.dynamicSmemBytes = mp.smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)mp.G;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, DU>, p);
 }
 

@@ -24,6 +24,13 @@ namespace pac {
 // ---------------------------------------------------------------------------
 // PTX wrappers
 // ---------------------------------------------------------------------------
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization
+// attribute may start while its predecessor in the stream is still running; pdl_wait() blocks
+// until the predecessor grid has completed and its writes are visible, pdl_trigger() lets the
+// successor start launching.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -86,6 +93,18 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+// The same with an L2 eviction-priority hint (a policy word from createpolicy).
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
     asm volatile(
@@ -212,15 +231,20 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
         tma_prefetch_desc(&map_w);
     }
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), (uint32_t)p.tmem_cols); tmem_relinquish(); }
+    pdl_trigger();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
+    pdl_wait();            // everything above overlapped the previous kernel; its results are needed from here on
 
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
+            // cache tiles are read once per pass: evict them first, so that u, du, the weight shadow and
+            // the optimizer state stay L2-resident
+            const uint64_t pol = l2_policy_evict_first();
             for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
                 const int sc = t % p.s_chunks, b = (t / p.s_chunks) % p.B, l = t / (p.s_chunks * p.B);
                 const int id = (int)safe_id(p.ids, b, p.N, nullptr);
@@ -230,7 +254,7 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
                     const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
                     mbar_expect_tx(full0 + 8 * s, a_bytes + b_bytes);
-                    tma_load_4d(dst, &map_cache, full0 + 8 * s, kc * KC, sc * FWD_ROWS, l, id);
+                    tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, sc * FWD_ROWS, l, id, pol);
                     for (int rb = 0; rb < r_blocks; ++rb)
                         tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full0 + 8 * s, rb * 64, kc * KC, 0, l);
                 }
@@ -353,15 +377,18 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
         tma_prefetch_desc(&map_du);
     }
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), (uint32_t)p.tmem_cols); tmem_relinquish(); }
+    pdl_trigger();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
+    pdl_wait();
 
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
+            const uint64_t pol = l2_policy_evict_first();
             for (int rt = rt0; rt < rt1; ++rt, ++it) {
                 const int sc = rt % p.s_chunks, b = rt / p.s_chunks;
                 const int id = (int)safe_id(p.ids, b, p.N, nullptr);
@@ -371,7 +398,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
                 const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
                 mbar_expect_tx(full0 + 8 * s, stage_bytes);
                 for (int q = 0; q < 2 * p.chunks; ++q)
-                    tma_load_4d(dst + q * box_bytes, &map_cache, full0 + 8 * s, col0 + q * 64, sc * BWD_KR, l, id);
+                    tma_load_4d_hint(dst + q * box_bytes, &map_cache, full0 + 8 * s, col0 + q * 64, sc * BWD_KR, l, id, pol);
                 for (int q = 0; q < p.r_blocks; ++q)
                     tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full0 + 8 * s, q * 64, b * p.S + sc * BWD_KR, l);
             }
@@ -466,6 +493,19 @@ struct TensorPlan {
 
 inline std::string& tensor_err() { static std::string e; return e; }
 inline const char* tensor_last_error() { return tensor_err().c_str(); }
+
+// Launch configuration with programmatic stream serialization allowed (see pdl_wait above).
+inline void pdl_launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t stream) {
+    cfg->gridDim = grid;
+    cfg->blockDim = block;
+    cfg->dynamicSmemBytes = smem;
+    cfg->stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg->attrs = attr;
+    cfg->numAttrs = 1;
+}
 
 inline bool tensor_shape_supported(const Dims& dm) {
     return dm.d % 8 == 0 && dm.d >= 64 && dm.r % 16 == 0 && dm.r >= 16 && dm.r <= 256;
@@ -610,9 +650,11 @@ inline pac_status tensor_down_projection(TensorPlan& tp, cudaStream_t stream, co
     p.ids = d_ids; p.B = B; p.u = u; p.status = status;
     const int tiles = p.L * B * p.s_chunks;
     const int grid = tiles < tp.sms ? tiles : tp.sms;
-    down_fwd_tc_kernel<<<grid, TC_THREADS, tp.smem_fwd, stream>>>(tp.map_cache_fwd, tp.map_w, p);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_launch_config(&cfg, attr, dim3((unsigned)grid), dim3(TC_THREADS), tp.smem_fwd, stream);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, down_fwd_tc_kernel, tp.map_cache_fwd, tp.map_w, p);
     (*launches)++;
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tensor_err() = cudaGetErrorString(e); return PAC_ERR_CUDA; }
     return PAC_OK;
 }
@@ -634,9 +676,11 @@ inline pac_status tensor_dw_down(TensorPlan& tp, cudaStream_t stream, const int*
     p.splits = J;
     p.out = J > 1 ? part : dW;
     const int grid = p.L * p.d_groups * J;
-    dw_down_tc_kernel<<<grid, TC_THREADS, tp.smem_bwd, stream>>>(tp.map_cache_bwd, tp.map_du, p);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_launch_config(&cfg, attr, dim3((unsigned)grid), dim3(TC_THREADS), tp.smem_bwd, stream);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, dw_down_tc_kernel, tp.map_cache_bwd, tp.map_du, p);
     (*launches)++;
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tensor_err() = cudaGetErrorString(e); return PAC_ERR_CUDA; }
     if (J > 1 && reduce_splits) {
         reduce_splits_kernel<<<(unsigned)((tp.dw_elems / 4 + 255) / 256), 256, 0, stream>>>(part, J, tp.dw_elems, dW);
