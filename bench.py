@@ -31,7 +31,7 @@ METRIC = "adapter_epoch_samples_per_sec"
 UNIT = "samples/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
 # capture summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES = {"t5_base": None}
+NCU_TRAFFIC_BYTES = {"t5_base": {"down_projection": 79848448, "dw_down": 83975936}}
 
 
 def load_peaks():
@@ -317,7 +317,7 @@ def main():
         a = kern[dominant]["gbs"]
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "traffic": NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]), "algorithmic_bytes_per_launch": pass_bytes,
+                    "traffic": (NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]) or {}).get(dominant), "algorithmic_bytes_per_launch": pass_bytes,
                     "kernels": kern}
     step_s = ms * 1e-3 / K
     stream_gbs = 2 * pass_bytes / step_s / 1e9
