@@ -191,6 +191,7 @@ struct FwdParams {
     int stages;
     int tmem_cols;                         // power of two >= 2 * r_pad
     int acc_stride;                        // column offset of the second accumulator
+    int wide_n;                            // 1: hi and lo blocks form one N = 128*r_blocks MMA, summed in the epilogue
     float* u; long long layer_stride;      // u[l][m][j], layer_stride = max_rows * r
     unsigned* status;
 };
@@ -262,7 +263,9 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(FWD_ROWS, r_pad, 0, 1);
+            // wide_n: the hi and lo blocks lie next to each other along N ([r block][hi|lo] in 64-column
+            // blocks), so one MMA of N = 128 * r_blocks yields u_hi | u_lo side by side in TMEM
+            const uint32_t idesc = p.wide_n ? instr_desc_bf16(FWD_ROWS, 128 * r_blocks, 0, 1) : instr_desc_bf16(FWD_ROWS, r_pad, 0, 1);
             uint32_t it = 0, tile_n = 0;
             for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++tile_n) {
                 const int buf = tile_n & 1;
@@ -281,10 +284,17 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     // (field in 16-byte units): +32 B per step in the K-major A tile, +2048 B (16 rows) in B
                     const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
                     const uint64_t bh0 = smem_desc_sw128(b0, 2 * b_box, 1024), bl0 = smem_desc_sw128(b0 + b_box, 2 * b_box, 1024);
+                    if (p.wide_n) {
+                        const uint64_t bw0 = smem_desc_sw128(b0, b_box, 1024);
 #pragma unroll
-                    for (int k = 0; k < KC / 16; ++k) {
-                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bh0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
-                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bl0 + (uint64_t)(k * 128), idesc, 1u);
+                        for (int k = 0; k < KC / 16; ++k)
+                            umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bw0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < KC / 16; ++k) {
+                            umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bh0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
+                            umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bl0 + (uint64_t)(k * 128), idesc, 1u);
+                        }
                     }
                     umma_commit(empty0 + 8 * s);          // frees the smem slot once these MMAs are done
                 }
@@ -307,8 +317,19 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_stride);
             for (int c0 = 0; c0 < p.r; c0 += 16) {
                 float v[16];
-                tmem_ld16(taddr + c0, v);
-                tmem_ld_wait();
+                if (p.wide_n) {
+                    // column c of u: hi part at TMEM column (c/64)*128 + c%64, lo part 64 columns further
+                    float w[16];
+                    const uint32_t col = (uint32_t)((c0 >> 6) * 128 + (c0 & 63));
+                    tmem_ld16(taddr + col, v);
+                    tmem_ld16(taddr + col + 64, w);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) v[c] += w[c];
+                } else {
+                    tmem_ld16(taddr + c0, v);
+                    tmem_ld_wait();
+                }
                 if (srow < p.S) {
 #pragma unroll
                     for (int c = 0; c < 16; c += 4)
@@ -588,7 +609,8 @@ inline pac_status tensor_plan_create(TensorPlan& tp, int device, const bf16* cac
     f.N = dm.N; f.L = dm.L; f.S = dm.S; f.d = dm.d; f.r = dm.r;
     f.s_chunks = (dm.S + FWD_ROWS - 1) / FWD_ROWS;
     f.k_chunks = (dm.d + KC - 1) / KC;
-    f.tmem_cols = pow2_at_least(2 * r_pad);
+    f.wide_n = dm.r <= 128 ? 1 : 0;          // N = 128 * r_blocks must stay within 256
+    f.tmem_cols = pow2_at_least(2 * (f.wide_n ? 128 * ((dm.r + 63) / 64) : r_pad));
     f.acc_stride = f.tmem_cols / 2;
     {
         const int stage = FWD_ROWS * KC * 2 + ((dm.r + 63) / 64) * 2 * KC * 128;
