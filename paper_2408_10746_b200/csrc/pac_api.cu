@@ -10,6 +10,7 @@
 #include "pac_simt.cuh"
 #include "pac_tensor.cuh"
 #include "pac_mid.cuh"
+#include "pac_gemm.cuh"
 
 using namespace pac;
 
@@ -39,6 +40,8 @@ struct Scratch {
     float* y = nullptr;            // [M][d]
     float* lm_logits = nullptr;    // [M][V]
     float* dy = nullptr;           // [M][d]
+    bf16* y16 = nullptr;           // [M][d] bf16 y (tensor-core LM head)
+    bf16* dlog16 = nullptr;        // [M][V] bf16 dlogits (tensor-core LM head)
     // tensor path
     bf16* wdT = nullptr;           // [L][2][d][r] bf16 hi/lo shadow of W_down
     float* dw_part = nullptr;      // split partials of dW_down
@@ -85,6 +88,8 @@ struct pac_ctx {
     long long launches = 0;
     TensorPlan tplan{};
     MidPlan mplan{};               // fused classifier-head kernel (when the shape allows)
+    GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
+    bool lm_tensor = false;
     std::string err;
 };
 
@@ -242,7 +247,10 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
         dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
         MatA_RowMajor Aa{{aL, 0, dm.r}};
         MatB_RowMajor Bu{{W_up, 0, dm.d}};
-        if (c->dtype == PAC_F32) {
+        if (c->lm_tensor) {
+            StorePlusLastLayerBf16<bf16> E{sc.y16, dm.d, CacheRows<bf16>{(const bf16*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, dm.L - 1}};
+            gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.r, Aa, Bu, E);
+        } else if (c->dtype == PAC_F32) {
             StorePlusLastLayer<float> E{sc.y, dm.d, CacheRows<float>{(const float*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, dm.L - 1}};
             gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.r, Aa, Bu, E);
         } else {
@@ -252,14 +260,20 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
         LAUNCH_CHECK(c);
         // logits = y W_lm^T
         float* lg = train ? sc.lm_logits : d_logits_out;
-        dim3 g2(cdiv(dm.C, SG_BN), cdiv(M, SG_BM), 1);
-        MatA_RowMajor Ay{{sc.y, 0, dm.d}};
-        MatB_Bf16Rows Bw{(const bf16*)c->cfg.lm_head, dm.d};
-        StoreRowMajor El{lg, 0, dm.C};
-        gemm_simt<<<g2, 256, 0, c->stream>>>(M, dm.C, dm.d, Ay, Bw, El);
-        LAUNCH_CHECK(c);
+        if (c->lm_tensor) {
+            st = gemm_launch(c->g_logits, c->stream, M, lg, dm.C, c->status, &c->launches);
+            if (st != PAC_OK) return fail(c, st, "tensor-core logits GEMM launch failed: %s", tensor_last_error());
+        } else {
+            dim3 g2(cdiv(dm.C, SG_BN), cdiv(M, SG_BM), 1);
+            MatA_RowMajor Ay{{sc.y, 0, dm.d}};
+            MatB_Bf16Rows Bw{(const bf16*)c->cfg.lm_head, dm.d};
+            StoreRowMajor El{lg, 0, dm.C};
+            gemm_simt<<<g2, 256, 0, c->stream>>>(M, dm.C, dm.d, Ay, Bw, El);
+            LAUNCH_CHECK(c);
+        }
         if (train) {
-            lm_ce_kernel<<<M, 256, 0, c->stream>>>(lg, d_ids, dm.N, c->labels, dm.S, dm.C, M, 1, sc.loss_b, c->status);
+            lm_ce_kernel<<<M, 256, 0, c->stream>>>(lg, d_ids, dm.N, c->labels, dm.S, dm.C, M, 1, sc.loss_b, c->status,
+                                                   c->lm_tensor ? sc.dlog16 : nullptr);
             LAUNCH_CHECK(c);
         }
     }
@@ -299,12 +313,17 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
         mean_kernel<<<1, 1024, 0, c->stream>>>(sc.loss_b, M, d_loss);
         LAUNCH_CHECK(c);
         // dy = dlogits W_lm   (the head is frozen: it receives no gradient)
-        dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
-        MatA_RowMajor Ad{{sc.lm_logits, 0, dm.C}};
-        MatB_Bf16Cols Bw{(const bf16*)c->cfg.lm_head, dm.d};
-        StoreRowMajor Ed{sc.dy, 0, dm.d};
-        gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.C, Ad, Bw, Ed);
-        LAUNCH_CHECK(c);
+        if (c->lm_tensor) {
+            pac_status gs = gemm_launch(c->g_dy, c->stream, M, sc.dy, dm.d, c->status, &c->launches);
+            if (gs != PAC_OK) return fail(c, gs, "tensor-core dy GEMM launch failed: %s", tensor_last_error());
+        } else {
+            dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
+            MatA_RowMajor Ad{{sc.lm_logits, 0, dm.C}};
+            MatB_Bf16Cols Bw{(const bf16*)c->cfg.lm_head, dm.d};
+            StoreRowMajor Ed{sc.dy, 0, dm.d};
+            gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.C, Ad, Bw, Ed);
+            LAUNCH_CHECK(c);
+        }
         // dW_up = a_L^T dy
         dim3 g2(cdiv(dm.d, SG_BN), cdiv(dm.r, SG_BM), 1);
         MatA_ColMajor At{{aL, 0, dm.r}};
@@ -473,7 +492,7 @@ pac_status refresh_shadow(pac_ctx* c) {
 void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
-                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.wdT, s.dw_part, c->params, c->grads,
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.dw_part, c->params, c->grads,
                     c->m, c->v, c->status, c->d_perm, c->d_losses};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -600,9 +619,22 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     } else {
         A(dmalloc(c, &s.loss_b, c->max_rows));
         A(dmalloc(c, &s.daL, Mr));
-        A(dmalloc(c, &s.y, (long long)c->max_rows * dm.d));
         A(dmalloc(c, &s.lm_logits, (long long)c->max_rows * dm.C));
         A(dmalloc(c, &s.dy, (long long)c->max_rows * dm.d));
+        // the two dense LM-head GEMMs go to the tensor cores for bf16 caches with 16-byte operand rows
+        c->lm_tensor = false;
+        if (st == PAC_OK && c->dtype == PAC_BF16 && !c->force_simt && dm.d % 8 == 0 && dm.C % 8 == 0) {
+            A(dmalloc(c, &s.y16, (long long)c->max_rows * dm.d));
+            A(dmalloc(c, &s.dlog16, (long long)c->max_rows * dm.C));
+            if (st == PAC_OK) {
+                pac_status g1 = gemm_plan_create(c->g_logits, c->device, s.y16, c->max_rows, (const bf16*)cfg->lm_head, dm.C, dm.d, 0);
+                pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_dy, c->device, s.dlog16, c->max_rows, (const bf16*)cfg->lm_head, dm.d, dm.C, 1) : g1;
+                if (g1 == PAC_OK && g2 == PAC_OK) c->lm_tensor = true;
+                else if ((g1 != PAC_OK && g1 != PAC_ERR_UNSUPPORTED) || (g2 != PAC_OK && g2 != PAC_ERR_UNSUPPORTED))
+                    st = fail(c, PAC_ERR_CUDA, "LM-head GEMM set-up failed: %s", tensor_last_error());
+            }
+        }
+        if (st == PAC_OK && !c->lm_tensor) A(dmalloc(c, &s.y, (long long)c->max_rows * dm.d));
     }
     if (st == PAC_OK && cudaMallocHost((void**)&c->h_ids, sizeof(int) * STAGE_SLOTS * cfg->max_batch) != cudaSuccess)
         st = fail(c, PAC_ERR_NOMEM, "pinned id staging allocation failed");

@@ -142,6 +142,12 @@ struct StorePlusLastLayer {            // y = h_L + a_L W_up
     __device__ void operator()(int, int i, int j, float v) const { out[(long long)i * ld + j] = v + h(0, i, j); }
 };
 
+template <typename T>
+struct StorePlusLastLayerBf16 {        // the same, rounded to bf16 (A operand of the tensor-core LM-head GEMM)
+    bf16* out; int ld; CacheRows<T> h;
+    __device__ void operator()(int, int i, int j, float v) const { out[(long long)i * ld + j] = __float2bfloat16(v + h(0, i, j)); }
+};
+
 // ---------------------------------------------------------------------------
 // The lambda-merge / adapter-body chain over saved u (forward) and its reverse.
 // One thread per (row, column) element e < n = M*r of the [M][r] state; layer l of a
@@ -379,11 +385,12 @@ __global__ void reduce_rows_kernel(const float* __restrict__ part, int n, float*
 
 // ---------------------------------------------------------------------------
 // LM head cross-entropy, one block per row of logits [M][V]: loss_row = logsumexp -
-// logit[target]; when train != 0 the row is overwritten by (softmax - onehot)/M.
+// logit[target]; when train != 0 the row is overwritten by (softmax - onehot)/M, or, when
+// dlog16 is given, that gradient goes to dlog16 [M][V] in bf16 instead (A operand of dy = dlogits W_lm).
 // ---------------------------------------------------------------------------
 __global__ void lm_ce_kernel(float* __restrict__ logits, const int* __restrict__ ids, long long N,
                              const int* __restrict__ targets, int S, int V, int M, int train,
-                             float* __restrict__ loss_row, unsigned* status) {
+                             float* __restrict__ loss_row, unsigned* status, bf16* __restrict__ dlog16) {
     __shared__ float red[32];
     const int m = blockIdx.x;
     float* row = logits + (long long)m * V;
@@ -400,7 +407,13 @@ __global__ void lm_ce_kernel(float* __restrict__ logits, const int* __restrict__
     if (!train) return;
     __syncthreads();
     const float inv = 1.f / se, invM = 1.f / (float)M;
-    for (int v = threadIdx.x; v < V; v += blockDim.x) row[v] = (expf(row[v] - mx) * inv - (v == tgt ? 1.f : 0.f)) * invM;
+    if (dlog16) {
+        bf16* out = dlog16 + (long long)m * V;
+        for (int v = threadIdx.x; v < V; v += blockDim.x)
+            out[v] = __float2bfloat16((expf(row[v] - mx) * inv - (v == tgt ? 1.f : 0.f)) * invM);
+    } else {
+        for (int v = threadIdx.x; v < V; v += blockDim.x) row[v] = (expf(row[v] - mx) * inv - (v == tgt ? 1.f : 0.f)) * invM;
+    }
 }
 
 // mean of n values in index order (single block).

@@ -348,3 +348,42 @@ def test_full_size_step_matches_oracle(name):
     ctx.sync()
     ref = pi.cache_samples(spec, 0, ids[:4], "cpu").permute(1, 0, 2, 3).contiguous()
     assert out.cpu().view(torch.uint8).flatten().equal(ref.view(torch.uint8).flatten())
+
+
+# ------------------------------------------------------------------ frozen LM head on the tensor cores
+LM_TC_SPECS = [
+    SMALL_LM,                                                                                   # one ragged tile each way
+    pi.CacheSpec("lm_ragged_tiles", N=8, L=2, S=160, d=256, dtype="bf16", r=32, n_out=2056, B=3, head="lm"),
+]
+
+
+@pytest.mark.parametrize("spec", LM_TC_SPECS, ids=lambda s: s.name)
+def test_lm_head_tensor_path_loss_and_gradients(spec):
+    """logits = y W_lm^T and dy = dlogits W_lm as tcgen05 GEMMs (bf16 operands, fp32 accumulate)."""
+    tc_check(spec, spec.B, 0, ids=[spec.N - 1, 0, 2, 2][:spec.B], head_tol=5e-3)
+
+
+def test_lm_head_tensor_path_eval_logits():
+    spec = LM_TC_SPECS[1]
+    case = Case(spec)
+    ctx = case.context()
+    flat = pi.random_params(spec, 4)
+    ctx.set_params(flat)
+    ids = [1, 7, 7]
+    out = torch.zeros((3, spec.S, spec.n_out), dtype=torch.float32, device="cuda")
+    ctx.eval_logits(ids, out)
+    ctx.sync()
+    ref = po.eval_logits(case.oracle_params(flat), case.H(ids), 0, case.lm_np)
+    assert rel_l2(out.cpu().numpy(), ref) < 3e-3             # y enters the GEMM rounded to bf16
+
+
+def test_full_size_llama_step_matches_oracle():
+    """LLaMA-7B-shaped cache (L=32, S=512, d=4096, V=32000) at full strides; two samples of the
+    batch of 16 are run so that the oracle finishes in seconds."""
+    spec = pi.CONFIGS["llama_7b"]
+    free, _ = torch.cuda.mem_get_info()
+    if spec.cache_bytes + (8 << 30) > free:
+        pytest.skip("cache does not fit this device")
+    ids = [spec.N - 1, 0]
+    case = SparseCase(spec, ids)
+    tc_check(spec, spec.B, 0, ids=ids, case=case, head_tol=5e-3)
