@@ -44,6 +44,7 @@ struct MidParams {
 };
 
 constexpr int MID_MAX_C = 32;
+constexpr size_t MID_SMEM_BUDGET = 220 * 1024;    // dynamic shared memory the fused kernel may use
 constexpr int MID_MAX_L = 32;     // ReLU masks of all layers live in one 32-bit word per element
 
 __device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
@@ -56,8 +57,12 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int ACT, typename DU>
-__global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
+// GPT: 4-column groups per thread.  SMEM_STATE: the per-layer chain state (u_l, then u_l - a_{l-1})
+// sits in shared memory (prefetched with cp.async); otherwise u is read from global memory and
+// u_l - a_{l-1} is parked, in du's type, in the very slot of the du buffer that the reverse pass
+// overwrites with du_l once it has consumed it.
+template <int ACT, typename DU, int GPT, bool SMEM_STATE>
+__global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidParams p) {
     constexpr int LT = MID_MAX_L;
     cg::cluster_group cluster = cg::this_cluster();
     const int q = (int)cluster.block_rank();
@@ -67,8 +72,8 @@ __global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
     const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
 
     extern __shared__ float4 sm4[];
-    float4* u_s = sm4;                           // [L][nt] each thread's own u values, later u_l - a_{l-1}
-    float* sm = reinterpret_cast<float*>(sm4 + (size_t)L * nt);
+    float4* u_s = sm4;                           // [L][GPT][nt] each thread's own u values, later u_l - a_{l-1}
+    float* sm = reinterpret_cast<float*>(sm4 + (SMEM_STATE ? (size_t)L * GPT * nt : 0));
     float* aL = sm;                              // [Sg][r]   a_L of this CTA's tokens
     float* colsum = aL + (size_t)p.Sg * r;       // [r]       exchanged through DSMEM
     float* lpart = colsum + r;                   // [MID_MAX_C] exchanged
@@ -87,12 +92,55 @@ __global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
     pdl_wait();             // u comes from the kernel before this one
     // ---- everything this CTA will read from global memory is requested up front ----
     const int groups_per_tok = r >> 2;
-    const int s_local = t / groups_per_tok, j4 = (t - s_local * groups_per_tok) << 2;
-    const int s = q * p.Sg + s_local;
-    const bool live = s_local < p.Sg && s < p.S;
-    const long long base = ((long long)b * p.S + s) * r + j4;
-    if (live)
-        for (int l = 0; l < L; ++l) cp_async_16(u_s + (size_t)l * nt + t, p.u + (long long)l * p.lstride + base);
+    int s_local[GPT], j4[GPT];
+    bool live[GPT];
+    long long base[GPT];
+#pragma unroll
+    for (int g = 0; g < GPT; ++g) {
+        const int gi = t + g * nt;                       // this thread's g-th group of 4 adapter columns
+        s_local[g] = gi / groups_per_tok;
+        j4[g] = (gi - s_local[g] * groups_per_tok) << 2;
+        const int s = q * p.Sg + s_local[g];
+        live[g] = s_local[g] < p.Sg && s < p.S;
+        base[g] = ((long long)b * p.S + s) * r + j4[g];
+    }
+    DU* du = reinterpret_cast<DU*>(p.du);
+    // layer l of group g: read u, park / fetch the reverse-pass state
+    auto load_u = [&](int l, int g) -> float4 {
+        if constexpr (SMEM_STATE) return u_s[((size_t)l * GPT + g) * nt + t];
+        else return *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base[g]);
+    };
+    auto store_w = [&](int l, int g, const float* wv) {
+        if constexpr (SMEM_STATE) {
+            u_s[((size_t)l * GPT + g) * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
+        } else if constexpr (sizeof(DU) == 2) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]), hi = __floats2bfloat162_rn(wv[2], wv[3]);
+            uint2 pk;
+            pk.x = *reinterpret_cast<unsigned*>(&lo);
+            pk.y = *reinterpret_cast<unsigned*>(&hi);
+            *reinterpret_cast<uint2*>(du + (long long)l * p.lstride + base[g]) = pk;
+        } else {
+            *reinterpret_cast<float4*>(du + (long long)l * p.lstride + base[g]) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+        }
+    };
+    auto load_w = [&](int l, int g) -> float4 {
+        if constexpr (SMEM_STATE) {
+            return u_s[((size_t)l * GPT + g) * nt + t];
+        } else if constexpr (sizeof(DU) == 2) {
+            const uint2 pk = *reinterpret_cast<const uint2*>(du + (long long)l * p.lstride + base[g]);
+            const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
+            const float2 c = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.y));
+            return make_float4(a.x, a.y, c.x, c.y);
+        } else {
+            return *reinterpret_cast<const float4*>(du + (long long)l * p.lstride + base[g]);
+        }
+    };
+    if constexpr (SMEM_STATE) {
+#pragma unroll
+        for (int g = 0; g < GPT; ++g)
+            if (live[g])
+                for (int l = 0; l < L; ++l) cp_async_16(u_s + ((size_t)l * GPT + g) * nt + t, p.u + (long long)l * p.lstride + base[g]);
+    }
     cp_async_commit();                                                          // group: u
     const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
     const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
@@ -107,37 +155,52 @@ __global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
     __syncthreads();
     cp_async_wait_group<1>();                                                   // own u values have landed
 
-    // ---- forward chain: thread owns 4 consecutive adapter columns of one token.  The slot that
-    // held u_l is overwritten with u_l - a_{l-1} (= d z_l / d lambda_l) for the reverse pass; the
-    // ReLU masks stay in four registers (bit l of mask[e]).  Loops are kept rolled on purpose:
-    // every CTA runs this code once, so small code beats unrolled code.
-    unsigned mask[4] = {0u, 0u, 0u, 0u};
-    float ap[4] = {0.f, 0.f, 0.f, 0.f};                 // a_0 = 0
-    if (live) {
-#pragma unroll 1
-        for (int l = 0; l < L; ++l) {
-            const float4 uu = u_s[(size_t)l * nt + t];
-            const float uv[4] = {uu.x, uu.y, uu.z, uu.w};
-            const float lm = lam_s[l];
-            float wv[4];
+    // ---- forward chain over each group of 4 adapter columns of one token.  The slot that held
+    // u_l is overwritten with u_l - a_{l-1} (= d z_l / d lambda_l) for the reverse pass; the ReLU
+    // masks stay in registers (bit l of mask[g][e]).  Layers are taken four at a time so that the
+    // loads of a batch are in flight together; the outer loops stay rolled (every CTA runs this
+    // code once, so small code beats unrolled code).
+    unsigned mask[GPT][4];
+    float ap[GPT][4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float z = lm * uv[e] + (1.f - lm) * ap[e];
-                wv[e] = uv[e] - ap[e];
-                if (ACT == PAC_ACT_RELU) {
-                    const bool on = z > 0.f;
-                    mask[e] |= (on ? 1u : 0u) << l;
-                    ap[e] = on ? z : 0.f;
-                } else {
-                    ap[e] = z;
+    for (int g = 0; g < GPT; ++g) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { mask[g][e] = 0u; ap[g][e] = 0.f; }      // a_0 = 0
+        if (live[g]) {
+#pragma unroll 1
+            for (int l0 = 0; l0 < L; l0 += 4) {
+                float4 uq[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (l0 + i < L) uq[i] = load_u(l0 + i, g);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int l = l0 + i;
+                    if (l < L) {
+                        const float uv[4] = {uq[i].x, uq[i].y, uq[i].z, uq[i].w};
+                        const float lm = lam_s[l];
+                        float wv[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float z = lm * uv[e] + (1.f - lm) * ap[g][e];
+                            wv[e] = uv[e] - ap[g][e];
+                            if (ACT == PAC_ACT_RELU) {
+                                const bool on = z > 0.f;
+                                mask[g][e] |= (on ? 1u : 0u) << l;
+                                ap[g][e] = on ? z : 0.f;
+                            } else {
+                                ap[g][e] = z;
+                            }
+                        }
+                        store_w(l, g, wv);
+                    }
                 }
             }
-            u_s[(size_t)l * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
         }
-    }
-    if (s_local < p.Sg) {
+        if (s_local[g] < p.Sg) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) aL[(size_t)s_local * r + j4 + e] = live ? ap[e] : 0.f;
+            for (int e = 0; e < 4; ++e) aL[(size_t)s_local[g] * r + j4[g] + e] = live[g] ? ap[g][e] : 0.f;
+        }
     }
     __syncthreads();
     // column sums over this CTA's tokens: `parts` partial sums per column over contiguous token
@@ -246,38 +309,54 @@ __global__ void __launch_bounds__(512) mid_cls_kernel(MidParams p) {
     }
     __syncthreads();
 
-    // ---- reverse chain from registers ----
-    float da[4];
+    // ---- reverse chain ----
+    float da[GPT][4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) da[e] = live ? daL[j4 + e] : 0.f;
-    DU* du = reinterpret_cast<DU*>(p.du);
+    for (int g = 0; g < GPT; ++g)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) da[g][e] = live[g] ? daL[j4[g] + e] : 0.f;
 #pragma unroll 1
-    for (int l = L - 1; l >= 0; --l) {
-        const float lm = lam_s[l];
-        float part = 0.f, dv[4] = {0.f, 0.f, 0.f, 0.f};
-        if (live) {
-            const float4 w4 = u_s[(size_t)l * nt + t];
-            const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
+    for (int l0 = L - 1; l0 >= 0; l0 -= 4) {
+        float4 wq[4][GPT];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float dz = (ACT == PAC_ACT_RELU) ? (((mask[e] >> l) & 1u) ? da[e] : 0.f) : da[e];
-                part = fmaf(dz, wv[e], part);
-                dv[e] = lm * dz;                           // du_l
-                da[e] = (1.f - lm) * dz;                   // da_{l-1}
-            }
-            DU* dst = du + (long long)l * p.lstride + base;
-            if constexpr (sizeof(DU) == 2) {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
-                uint2 pk;
-                pk.x = *reinterpret_cast<unsigned*>(&lo);
-                pk.y = *reinterpret_cast<unsigned*>(&hi);
-                *reinterpret_cast<uint2*>(dst) = pk;
-            } else {
-                *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int g = 0; g < GPT; ++g)
+                if (l0 - i >= 0 && live[g]) wq[i][g] = load_w(l0 - i, g);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int l = l0 - i;
+            if (l >= 0) {
+                const float lm = lam_s[l];
+                float part = 0.f;
+#pragma unroll
+                for (int g = 0; g < GPT; ++g) {
+                    if (live[g]) {
+                        const float wv[4] = {wq[i][g].x, wq[i][g].y, wq[i][g].z, wq[i][g].w};
+                        float dv[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float dz = (ACT == PAC_ACT_RELU) ? (((mask[g][e] >> l) & 1u) ? da[g][e] : 0.f) : da[g][e];
+                            part = fmaf(dz, wv[e], part);
+                            dv[e] = lm * dz;                           // du_l
+                            da[g][e] = (1.f - lm) * dz;                // da_{l-1}
+                        }
+                        DU* dst = du + (long long)l * p.lstride + base[g];
+                        if constexpr (sizeof(DU) == 2) {
+                            __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
+                            uint2 pk;
+                            pk.x = *reinterpret_cast<unsigned*>(&lo);
+                            pk.y = *reinterpret_cast<unsigned*>(&hi);
+                            *reinterpret_cast<uint2*>(dst) = pk;
+                        } else {
+                            *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+                        }
+                    }
+                }
+                part = warp_sum(part);                             // this warp's share of dlambda_l
+                if (lane == 0) lred[warp * LT + l] = part;
             }
         }
-        part = warp_sum(part);                             // this warp's share of dlambda_l
-        if (lane == 0) lred[warp * LT + l] = part;
     }
     __syncthreads();
     if (t < L) {
@@ -372,46 +451,70 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
 struct MidPlan {
     bool ok = false;
     int G = 1, Sg = 0, dg = 0, threads = 0, scratch = 0, wup_smem = 0;
+    int gpt = 1, smem_state = 1;      // 4-column groups per thread; chain state in shared memory or parked in the du buffer
     size_t smem = 0;
 };
+
+// Shared-memory floats the kernel needs besides the chain state and the W_up slice.
+inline size_t mid_base_floats(const Dims& dm, int Sg, int dg, int th, int* scratch_out) {
+    const int nw = th / 32;
+    int scratch = nw * MID_MAX_L;
+    if (nw * MID_MAX_C > scratch) scratch = nw * MID_MAX_C;
+    const int parts = th / dm.r > 0 ? th / dm.r : 1;
+    if (parts * dm.r > scratch) scratch = parts * dm.r;
+    *scratch_out = scratch;
+    return (size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)dg + 2 * MID_MAX_C + MID_MAX_L + scratch + (size_t)dg * dm.C + 4;
+}
 
 inline MidPlan mid_plan(const Dims& dm) {
     MidPlan mp;
     if (dm.r % 4 != 0 || dm.C > MID_MAX_C || dm.L > MID_MAX_L) return mp;
-    const int max_threads = 512;
+    const size_t budget = MID_SMEM_BUDGET / sizeof(float);
+    // first choice: one group per thread, chain state in shared memory, fewest CTAs per sample
     for (int G = 1; G <= 8; G *= 2) {
-        const int Sg = (dm.S + G - 1) / G;
+        const int Sg = (dm.S + G - 1) / G, dg = (dm.d + G - 1) / G;
         const long long need = (long long)Sg * (dm.r / 4);
-        if (need > max_threads) continue;
+        if (need > 512) continue;
         int th = (int)((need + 31) / 32 * 32);
         if (th < 128) th = 128;
-        const int dg = (dm.d + G - 1) / G;
-        const int nw = th / 32;
-        int scratch = nw * MID_MAX_L;
-        if (nw * MID_MAX_C > scratch) scratch = nw * MID_MAX_C;
-        const int parts = th / dm.r > 0 ? th / dm.r : 1;
-        if (parts * dm.r > scratch) scratch = parts * dm.r;
-        size_t floats = (size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)dg + 2 * MID_MAX_C + MID_MAX_L + scratch +
-                        (size_t)dg * dm.C + 4;
-        const size_t budget = 200 * 1024 / sizeof(float);
-        const size_t ufl = 4 * (size_t)dm.L * th, wup = (size_t)dm.r * dg;
-        if (floats + ufl > budget) continue;              // the chain state must fit in shared memory: try more CTAs per sample
-        floats += ufl;
-        mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch;
+        int scratch;
+        size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch) + 4 * (size_t)dm.L * th;
+        if (floats > budget) continue;
+        const size_t wup = (size_t)dm.r * dg;
+        mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch; mp.gpt = 1; mp.smem_state = 1;
         mp.wup_smem = floats + wup <= budget ? 1 : 0;
         if (mp.wup_smem) floats += wup;
         mp.smem = sizeof(float) * floats;
         mp.ok = true;
         return mp;
     }
+    // otherwise: 8 CTAs per sample, up to 4 groups per thread, state parked in the du buffer
+    {
+        const int G = 8, Sg = (dm.S + G - 1) / G, dg = (dm.d + G - 1) / G;
+        const long long need = (long long)Sg * (dm.r / 4);
+        if (need > 4 * 512) return mp;
+        const int gpt = need <= 512 ? 1 : need <= 1024 ? 2 : 4;
+        int th = (int)(((need + gpt - 1) / gpt + 31) / 32 * 32);
+        if (th < 128) th = 128;
+        int scratch;
+        size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
+        if (floats > budget) return mp;
+        const size_t wup = (size_t)dm.r * dg;
+        mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch; mp.gpt = gpt; mp.smem_state = 0;
+        mp.wup_smem = floats + wup <= 96 * 1024 / sizeof(float) ? 1 : 0;     // keep several CTAs per SM
+        if (mp.wup_smem) floats += wup;
+        mp.smem = sizeof(float) * floats;
+        mp.ok = true;
+    }
     return mp;
 }
 
-template <int ACT, typename DU>
+template <int ACT, typename DU, int GPT, bool SMEM_STATE>
 inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
     static bool opted_in = false;                    // dynamic shared memory above 48 KB needs an opt-in per kernel
-    if (mp.smem > 48 * 1024 && !opted_in) {
-        cudaError_t e = cudaFuncSetAttribute(mid_cls_kernel<ACT, DU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (!opted_in) {
+        cudaError_t e = cudaFuncSetAttribute(mid_cls_kernel<ACT, DU, GPT, SMEM_STATE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)MID_SMEM_BUDGET);
         if (e != cudaSuccess) return e;
         opted_in = true;
     }
@@ -429,13 +532,23 @@ inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStr
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, DU>, p);
+    return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, DU, GPT, SMEM_STATE>, p);
+}
+
+template <int ACT, typename DU>
+inline cudaError_t mid_launch_shape(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
+    if (mp.smem_state) return mid_launch_one<ACT, DU, 1, true>(mp, p, stream);
+    switch (mp.gpt) {
+        case 1: return mid_launch_one<ACT, DU, 1, false>(mp, p, stream);
+        case 2: return mid_launch_one<ACT, DU, 2, false>(mp, p, stream);
+        default: return mid_launch_one<ACT, DU, 4, false>(mp, p, stream);
+    }
 }
 
 inline cudaError_t mid_launch(const MidPlan& mp, const MidParams& p, int act, bool du_bf16, cudaStream_t stream) {
     if (act == PAC_ACT_RELU)
-        return du_bf16 ? mid_launch_one<PAC_ACT_RELU, bf16>(mp, p, stream) : mid_launch_one<PAC_ACT_RELU, float>(mp, p, stream);
-    return du_bf16 ? mid_launch_one<PAC_ACT_IDENTITY, bf16>(mp, p, stream) : mid_launch_one<PAC_ACT_IDENTITY, float>(mp, p, stream);
+        return du_bf16 ? mid_launch_shape<PAC_ACT_RELU, bf16>(mp, p, stream) : mid_launch_shape<PAC_ACT_RELU, float>(mp, p, stream);
+    return du_bf16 ? mid_launch_shape<PAC_ACT_IDENTITY, bf16>(mp, p, stream) : mid_launch_shape<PAC_ACT_IDENTITY, float>(mp, p, stream);
 }
 
 }  // namespace pac

@@ -251,6 +251,9 @@ TC_SPECS = [
     (TC_BASE.scaled(name="tc_r256", S=64, d=320, r=256, L=2, B=2), 2, 0),   # widest adapter the path takes
     (TC_BASE.scaled(name="tc_identity", S=64, d=512, r=32, L=4, B=2), 2, 1),
     (TC_BASE.scaled(name="tc_deep", S=32, d=128, r=32, L=30, B=3, N=8), 3, 0),
+    # per-sample chain state too large for shared memory: 2 and 4 column groups per thread, state parked in du
+    (TC_BASE.scaled(name="tc_long_S", S=300, d=128, r=64, L=3, B=2, N=6), 2, 0),
+    (TC_BASE.scaled(name="tc_long_S_wide_r", S=500, d=128, r=128, L=2, B=2, N=4), 2, 1),
 ]
 
 
