@@ -390,3 +390,27 @@ def test_full_size_llama_step_matches_oracle():
     ids = [spec.N - 1, 0]
     case = SparseCase(spec, ids)
     tc_check(spec, spec.B, 0, ids=ids, case=case, head_tol=5e-3)
+
+
+def test_tensor_path_epoch_equals_step_loop():
+    """AdamW fused into the dW_down and finalisation kernels (epoch call) gives the same bits as
+    the separate optimizer kernel of the per-step calls."""
+    import paper_2408_10746_b200 as pac
+    spec = TC_BASE.scaled(N=32, name="tc_epoch")
+    case = Case(spec, materialize_cpu=False)
+    hp = pac.AdamW()
+    perm = pi.epoch_permutation(spec.N, 2)[:6 * spec.B]
+    a = case.context()
+    a.set_params(pi.random_params(spec, 3))
+    losses_a = a.train_epoch(perm, spec.B, hp)
+    b = case.context()
+    b.set_params(pi.random_params(spec, 3))
+    losses_b = []
+    for i in range(6):
+        losses_b.append(b.train_step(perm[i * spec.B:(i + 1) * spec.B]))
+        b.adam_step(hp)
+    assert np.array_equal(losses_a, np.array(losses_b, dtype=np.float32))
+    assert np.array_equal(a.get_params(), b.get_params())
+    ma, va, sa = a.get_opt_state()
+    mb, vb, sb = b.get_opt_state()
+    assert sa == sb == 6 and np.array_equal(ma, mb) and np.array_equal(va, vb)
