@@ -181,6 +181,48 @@ def run_reference(args, spec):
     }))
 
 
+def run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world):
+    """N > 1 with a real exchange step: every rank trains on its own cache shard and local
+    minibatch of B samples, gradients are averaged with one NCCL all-reduce per step (global
+    minibatch world*B), then every rank applies the same AdamW step."""
+    import torch
+    import paper_2408_10746_b200 as pac
+    from paper_2408_10746_b200.data_parallel import DataParallel, PacLocalTrainer
+    K, W, B = args.steps, args.warmup, spec.B
+    hp = pac.AdamW()
+    with torch.cuda.stream(stream):
+        dp = DataParallel(PacLocalTrainer(ctx))
+        for i in range(W):
+            dp.train_step(ids_host[(i % K) * B:(i % K + 1) * B]); dp.adam_step(hp)
+        sampler = ClockSampler(torch.cuda.current_device())
+        l0 = ctx.launch_count()
+        dist.barrier(); torch.cuda.synchronize()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(K):
+            dp.train_step(ids_host[i * B:(i + 1) * B]); dp.adam_step(hp)
+        e1.record(stream)
+        dist.barrier(); torch.cuda.synchronize()
+    clocks = sampler.finish()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    value = world * K * B / (ms * 1e-3)
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if spec.dtype == "bf16" else "f32",
+           "data": "synthetic",
+           "config": {"workload": workload_name(spec), "kernel_path": ctx.kernel_path(), "parallelism": f"dp{world}",
+                      "global_batch": world * B, "collective": "NCCL all-reduce of the flat fp32 adapter gradient per step"},
+           "clocks": clocks, "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 4 * B, "d2h_bytes_per_step": 4, "steps": K},
+           "gpu_launches": int(ctx.launch_count() - l0), "roofline": None, "cpu_baseline": None}
+    ctx.close()
+    dist.barrier()
+    dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -191,6 +233,9 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--force-simt", action="store_true", help="use the plain fp32-FMA kernels")
+    ap.add_argument("--parallelism", default="replicas", choices=["replicas", "dp"],
+                    help="N > 1: independent replicas (default) or data parallel with a per-step all-reduce of "
+                         "the adapter gradients (paper Section V-B)")
     ap.add_argument("--n-samples", type=int, default=0,
                     help="profiling aid: shrink the cache to this many samples (same per-step shapes); "
                          "the JSON line then names the reduced workload")
@@ -249,6 +294,9 @@ def main():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if world > 1 and args.parallelism == "dp":
+        return run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world)
 
     # ---------------- device-resident timing (value) ----------------
     ctx.train_epoch_dev(d_warm, B, hp, None)

@@ -137,6 +137,16 @@ pac_status pac_get_grads(pac_ctx* ctx, float* host);
 pac_status pac_get_opt_state(pac_ctx* ctx, float* m, float* v, long long* step);
 pac_status pac_set_opt_state(pac_ctx* ctx, const float* m, const float* v, long long step);
 
+/* Device addresses of the context's flat fp32 parameter and gradient vectors (pac_param_count
+ * floats each, owned by the context, valid until pac_destroy).  For data-parallel training
+ * (Section V-B: every device holds the adapter parameters, trains on its share of the minibatch
+ * and the devices combine gradients): a collective library can reduce *dev_grads in place between
+ * pac_train_step and pac_adam_step, and broadcast *dev_params once at the start.  After writing
+ * to the parameters through this pointer call pac_params_changed() so that derived copies (the
+ * bf16 weight shadow) are refreshed.  Order all accesses on the context's stream. */
+pac_status pac_device_buffers(pac_ctx* ctx, float** dev_params, float** dev_grads);
+pac_status pac_params_changed(pac_ctx* ctx);
+
 pac_status pac_set_option(pac_ctx* ctx, int option, int value);
 /* Per-kernel device times.  With PAC_OPT_KERNEL_TIMING = 1 the kernels of every later train
  * step are bracketed by CUDA events on the context's stream, in four groups:

@@ -25,7 +25,7 @@ STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_S
 EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init", "pac_train_step",
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
-           "pac_set_opt_state", "pac_set_option", "pac_kernel_times", "pac_launch_count", "pac_sync", "pac_last_error",
+           "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_launch_count", "pac_sync", "pac_last_error",
            "pac_kernel_path", "pac_eval_logits_static"]
 
 
@@ -89,6 +89,7 @@ def load_library() -> C.CDLL:
         "pac_set_opt_state": [P, P, P, LL], "pac_set_option": [P, I, I],
         "pac_launch_count": [P, C.POINTER(LL)], "pac_sync": [P],
         "pac_kernel_times": [P, C.POINTER(C.c_double), C.POINTER(LL)],
+        "pac_device_buffers": [P, C.POINTER(P), C.POINTER(P)], "pac_params_changed": [P],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -242,6 +243,22 @@ class PacContext:
         self._ck(self._lib.pac_kernel_times(self._h, ms, cnt))
         names = ["down_projection", "chain_head", "dw_down", "finalize"]
         return {n: (ms[i], cnt[i]) for i, n in enumerate(names)}
+
+    def device_buffers(self):
+        """Zero-copy torch views (CUDA, fp32) of the context's parameter and gradient vectors."""
+        import torch
+        pp, gp = C.c_void_p(), C.c_void_p()
+        self._ck(self._lib.pac_device_buffers(self._h, C.byref(pp), C.byref(gp)))
+        n = self.param_count()
+
+        class _View:
+            def __init__(self, ptr):
+                self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<f4", "data": (ptr, False), "version": 2}
+
+        return torch.as_tensor(_View(pp.value), device="cuda"), torch.as_tensor(_View(gp.value), device="cuda")
+
+    def params_changed(self):
+        self._ck(self._lib.pac_params_changed(self._h))
 
     def launch_count(self) -> int:
         n = C.c_longlong()

@@ -835,6 +835,19 @@ pac_status pac_set_opt_state(pac_ctx* c, const float* m, const float* v, long lo
     return PAC_OK;
 }
 
+pac_status pac_device_buffers(pac_ctx* c, float** dev_params, float** dev_grads) {
+    NEED_INIT(c, "pac_device_buffers");
+    if (!dev_params || !dev_grads) return fail(c, PAC_ERR_INVALID_ARG, "pac_device_buffers: NULL argument");
+    *dev_params = c->params;
+    *dev_grads = c->grads;
+    return PAC_OK;
+}
+
+pac_status pac_params_changed(pac_ctx* c) {
+    NEED_INIT(c, "pac_params_changed");
+    return refresh_shadow(c);
+}
+
 pac_status pac_set_option(pac_ctx* c, int option, int value) {
     NEED_CTX(c);
     if (option == PAC_OPT_KERNEL_PATH) {

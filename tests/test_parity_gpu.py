@@ -414,3 +414,37 @@ def test_tensor_path_epoch_equals_step_loop():
     ma, va, sa = a.get_opt_state()
     mb, vb, sb = b.get_opt_state()
     assert sa == sb == 6 and np.array_equal(ma, mb) and np.array_equal(va, vb)
+
+
+def test_device_buffer_views_and_single_rank_data_parallel(tiny):
+    """The zero-copy views alias the library's buffers (what an in-place all-reduce needs), and
+    the data-parallel wrapper with one rank is the plain trainer."""
+    import paper_2408_10746_b200 as pac
+    from paper_2408_10746_b200.data_parallel import DataParallel, PacLocalTrainer
+    hp = pac.AdamW()
+    ids = list(range(8))
+    ref = tiny.context()
+    ref.set_params(pi.random_params(TINY, 3))
+    ref_loss = ref.train_step(ids)
+    ref.adam_step(hp)
+
+    ctx = tiny.context()
+    params, grads = ctx.device_buffers()
+    params.copy_(torch.from_numpy(pi.random_params(TINY, 3)).cuda())      # write through the view ...
+    torch.cuda.synchronize()
+    ctx.params_changed()
+    assert np.array_equal(ctx.get_params(), pi.random_params(TINY, 3))    # ... is seen by the library
+    import torch.distributed as dist
+    created = False
+    if not dist.is_initialized():
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29517", rank=0, world_size=1)
+        created = True
+    try:
+        dp = DataParallel(PacLocalTrainer(ctx))
+        loss = dp.train_step(ids)
+        assert np.array_equal(grads.cpu().numpy(), ctx.get_grads())
+        dp.adam_step(hp)
+    finally:
+        if created:
+            dist.destroy_process_group()
+    assert loss == ref_loss and np.array_equal(ctx.get_params(), ref.get_params())
