@@ -434,9 +434,11 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         bias_corrections(hp, c->step, &f.bc1, &f.bc2);
         f.wdT = sc.wdT;
     }
+    f.wd_blocks = (int)cdiv(c->lay.lam / 4, 256);
+    const unsigned rest_blocks = cdiv(c->lay.total - c->lay.lam, 256);
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    pdl_launch_config(&cfg, attr, dim3(cdiv(c->lay.total, 256) + 1), dim3(256), 0, c->stream);   // + one block for lambda and the loss
+    pdl_launch_config(&cfg, attr, dim3(f.wd_blocks + rest_blocks + 1), dim3(256), 0, c->stream);   // + one block for lambda and the loss
     cudaError_t le = cudaLaunchKernelEx(&cfg, finalize_cls_kernel, f);
     c->launches++;
     if (le != cudaSuccess) return fail(c, PAC_ERR_CUDA, "finalize kernel launch failed: %s", cudaGetErrorString(le));
@@ -467,8 +469,10 @@ pac_status adam_enqueue(pac_ctx* c, const pac_adamw* hp) {
     c->step += 1;
     float bc1, bc2;
     bias_corrections(hp, c->step, &bc1, &bc2);
-    adamw_kernel<<<cdiv(c->lay.total, 256), 256, 0, c->stream>>>(c->params, c->grads, c->m, c->v, c->lay.total, c->lay,
-                                                                 *hp, bc1, bc2, c->sc.wdT, c->dm.d, c->dm.r);
+    const int wd_blocks = (c->lay.lam % 4 == 0) ? (int)cdiv(c->lay.lam / 4, 256) : 0;
+    const unsigned rest = cdiv(c->lay.total - (wd_blocks ? c->lay.lam : 0), 256);
+    adamw_kernel<<<wd_blocks + rest, 256, 0, c->stream>>>(c->params, c->grads, c->m, c->v, c->lay.total, c->lay, *hp, bc1, bc2,
+                                                          c->sc.wdT, c->dm.d, c->dm.r, wd_blocks);
     LAUNCH_CHECK(c);
     return PAC_OK;
 }

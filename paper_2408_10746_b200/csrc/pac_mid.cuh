@@ -381,6 +381,7 @@ struct FinalizeParams {
     const float* lam_part; int lam_blocks;
     const float *pooled_a, *gvec, *pooled_y, *dlogits, *loss_b;
     float* grads; float* loss_out;
+    int wd_blocks;                                           // leading blocks that handle W_down, 4 elements per thread
     // AdamW
     int adam;
     float *params, *m, *v;
@@ -414,18 +415,29 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         }
         return;
     }
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if ((int)blockIdx.x < f.wd_blocks) {
+        // W_down block, four consecutive elements per thread
+        const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+        if (i >= lay.lam) return;
+        float4 g4;
+        if (f.splits > 1) {
+            g4 = *reinterpret_cast<const float4*>(f.dw_part + i);
+            for (int j = 1; j < f.splits; ++j) {                 // split order
+                const float4 q = *reinterpret_cast<const float4*>(f.dw_part + (long long)j * f.dw_elems + i);
+                g4.x += q.x; g4.y += q.y; g4.z += q.z; g4.w += q.w;
+            }
+            *reinterpret_cast<float4*>(f.grads + i) = g4;
+        } else {
+            g4 = *reinterpret_cast<const float4*>(f.grads + i);
+        }
+        if (f.adam) adamw_w_down4(f.params, f.m, f.v, i, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        return;
+    }
+    const long long i = lay.lam + (long long)(blockIdx.x - f.wd_blocks) * blockDim.x + threadIdx.x;
     if (i >= lay.total) return;
     float g;
-    if (i >= lay.lam && i < lay.w_up) return;            // lambda is handled by the last block
-    if (i < lay.lam) {
-        if (f.splits > 1) {
-            g = f.dw_part[i];
-            for (int j = 1; j < f.splits; ++j) g += f.dw_part[(long long)j * f.dw_elems + i];
-        } else {
-            g = f.grads[i];
-        }
-    } else if (i < lay.w_head) {
+    if (i < lay.w_up) return;                            // lambda is handled by the last block
+    if (i < lay.w_head) {
         const long long e = i - lay.w_up;
         const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
         g = 0.f;

@@ -432,20 +432,26 @@ __global__ void mean_kernel(const float* __restrict__ x, int n, float* __restric
 // ---------------------------------------------------------------------------
 // One element of the update, shared by every kernel that applies AdamW so that fused and
 // separate updates are bit-identical.
+// The arithmetic of one element: returns the new parameter, updates mi / vi in place.
+__device__ __forceinline__ float adamw_math(float th, float& mi, float& vi, float gi, bool decays, const pac_adamw& hp,
+                                            float bc1, float bc2) {
+    // every rounding is spelled out (no contraction into FMAs), in the order the update is written:
+    // m = b1 m + (1-b1) g;  v = b2 v + ((1-b2) g) g;  theta = (theta - lr wd theta) - (lr mhat)/(sqrt(vhat)+eps)
+    mi = __fadd_rn(__fmul_rn(hp.beta1, mi), __fmul_rn(__fsub_rn(1.f, hp.beta1), gi));
+    vi = __fadd_rn(__fmul_rn(hp.beta2, vi), __fmul_rn(__fmul_rn(__fsub_rn(1.f, hp.beta2), gi), gi));
+    const float mhat = __fdiv_rn(mi, bc1), vhat = __fdiv_rn(vi, bc2);
+    const float decay = decays ? __fmul_rn(__fmul_rn(hp.lr, hp.weight_decay), th) : 0.f;
+    return __fsub_rn(__fsub_rn(th, decay), __fdiv_rn(__fmul_rn(hp.lr, mhat), __fadd_rn(__fsqrt_rn(vhat), hp.eps)));
+}
+
 __device__ __forceinline__ void adamw_element(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
                                               long long i, float gi, const ParamLayout& lay, const pac_adamw& hp,
                                               float bc1, float bc2, bf16* __restrict__ wdT, int d, int r) {
     const bool decays = (i < lay.lam) || (i >= lay.w_up && i < lay.b_head);
-    float th = p[i];
-    // every rounding is spelled out (no contraction into FMAs), in the order the update is written:
-    // m = b1 m + (1-b1) g;  v = b2 v + ((1-b2) g) g;  theta = (theta - lr wd theta) - (lr mhat)/(sqrt(vhat)+eps)
-    const float mi = __fadd_rn(__fmul_rn(hp.beta1, m[i]), __fmul_rn(__fsub_rn(1.f, hp.beta1), gi));
-    const float vi = __fadd_rn(__fmul_rn(hp.beta2, v[i]), __fmul_rn(__fmul_rn(__fsub_rn(1.f, hp.beta2), gi), gi));
+    float mi = m[i], vi = v[i];
+    const float th = adamw_math(p[i], mi, vi, gi, decays, hp, bc1, bc2);
     m[i] = mi;
     v[i] = vi;
-    const float mhat = __fdiv_rn(mi, bc1), vhat = __fdiv_rn(vi, bc2);
-    const float decay = decays ? __fmul_rn(__fmul_rn(hp.lr, hp.weight_decay), th) : 0.f;
-    th = __fsub_rn(__fsub_rn(th, decay), __fdiv_rn(__fmul_rn(hp.lr, mhat), __fadd_rn(__fsqrt_rn(vhat), hp.eps)));
     p[i] = th;
     if (wdT && i < lay.lam) {
         const long long dr = (long long)d * r, l = i / dr, rem = i - l * dr;
@@ -455,10 +461,44 @@ __device__ __forceinline__ void adamw_element(float* __restrict__ p, float* __re
     }
 }
 
+// Four consecutive elements of the W_down block (i a multiple of 4; d*r is a multiple of 4, so
+// the four share a layer): vector loads and stores, the same arithmetic per element.
+__device__ __forceinline__ void adamw_w_down4(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
+                                              long long i, float4 g4, const pac_adamw& hp, float bc1, float bc2,
+                                              bf16* __restrict__ wdT, int d, int r) {
+    float4 p4 = *reinterpret_cast<float4*>(p + i), m4 = *reinterpret_cast<float4*>(m + i), v4 = *reinterpret_cast<float4*>(v + i);
+    p4.x = adamw_math(p4.x, m4.x, v4.x, g4.x, true, hp, bc1, bc2);
+    p4.y = adamw_math(p4.y, m4.y, v4.y, g4.y, true, hp, bc1, bc2);
+    p4.z = adamw_math(p4.z, m4.z, v4.z, g4.z, true, hp, bc1, bc2);
+    p4.w = adamw_math(p4.w, m4.w, v4.w, g4.w, true, hp, bc1, bc2);
+    *reinterpret_cast<float4*>(p + i) = p4;
+    *reinterpret_cast<float4*>(m + i) = m4;
+    *reinterpret_cast<float4*>(v + i) = v4;
+    if (wdT) {
+        const long long dr = (long long)d * r, l = i / dr, rem = i - l * dr;
+        const float th[4] = {p4.x, p4.y, p4.z, p4.w};
+        bf16 hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            hi[e] = __float2bfloat16(th[e]);
+            lo[e] = __float2bfloat16(th[e] - __bfloat162float(hi[e]));
+        }
+        *reinterpret_cast<uint2*>(wdT + (l * 2 + 0) * dr + rem) = *reinterpret_cast<const uint2*>(hi);
+        *reinterpret_cast<uint2*>(wdT + (l * 2 + 1) * dr + rem) = *reinterpret_cast<const uint2*>(lo);
+    }
+}
+
+// wd_blocks leading blocks take the W_down block four elements per thread (0 when its size is
+// not a multiple of 4); the remaining blocks take everything else one element per thread.
 __global__ void adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
                              float* __restrict__ v, long long n, ParamLayout lay, pac_adamw hp, float bc1,
-                             float bc2, bf16* __restrict__ wdT, int d, int r) {
-    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+                             float bc2, bf16* __restrict__ wdT, int d, int r, int wd_blocks) {
+    if ((int)blockIdx.x < wd_blocks) {
+        const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+        if (i < lay.lam) adamw_w_down4(p, m, v, i, *reinterpret_cast<const float4*>(g + i), hp, bc1, bc2, wdT, d, r);
+        return;
+    }
+    const long long i = (wd_blocks ? lay.lam : 0) + (long long)(blockIdx.x - wd_blocks) * blockDim.x + threadIdx.x;
     if (i >= n) return;
     adamw_element(p, m, v, i, g[i], lay, hp, bc1, bc2, wdT, d, r);
 }
