@@ -223,6 +223,35 @@ def run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world)
         print(json.dumps(out))
 
 
+def run_codec(args):
+    """Streaming throughput of pac_quantize_absmax / pac_dequantize_absmax on 2^28 fp32 values
+    (1 GiB in, far above L2), against the measured copy bandwidth; 5 algorithmic bytes per element."""
+    import torch
+    import paper_2408_10746_b200 as pac
+    n = 1 << 28
+    x = torch.randn(n, device="cuda")
+    peaks = load_peaks()
+    res = {}
+    for block in (64, 4096):
+        q, c = pac.quantize_absmax(x, block)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        for _ in range(3):
+            q, c = pac.quantize_absmax(x, block)
+            out = pac.dequantize_absmax(q, c, block)
+        torch.cuda.synchronize()
+        tq, td = [], []
+        for _ in range(5):
+            e[0].record(); q, c = pac.quantize_absmax(x, block)
+            e[1].record(); out = pac.dequantize_absmax(q, c, block)
+            e[2].record(); torch.cuda.synchronize()
+            tq.append(e[0].elapsed_time(e[1])); td.append(e[1].elapsed_time(e[2]))
+        gq, gd = 5 * n / (np.median(tq) * 1e-3) / 1e9, 5 * n / (np.median(td) * 1e-3) / 1e9
+        res[f"block{block}"] = {"quantize_gbs": gq, "quantize_frac": gq / peaks["hbm_gbs"], "dequantize_gbs": gd,
+                                "dequantize_frac": gd / peaks["hbm_gbs"]}
+    print(json.dumps({"metric": "absmax_int8_codec_stream", "unit": "GB/s", "n_elements": n, "dtype": "f32->i8",
+                      "data": "synthetic", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "results": res}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -236,6 +265,8 @@ def main():
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "dp"],
                     help="N > 1: independent replicas (default) or data parallel with a per-step all-reduce of "
                          "the adapter gradients (paper Section V-B)")
+    ap.add_argument("--codec", action="store_true",
+                    help="measure the block-wise absmax INT8 codec (paper Eq. 1-2) instead of the train step")
     ap.add_argument("--n-samples", type=int, default=0,
                     help="profiling aid: shrink the cache to this many samples (same per-step shapes); "
                          "the JSON line then names the reduced workload")
@@ -247,6 +278,8 @@ def main():
         spec = spec.scaled(N=args.n_samples, name=f"{spec.name}[N={args.n_samples}]")
     if args.impl == "reference":
         return run_reference(args, spec)
+    if args.codec:
+        return run_codec(args)
 
     import torch
     import paper_2408_10746_b200 as pac

@@ -167,6 +167,20 @@ const char* pac_last_error(const pac_ctx* ctx);
 /* "tensor" or "simt": which kernels the next train step will use (valid after adapter_init). */
 const char* pac_kernel_path(const pac_ctx* ctx);
 
+/* Block-wise absmax INT8 quantisation, Section IV-D, Eq. 1 (the paper applies it to the frozen
+ * backbone's weights; here it is a stand-alone codec over any fp32 device array):
+ *     c_j = 127 / absmax(block j),   q = round(c_j * x)  (fp32 arithmetic, ties to even)
+ * for every block j of `block` consecutive elements (the last may be shorter); an all-zero block
+ * gets c_j = 0 and codes 0.  dev_x: device, n floats, read-only.  dev_q: device, n int8 codes.
+ * dev_c: device, ceil(n / block) quantisation constants.  Enqueued on cuda_stream (NULL: default
+ * stream) of `device`; nothing is allocated.  Errors: PAC_ERR_INVALID_ARG for NULL pointers or
+ * non-positive sizes, PAC_ERR_CUDA when the launch fails. */
+pac_status pac_quantize_absmax(int device, void* cuda_stream, const float* dev_x, long long n, int block,
+                               signed char* dev_q, float* dev_c);
+/* Dequantisation, Eq. 2: dev_out[i] = dev_q[i] / c_j (0 where c_j == 0), fp32.  Same conventions. */
+pac_status pac_dequantize_absmax(int device, void* cuda_stream, const signed char* dev_q, const float* dev_c, long long n,
+                                 int block, float* dev_out);
+
 /* Evaluation forward that allocates nothing (the paper has no counterpart; this is a
  * packaging variant of pac_eval_logits for the mean-pool classifier head).
  *

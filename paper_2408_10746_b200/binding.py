@@ -26,7 +26,7 @@ EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init"
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
            "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_launch_count", "pac_sync", "pac_last_error",
-           "pac_kernel_path", "pac_eval_logits_static"]
+           "pac_kernel_path", "pac_eval_logits_static", "pac_quantize_absmax", "pac_dequantize_absmax"]
 
 
 class PacError(RuntimeError):
@@ -97,6 +97,10 @@ def load_library() -> C.CDLL:
         fn.restype = I
     lib.pac_eval_logits_static.argtypes = [I, P, P, I, LL, I, I, I, P, I, I, I, P, I, P, C.c_char_p, I]
     lib.pac_eval_logits_static.restype = I
+    lib.pac_quantize_absmax.argtypes = [I, P, P, LL, I, P, P]
+    lib.pac_quantize_absmax.restype = I
+    lib.pac_dequantize_absmax.argtypes = [I, P, P, P, LL, I, P]
+    lib.pac_dequantize_absmax.restype = I
     lib.pac_last_error.argtypes = [P]
     lib.pac_last_error.restype = C.c_char_p
     lib.pac_kernel_path.argtypes = [P]
@@ -296,4 +300,29 @@ def eval_logits_static(cache, dev_params, r: int, n_out: int, dev_sample_ids, ou
                                     dev_sample_ids.numel(), out.data_ptr(), err, 512)
     if st != 0:
         raise PacError(st, err.value.decode())
+    return out
+
+
+def quantize_absmax(x, block: int, device: int = 0, stream: Optional[int] = None):
+    """Block-wise absmax INT8 codes and constants of a CUDA fp32 tensor (paper Eq. 1)."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    n = x.numel()
+    q = torch.empty(n, dtype=torch.int8, device=x.device)
+    c = torch.empty((n + block - 1) // block, dtype=torch.float32, device=x.device)
+    st = load_library().pac_quantize_absmax(device, C.c_void_p(stream) if stream else None, x.data_ptr(), n, block,
+                                            q.data_ptr(), c.data_ptr())
+    if st != 0:
+        raise PacError(st, "pac_quantize_absmax failed")
+    return q, c
+
+
+def dequantize_absmax(q, c, block: int, device: int = 0, stream: Optional[int] = None):
+    """fp32 tensor from codes and constants (paper Eq. 2)."""
+    import torch
+    out = torch.empty(q.numel(), dtype=torch.float32, device=q.device)
+    st = load_library().pac_dequantize_absmax(device, C.c_void_p(stream) if stream else None, q.data_ptr(), c.data_ptr(),
+                                              q.numel(), block, out.data_ptr())
+    if st != 0:
+        raise PacError(st, "pac_dequantize_absmax failed")
     return out

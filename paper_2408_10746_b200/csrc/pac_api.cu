@@ -11,6 +11,7 @@
 #include "pac_tensor.cuh"
 #include "pac_mid.cuh"
 #include "pac_gemm.cuh"
+#include "pac_quant.cuh"
 
 using namespace pac;
 
@@ -1022,4 +1023,52 @@ extern "C" pac_status pac_eval_logits_static(int device, void* cuda_stream, cons
             : static_forward<bf16>(st, (const bf16*)dev_cache, N, L, S, d, dev_params, lay, r, act, n_out, dev_sample_ids, B, dev_out, u, a, pooled_a, hbar_b, iota);
     if (e != cudaSuccess) return static_fail(err, err_len, PAC_ERR_CUDA, "pac_eval_logits_static: kernel launch failed: %s", cudaGetErrorString(e));
     return PAC_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Block-wise absmax INT8 codec (Section IV-D, Eq. 1-2)
+// ---------------------------------------------------------------------------
+extern "C" pac_status pac_quantize_absmax(int device, void* cuda_stream, const float* dev_x, long long n, int block,
+                                          signed char* dev_q, float* dev_c) {
+    if (!dev_x || !dev_q || !dev_c || n < 1 || block < 1) return PAC_ERR_INVALID_ARG;
+    if (cudaSetDevice(device) != cudaSuccess) return PAC_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const long long n_blocks = (n + block - 1) / block;
+    const bool vec = (n % 4 == 0) && (((uintptr_t)dev_x & 15) == 0) && (((uintptr_t)dev_q & 3) == 0);
+    if (vec && (block == 16 || block == 32 || block == 64 || block == 128)) {
+        const long long n4 = n / 4, want = (n4 + 255) / 256;
+        const unsigned grid = (unsigned)(want < 148LL * 32 ? want : 148LL * 32);
+        quantize_absmax_subwarp_kernel<<<grid, 256, 0, st>>>((const float4*)dev_x, n4, block / 4, (char4*)dev_q, dev_c);
+    } else if (vec && block % 1024 == 0 && block <= 4096 && n_blocks <= 0x7fffffffLL) {
+        const long long n4 = n / 4;
+        switch (block / 1024) {
+            case 1: quantize_absmax_cta_reg_kernel<1><<<(unsigned)n_blocks, 256, 0, st>>>((const float4*)dev_x, n4, (char4*)dev_q, dev_c); break;
+            case 2: quantize_absmax_cta_reg_kernel<2><<<(unsigned)n_blocks, 256, 0, st>>>((const float4*)dev_x, n4, (char4*)dev_q, dev_c); break;
+            case 3: quantize_absmax_cta_reg_kernel<3><<<(unsigned)n_blocks, 256, 0, st>>>((const float4*)dev_x, n4, (char4*)dev_q, dev_c); break;
+            default: quantize_absmax_cta_reg_kernel<4><<<(unsigned)n_blocks, 256, 0, st>>>((const float4*)dev_x, n4, (char4*)dev_q, dev_c); break;
+        }
+    } else if (block <= QUANT_WARP_MAX) {
+        const long long warps = n_blocks < 148LL * 64 ? n_blocks : 148LL * 64;      // up to 8 CTAs of 8 warps per SM
+        quantize_absmax_warp_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dev_x, n, block, n_blocks, dev_q, dev_c);
+    } else {
+        if (n_blocks > 0x7fffffffLL) return PAC_ERR_UNSUPPORTED;
+        quantize_absmax_cta_kernel<<<(unsigned)n_blocks, 256, 0, st>>>(dev_x, n, block, dev_q, dev_c);
+    }
+    return cudaGetLastError() == cudaSuccess ? PAC_OK : PAC_ERR_CUDA;
+}
+
+extern "C" pac_status pac_dequantize_absmax(int device, void* cuda_stream, const signed char* dev_q, const float* dev_c,
+                                            long long n, int block, float* dev_out) {
+    if (!dev_q || !dev_c || !dev_out || n < 1 || block < 1) return PAC_ERR_INVALID_ARG;
+    if (cudaSetDevice(device) != cudaSuccess) return PAC_ERR_CUDA;
+    if (n % 4 == 0 && block % 4 == 0 && ((uintptr_t)dev_q & 3) == 0 && ((uintptr_t)dev_out & 15) == 0) {
+        const long long n4 = n / 4, want = (n4 + 1023) / 1024;
+        const unsigned grid = (unsigned)(want < 148LL * 32 ? want : 148LL * 32);
+        dequantize_absmax_vec_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>((const char4*)dev_q, dev_c, n4, block / 4, (float4*)dev_out);
+    } else {
+        const long long want = (n + 255) / 256;
+        const unsigned grid = (unsigned)(want < 148LL * 16 ? want : 148LL * 16);
+        dequantize_absmax_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(dev_q, dev_c, n, block, dev_out);
+    }
+    return cudaGetLastError() == cudaSuccess ? PAC_OK : PAC_ERR_CUDA;
 }
