@@ -198,9 +198,14 @@ class PacContext:
         self._ck(self._lib.pac_gather(self._h, ids.ctypes.data, ids.size, out.data_ptr()))
         return out
 
-    def train_epoch(self, perm, B: int, hp: AdamW, want_losses: bool = True) -> Optional[np.ndarray]:
+    def train_epoch(self, perm, B: int, hp: AdamW, want_losses: bool = True, losses_out: Optional[np.ndarray] = None):
+        """perm: host int32 ids (n a multiple of B).  losses_out: optional host float32 array of n/B
+        entries to receive the losses (e.g. a view of pinned memory); otherwise one is allocated."""
         ids = _ids(perm)
-        losses = np.empty(max(1, ids.size // max(B, 1)), dtype=np.float32) if want_losses else None
+        losses = None
+        if want_losses:
+            losses = losses_out if losses_out is not None else np.empty(max(1, ids.size // max(B, 1)), dtype=np.float32)
+            assert losses.dtype == np.float32 and losses.size >= ids.size // max(B, 1)
         self._ck(self._lib.pac_train_epoch(self._h, ids.ctypes.data, ids.size, B, C.byref(hp._c()),
                                            losses.ctypes.data if want_losses else None))
         return losses
