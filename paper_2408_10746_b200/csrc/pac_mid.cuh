@@ -30,6 +30,7 @@ struct MidParams {
     int train;
     int scratch;                // floats of block-local reduction scratch
     int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
+    int layers_per_cta;         // STATE_CLUSTER: layers whose u tiles each CTA of the cluster holds
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
     void* du;                   // [L][max_rows][r] bf16 or fp32
@@ -57,40 +58,68 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// GPT: 4-column groups per thread.  SMEM_STATE: the per-layer chain state (u_l, then u_l - a_{l-1})
-// sits in shared memory (prefetched with cp.async); otherwise u is read from global memory and
-// u_l - a_{l-1} is parked, in du's type, in the very slot of the du buffer that the reverse pass
-// overwrites with du_l once it has consumed it.
-template <int ACT, typename DU, int GPT, bool SMEM_STATE>
-__global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidParams p) {
+// Where the per-layer chain state (u_l on the way in, u_l - a_{l-1} for the reverse pass) lives.
+enum {
+    STATE_SMEM = 0,      // this CTA's shared memory, prefetched from the global u buffer with cp.async
+    STATE_DU = 1,        // u read from global memory; u_l - a_{l-1} parked, in du's type, in the du slot
+                         // that the reverse pass overwrites with du_l once it has consumed it
+    STATE_CLUSTER = 2    // u tiles produced by the cluster's own GEMMs: layer l sits in the shared memory
+                         // of CTA l / layers_per_cta as [layer][128 tokens][r] fp32 and is updated in place
+                         // through distributed shared memory (every element has exactly one owner thread)
+};
+
+// The small per-CTA vectors of the head computation, carved from one shared-memory region.
+struct MidShared {
+    float *aL, *colsum, *lpart, *dpart, *pooled, *daL, *py, *gk, *lg, *lam_s, *wh_s, *lred, *wup_s;
+};
+__device__ __forceinline__ MidShared mid_carve(float* sm, const MidParams& p) {
+    MidShared h;
+    h.aL = sm;                                        // [Sg][r]   a_L of this CTA's tokens
+    h.colsum = h.aL + (size_t)p.Sg * p.r;             // [r]       exchanged through DSMEM
+    h.lpart = h.colsum + p.r;                         // [MID_MAX_C] exchanged
+    h.dpart = h.lpart + MID_MAX_C;                    // [r]       exchanged
+    h.pooled = h.dpart + p.r;                         // [r]
+    h.daL = h.pooled + p.r;                           // [r]
+    h.py = h.daL + p.r;                               // [dg]  hbar slice, then mean_s y
+    h.gk = h.py + p.dg;                               // [dg]
+    h.lg = h.gk + p.dg;                               // [MID_MAX_C] logits, then dlogits
+    h.lam_s = h.lg + MID_MAX_C;                       // [MID_MAX_L]
+    h.wh_s = h.lam_s + MID_MAX_L;                     // [dg][C] slice of W_head
+    h.lred = h.wh_s + (size_t)p.dg * p.C;             // [nwarps][MID_MAX_L]; also [nwarps][MID_MAX_C] and [parts][r] scratch
+    h.wup_s = h.lred + (size_t)p.scratch;             // [r][dg] slice of W_up (when p.wup_smem)
+    return h;
+}
+
+// cp.async requests for the head operands of CTA rank q (hbar slice of sample `id`, W_head and W_up
+// slices) and plain loads of lambda, issued by threads t0 .. t0 + nthr - 1 of the block.
+__device__ __forceinline__ void mid_prefetch_head(const MidParams& p, const MidShared& h, int q, long long id, int t, int nthr) {
+    const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));
+    for (int kk = t; kk < kn; kk += nthr) cp_async_4(h.py + kk, p.hbar + id * p.d + k0 + kk);
+    for (int e = t; e < kn * p.C; e += nthr) cp_async_4(h.wh_s + e, p.W_head + (long long)k0 * p.C + e);
+    if (p.wup_smem) {
+        const int w = t >> 5, ln = t & 31, nw = nthr >> 5;
+        for (int j = w; j < p.r; j += nw)
+            for (int kk = ln; kk < kn; kk += 32) cp_async_4(h.wup_s + (size_t)j * p.dg + kk, p.W_up + (long long)j * p.d + k0 + kk);
+    }
+    for (int l = t; l < MID_MAX_L; l += nthr) h.lam_s[l] = l < p.L ? p.lam[l] : 0.f;
+}
+
+// Everything after the down-projections for one sample, executed by one CTA (rank q) of the
+// sample's cluster.  GPT: 4-column groups per thread.  u_s: STATE_SMEM: [L][GPT][nt] float4 state;
+// STATE_CLUSTER: this CTA's [layers_per_cta][128][r] fp32 u tiles.  head_prefetched: the caller has
+// already issued mid_prefetch_head (its threads still have to wait for their copies here).
+template <int ACT, typename DU, int GPT, int STATE>
+__device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& cluster, float4* u_s, const MidShared& h,
+                                         bool head_prefetched) {
     constexpr int LT = MID_MAX_L;
-    cg::cluster_group cluster = cg::this_cluster();
     const int q = (int)cluster.block_rank();
     const int b = blockIdx.x / p.G;
     const int t = threadIdx.x, nt = blockDim.x;
     const int r = p.r, L = p.L, C = p.C;
     const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
+    float *aL = h.aL, *colsum = h.colsum, *lpart = h.lpart, *dpart = h.dpart, *pooled = h.pooled, *daL = h.daL, *py = h.py,
+          *gk = h.gk, *lg = h.lg, *lam_s = h.lam_s, *wh_s = h.wh_s, *lred = h.lred, *wup_s = h.wup_s;
 
-    extern __shared__ float4 sm4[];
-    float4* u_s = sm4;                           // [L][GPT][nt] each thread's own u values, later u_l - a_{l-1}
-    float* sm = reinterpret_cast<float*>(sm4 + (SMEM_STATE ? (size_t)L * GPT * nt : 0));
-    float* aL = sm;                              // [Sg][r]   a_L of this CTA's tokens
-    float* colsum = aL + (size_t)p.Sg * r;       // [r]       exchanged through DSMEM
-    float* lpart = colsum + r;                   // [MID_MAX_C] exchanged
-    float* dpart = lpart + MID_MAX_C;            // [r]       exchanged
-    float* pooled = dpart + r;                   // [r]
-    float* daL = pooled + r;                     // [r]
-    float* py = daL + r;                         // [dg]  hbar slice, then mean_s y
-    float* gk = py + p.dg;                       // [dg]
-    float* lg = gk + p.dg;                       // [MID_MAX_C] logits, then dlogits
-    float* lam_s = lg + MID_MAX_C;               // [LT]
-    float* wh_s = lam_s + LT;                    // [dg][C] slice of W_head
-    float* lred = wh_s + (size_t)p.dg * C;       // [nwarps][LT]; also [nwarps][MID_MAX_C] and [parts][r] scratch
-    float* wup_s = lred + (size_t)p.scratch;     // [r][dg] slice of W_up (when p.wup_smem)
-
-    pdl_trigger();
-    pdl_wait();             // u comes from the kernel before this one
-    // ---- everything this CTA will read from global memory is requested up front ----
     const int groups_per_tok = r >> 2;
     int s_local[GPT], j4[GPT];
     bool live[GPT];
@@ -106,13 +135,21 @@ __global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidPar
     }
     DU* du = reinterpret_cast<DU*>(p.du);
     // layer l of group g: read u, park / fetch the reverse-pass state
+    auto cluster_slot = [&](int l, int g) -> float4* {      // STATE_CLUSTER: the element's home in the cluster
+        const int owner = l / p.layers_per_cta, li = l - owner * p.layers_per_cta;
+        float* tile = cluster.map_shared_rank(reinterpret_cast<float*>(u_s), owner);
+        return reinterpret_cast<float4*>(tile + ((size_t)li * 128 + (q * p.Sg + s_local[g])) * r + j4[g]);
+    };
     auto load_u = [&](int l, int g) -> float4 {
-        if constexpr (SMEM_STATE) return u_s[((size_t)l * GPT + g) * nt + t];
+        if constexpr (STATE == STATE_SMEM) return u_s[((size_t)l * GPT + g) * nt + t];
+        else if constexpr (STATE == STATE_CLUSTER) return *cluster_slot(l, g);
         else return *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base[g]);
     };
     auto store_w = [&](int l, int g, const float* wv) {
-        if constexpr (SMEM_STATE) {
+        if constexpr (STATE == STATE_SMEM) {
             u_s[((size_t)l * GPT + g) * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
+        } else if constexpr (STATE == STATE_CLUSTER) {
+            *cluster_slot(l, g) = make_float4(wv[0], wv[1], wv[2], wv[3]);
         } else if constexpr (sizeof(DU) == 2) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]), hi = __floats2bfloat162_rn(wv[2], wv[3]);
             uint2 pk;
@@ -124,8 +161,10 @@ __global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidPar
         }
     };
     auto load_w = [&](int l, int g) -> float4 {
-        if constexpr (SMEM_STATE) {
+        if constexpr (STATE == STATE_SMEM) {
             return u_s[((size_t)l * GPT + g) * nt + t];
+        } else if constexpr (STATE == STATE_CLUSTER) {
+            return *cluster_slot(l, g);
         } else if constexpr (sizeof(DU) == 2) {
             const uint2 pk = *reinterpret_cast<const uint2*>(du + (long long)l * p.lstride + base[g]);
             const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
@@ -135,7 +174,7 @@ __global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidPar
             return *reinterpret_cast<const float4*>(du + (long long)l * p.lstride + base[g]);
         }
     };
-    if constexpr (SMEM_STATE) {
+    if constexpr (STATE == STATE_SMEM) {
 #pragma unroll
         for (int g = 0; g < GPT; ++g)
             if (live[g])
@@ -144,14 +183,9 @@ __global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidPar
     cp_async_commit();                                                          // group: u
     const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
     const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
-    for (int kk = t; kk < kn; kk += nt) cp_async_4(py + kk, p.hbar + id * p.d + k0 + kk);
-    for (int e = t; e < kn * C; e += nt) cp_async_4(wh_s + e, p.W_head + (long long)k0 * C + e);
-    if (p.wup_smem)
-        for (int j = warp; j < r; j += nwarps)
-            for (int kk = lane; kk < kn; kk += 32) cp_async_4(wup_s + (size_t)j * p.dg + kk, p.W_up + (long long)j * p.d + k0 + kk);
+    if (!head_prefetched) mid_prefetch_head(p, h, q, id, t, nt);
     cp_async_commit();                                                          // group: head operands
     const int label = p.train ? p.labels[id] : 0;
-    if (t < LT) lam_s[t] = t < L ? p.lam[t] : 0.f;
     __syncthreads();
     cp_async_wait_group<1>();                                                   // own u values have landed
 
@@ -365,6 +399,19 @@ __global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidPar
         p.lam_part[(long long)t * (p.B * p.G) + blockIdx.x] = acc;
     }
     cluster.sync();                                       // keep shared memory alive until every peer has read it
+}
+
+// The stand-alone kernel: u comes from the global buffer written by the down-projection kernel.
+template <int ACT, typename DU, int GPT, bool SMEM_STATE>
+__global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ float4 sm4[];
+    float4* u_s = sm4;                           // [L][GPT][nt] each thread's own u values, later u_l - a_{l-1}
+    float* sm = reinterpret_cast<float*>(sm4 + (SMEM_STATE ? (size_t)p.L * GPT * blockDim.x : 0));
+    const MidShared h = mid_carve(sm, p);
+    pdl_trigger();
+    pdl_wait();             // u comes from the kernel before this one
+    mid_body<ACT, DU, GPT, SMEM_STATE ? STATE_SMEM : STATE_DU>(p, cluster, u_s, h, false);
 }
 
 // ---------------------------------------------------------------------------
