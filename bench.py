@@ -34,6 +34,14 @@ UNIT = "samples/s"
 NCU_TRAFFIC_BYTES = {"t5_base": {"down_projection": 80058880, "dw_down": 83782912}}
 
 
+def ncu_traffic(spec, kernel_path, kernel):
+    """DRAM bytes per launch from the committed ncu capture; None for kernels it does not cover
+    (the counters were taken on the separate down-projection kernel, not the one-kernel forward)."""
+    if kernel == "down_projection" and kernel_path != "tensor":
+        return None
+    return (NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]) or {}).get(kernel)
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -262,6 +270,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--force-simt", action="store_true", help="use the plain fp32-FMA kernels")
+    ap.add_argument("--one-kernel-forward", action="store_true",
+                    help="tensor-core path with the down-projections and the head phase in one kernel")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "dp"],
                     help="N > 1: independent replicas (default) or data parallel with a per-step all-reduce of "
                          "the adapter gradients (paper Section V-B)")
@@ -312,6 +322,8 @@ def main():
     ctx = pac.PacContext(local, stream.cuda_stream)
     if args.force_simt:
         ctx.set_option(binding.PAC_OPT_KERNEL_PATH, 1)
+    elif args.one_kernel_forward:
+        ctx.set_option(binding.PAC_OPT_KERNEL_PATH, 3)
     ctx.cache_register(cache, labels)
     ctx.adapter_init(r=spec.r, n_out=spec.n_out, max_batch=spec.B,
                      head=pac.PAC_HEAD_FROZEN_LM if spec.head == "lm" else pac.PAC_HEAD_MEANPOOL_CLS, lm_head=lm)
@@ -398,7 +410,7 @@ def main():
         a = kern[dominant]["gbs"]
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "traffic": (NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]) or {}).get(dominant), "algorithmic_bytes_per_launch": pass_bytes,
+                    "traffic": ncu_traffic(spec, ctx.kernel_path(), dominant), "algorithmic_bytes_per_launch": pass_bytes,
                     "kernels": kern}
     step_s = ms * 1e-3 / K
     stream_gbs = 2 * pass_bytes / step_s / 1e9

@@ -71,8 +71,14 @@ typedef struct { float lr, beta1, beta2, eps, weight_decay; } pac_adamw;
 
 /* Options for pac_set_option. */
 typedef enum {
-    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic (tensor-core path when the shape allows),
-                                 1 = force the plain fp32-FMA kernels; set before adapter_init */
+    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic (tensor-core path when the shape allows; currently the
+                                     same kernels as 2),
+                                 1 = force the plain fp32-FMA kernels,
+                                 2 = tensor-core path with the down-projections and the classifier-head
+                                     kernel as separate launches,
+                                 3 = tensor-core path with both in ONE launch per step where the shape
+                                     allows (bf16 cache, classifier head, S <= 128, r <= 64), else as 2;
+                                 set before adapter_init */
     PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events */
 } pac_option;
 
@@ -154,6 +160,8 @@ pac_status pac_set_option(pac_ctx* ctx, int option, int value);
  *   [1] merge/activation chain, head, loss and the reverse chain
  *   [2] dW_down = h_l^T du_l over all layers (second pass over the cache)
  *   [3] gradient finalisation (+ AdamW when fused into the step)
+ * When the forward half runs as one kernel (pac_kernel_path() == "tensor+fused_forward") that
+ * kernel is counted in group [0] and group [1] stays empty.
  * This call waits for the stream, then stores the summed milliseconds and the number of
  * bracketed launches since the last call in out_ms[4] and out_count[4] (host arrays).
  * At most 4096 brackets per group are kept between two calls. */
@@ -164,7 +172,9 @@ pac_status pac_launch_count(pac_ctx* ctx, long long* n);
  * ran out, ids clamped by pac_train_epoch_dev). */
 pac_status pac_sync(pac_ctx* ctx);
 const char* pac_last_error(const pac_ctx* ctx);
-/* "tensor" or "simt": which kernels the next train step will use (valid after adapter_init). */
+/* Which kernels the next train step will use (valid after adapter_init): "simt", "tensor", or
+ * "tensor+fused_forward" when the down-projections (Section IV-A) and the whole classifier-head
+ * phase run as one launch per step (bf16 cache, S <= 128, r <= 64). */
 const char* pac_kernel_path(const pac_ctx* ctx);
 
 /* Block-wise absmax INT8 quantisation, Section IV-D, Eq. 1 (the paper applies it to the frozen

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libpac_b200.so")
 SOURCES = [os.path.join(HERE, "csrc", "pac_api.cu")]
-HEADERS = [os.path.join(HERE, "csrc", f) for f in ("pac_common.cuh", "pac_simt.cuh", "pac_tensor.cuh", "pac_mid.cuh", "pac_gemm.cuh", "pac_quant.cuh")] + \
+HEADERS = [os.path.join(HERE, "csrc", f) for f in ("pac_common.cuh", "pac_simt.cuh", "pac_tensor.cuh", "pac_mid.cuh", "pac_fused_fwd.cuh", "pac_gemm.cuh", "pac_quant.cuh")] + \
           [os.path.join(ROOT, "include", "pac.h")]
 
 

@@ -10,6 +10,7 @@
 #include "pac_simt.cuh"
 #include "pac_tensor.cuh"
 #include "pac_mid.cuh"
+#include "pac_fused_fwd.cuh"
 #include "pac_gemm.cuh"
 #include "pac_quant.cuh"
 
@@ -89,6 +90,8 @@ struct pac_ctx {
     long long launches = 0;
     TensorPlan tplan{};
     MidPlan mplan{};               // fused classifier-head kernel (when the shape allows)
+    FusedFwdPlan fplan{};          // down-projections + classifier-head kernel in one launch (short sequences)
+    int one_kernel_forward = 0;    // 1: down-projections and head phase as one launch when the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
     bool lm_tensor = false;
     std::string err;
@@ -360,6 +363,8 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
 }
 
 bool use_fused_cls(const pac_ctx* c) { return c->cfg.head == PAC_HEAD_MEANPOOL_CLS && c->mplan.ok; }
+bool use_fused_fwd(const pac_ctx* c) { return use_fused_cls(c) && use_tensor(c) && c->fplan.ok; }
+int cls_cluster_size(const pac_ctx* c) { return use_fused_fwd(c) ? c->fplan.mp.G : c->mplan.G; }
 
 pac_status down_projection(pac_ctx* c, const int* d_ids, int B) {
     pac_status st;
@@ -390,26 +395,61 @@ pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     return PAC_OK;
 }
 
-pac_status mid_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+MidParams mid_params(pac_ctx* c, const MidPlan& mp, const int* d_ids, int B, bool train, float* d_logits_out) {
     const Dims& dm = c->dm;
     Scratch& sc = c->sc;
     MidParams p{};
     p.ids = d_ids; p.N = dm.N; p.labels = c->labels;
     p.L = dm.L; p.S = dm.S; p.d = dm.d; p.r = dm.r; p.C = dm.C; p.B = B;
-    p.G = c->mplan.G; p.Sg = c->mplan.Sg; p.dg = c->mplan.dg; p.train = train ? 1 : 0;
-    p.scratch = c->mplan.scratch; p.wup_smem = c->mplan.wup_smem;
+    p.G = mp.G; p.Sg = mp.Sg; p.dg = mp.dg; p.train = train ? 1 : 0;
+    p.scratch = mp.scratch; p.wup_smem = mp.wup_smem;
     p.u = sc.u; p.lstride = (long long)c->max_rows * dm.r;
     p.lam = c->params + c->lay.lam; p.W_up = c->params + c->lay.w_up;
     p.W_head = c->params + c->lay.w_head; p.b_head = c->params + c->lay.b_head; p.hbar = sc.hbar;
-    const bool tens = use_tensor(c);
-    p.du = tens ? (void*)sc.du16 : (void*)sc.du;
+    p.du = use_tensor(c) ? (void*)sc.du16 : (void*)sc.du;
     p.pooled_a = sc.pooled_a; p.pooled_y = sc.pooled_y; p.gvec = sc.gvec; p.dlogits = sc.dlogits;
     p.loss_b = sc.loss_b; p.lam_part = sc.lam_part; p.logits_out = train ? sc.logits : d_logits_out;
     p.status = c->status;
-    cudaError_t e = mid_launch(c->mplan, p, c->cfg.act, tens, c->stream);
+    return p;
+}
+
+pac_status mid_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    const MidParams p = mid_params(c, c->mplan, d_ids, B, train, d_logits_out);
+    cudaError_t e = mid_launch(c->mplan, p, c->cfg.act, use_tensor(c), c->stream);
     c->launches++;
     if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "fused head kernel launch failed: %s", cudaGetErrorString(e));
     return PAC_OK;
+}
+
+// Down-projections, chain, head, loss and reverse chain of a batch in one cluster launch.
+pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    const FusedFwdPlan& pl = c->fplan;
+    FusedFwdParams fp{};
+    fp.mid = mid_params(c, pl.mp, d_ids, B, train, d_logits_out);
+    fp.mid.u = nullptr;
+    fp.mid.layers_per_cta = pl.layers_per_cta;
+    fp.mid.u_swz = pl.u_swz;
+    fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset;
+    cudaError_t e = fused_fwd_launch(pl, c->tplan.map_cache_fwd, c->tplan.map_w, fp, c->cfg.act, c->stream);
+    c->launches++;
+    if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "fused forward kernel launch failed: %s", cudaGetErrorString(e));
+    return PAC_OK;
+}
+
+// Forward half of a classifier-head step (everything up to du and the per-sample head vectors).
+pac_status cls_forward_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    pac_status st;
+    if (use_fused_fwd(c)) {
+        time_mark(c, 0, false);
+        st = fused_fwd_enqueue(c, d_ids, B, train, d_logits_out);
+        time_mark(c, 0, true);
+        return st;
+    }
+    if ((st = down_projection(c, d_ids, B)) != PAC_OK) return st;
+    time_mark(c, 1, false);
+    st = mid_enqueue(c, d_ids, B, train, d_logits_out);
+    time_mark(c, 1, true);
+    return st;
 }
 
 void bias_corrections(const pac_adamw* hp, long long step, float* bc1, float* bc2) {
@@ -425,7 +465,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
     f.dw_part = sc.dw_part;
     f.splits = use_tensor(c) ? tensor_splits(c->tplan, B) : 1;
     f.dw_elems = (long long)dm.L * dm.d * dm.r;
-    f.lam_part = sc.lam_part; f.lam_blocks = B * c->mplan.G;
+    f.lam_part = sc.lam_part; f.lam_blocks = B * cls_cluster_size(c);
     f.pooled_a = sc.pooled_a; f.gvec = sc.gvec; f.pooled_y = sc.pooled_y; f.dlogits = sc.dlogits; f.loss_b = sc.loss_b;
     f.grads = c->grads; f.loss_out = d_loss;
     f.adam = hp ? 1 : 0;
@@ -450,10 +490,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
 pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, const pac_adamw* hp) {
     pac_status st;
     if (use_fused_cls(c)) {
-        if ((st = down_projection(c, d_ids, B)) != PAC_OK) return st;
-        time_mark(c, 1, false);
-        if ((st = mid_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
-        time_mark(c, 1, true);
+        if ((st = cls_forward_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
         if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
         time_mark(c, 3, false);
         st = finalize_enqueue(c, B, d_loss, hp);
@@ -603,6 +640,14 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     c->chain_blocks_max = (int)cdiv(Mr, 256);
     c->mplan = cls ? mid_plan(dm) : MidPlan{};
     if (c->mplan.ok && cfg->max_batch * c->mplan.G > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * c->mplan.G;
+    FusedFwdPlan fwd_plan{};
+    if (c->mplan.ok && c->dtype == PAC_BF16 && tensor_shape_supported(dm) && !c->force_simt && c->one_kernel_forward) {
+        int max_smem = 0;
+        CU_OK(c, cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device));
+        fwd_plan = fused_fwd_plan(dm, max_smem);
+        if (fwd_plan.ok && cfg->max_batch * fwd_plan.mp.G > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * fwd_plan.mp.G;
+    }
+    c->fplan = FusedFwdPlan{};
     Scratch& s = c->sc;
     pac_status st = PAC_OK;
     auto A = [&](pac_status x) { if (st == PAC_OK) st = x; };
@@ -655,6 +700,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             if (ts == PAC_OK) {
                 A(dmalloc(c, &s.dw_part, part_floats));
                 c->tensor_ok = (st == PAC_OK);
+                if (c->tensor_ok) c->fplan = fwd_plan;
             } else if (ts != PAC_ERR_UNSUPPORTED) {
                 st = fail(c, ts, "tensor path set-up failed: %s", tensor_last_error());
             }
@@ -712,10 +758,7 @@ pac_status pac_eval_logits(pac_ctx* c, const int* sample_ids, int B, float* dev_
     if (!dev_out) return fail(c, PAC_ERR_INVALID_ARG, "pac_eval_logits: dev_out is NULL");
     pac_status st = stage_ids(c, sample_ids, B, "pac_eval_logits");
     if (st != PAC_OK) return st;
-    if (use_fused_cls(c)) {
-        if ((st = down_projection(c, c->sc.ids, B)) != PAC_OK) return st;
-        return mid_enqueue(c, c->sc.ids, B, false, dev_out);
-    }
+    if (use_fused_cls(c)) return cls_forward_enqueue(c, c->sc.ids, B, false, dev_out);
     return forward(c, c->sc.ids, B, false, dev_out);
 }
 
@@ -856,9 +899,10 @@ pac_status pac_params_changed(pac_ctx* c) {
 pac_status pac_set_option(pac_ctx* c, int option, int value) {
     NEED_CTX(c);
     if (option == PAC_OPT_KERNEL_PATH) {
-        if (value != 0 && value != 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0 or 1");
+        if (value < 0 || value > 3) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0, 1, 2 or 3");
         if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_set_option: set the kernel path before pac_adapter_init");
-        c->force_simt = value;
+        c->force_simt = value == 1;
+        c->one_kernel_forward = value == 3;
         return PAC_OK;
     }
     if (option == PAC_OPT_KERNEL_TIMING) {
@@ -909,7 +953,10 @@ pac_status pac_sync(pac_ctx* c) {
 
 const char* pac_last_error(const pac_ctx* c) { return c ? c->err.c_str() : "null context"; }
 
-const char* pac_kernel_path(const pac_ctx* c) { return (c && c->inited && use_tensor(c)) ? "tensor" : "simt"; }
+const char* pac_kernel_path(const pac_ctx* c) {
+    if (!c || !c->inited || !use_tensor(c)) return "simt";
+    return use_fused_fwd(c) ? "tensor+fused_forward" : "tensor";
+}
 
 }  // extern "C"
 

@@ -1,0 +1,221 @@
+// Forward-fused sample kernel for short sequences (S <= 128, r <= 64, classifier head):
+// one thread-block cluster per batch sample does, in ONE launch,
+//   1. the down-projections u_l = h_l W_down^l of the sample's 128-token tile, the L layers
+//      split over the cluster's CTAs (each CTA: TMA-fed tcgen05 MMAs into one TMEM accumulator
+//      per layer, weights as bf16 hi|lo side by side along N),
+//   2. the hand-over of u through distributed shared memory - the u tiles never go to global
+//      memory: every CTA parks its layers' tiles in its own shared memory and the chain reads and
+//      updates them in place across the cluster,
+//   3. everything the stand-alone fused kernel does afterwards (mid_body): merge/activation
+//      chain, pooling, head, loss, head gradients, reverse chain -> du_l and dlambda partials.
+// During the GEMM phase the otherwise idle warps prefetch the head operands.
+#pragma once
+#include "pac_mid.cuh"
+#include "pac_tensor.cuh"
+
+namespace pac {
+
+struct FusedFwdParams {
+    MidParams mid;             // G, Sg, dg, layers_per_cta, head operands, outputs (u / lstride unused)
+    int k_chunks;              // ceil(d / 64)
+    int stages;                // pipeline depth of the GEMM phase
+    size_t mid_offset;         // byte offset of the head vectors behind the stage / u-tile region
+};
+
+constexpr int FUSED_N = 128;   // MMA N: 64 hi columns | 64 lo columns
+
+template <int ACT>
+__global__ void __launch_bounds__(512, 1)
+fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_constant__ CUtensorMap map_w, FusedFwdParams fp) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    cg::cluster_group cluster = cg::this_cluster();
+    const MidParams& p = fp.mid;
+    const int q = (int)cluster.block_rank();
+    const int b = blockIdx.x / p.G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const uint32_t a_bytes = FWD_ROWS * KC * 2, b_bytes = 2 * KC * 128, stage_bytes = a_bytes + b_bytes;
+    float* u_loc = reinterpret_cast<float*>(smem);                       // [layers_per_cta][128][r] after the GEMM phase
+    const MidShared h = mid_carve(reinterpret_cast<float*>(smem + fp.mid_offset), p);
+    __shared__ __align__(8) unsigned long long bars[2 * 16 + 1];
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ int abort_sh;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]), accf = smem_u32(&bars[32]);
+    const int l_begin = q * p.layers_per_cta, l_end = min(p.L, l_begin + p.layers_per_cta);
+    const int n_layers = max(0, l_end - l_begin);
+
+    if (threadIdx.x == 0) {
+        abort_sh = 0;
+        for (int s = 0; s < fp.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(accf, 1);
+        fence_mbar_init();
+        tma_prefetch_desc(&map_cache);
+        tma_prefetch_desc(&map_w);
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), 512u); tmem_relinquish(); }
+    pdl_trigger();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sh;
+    volatile int* abort_flag = &abort_sh;
+    pdl_wait();                 // weights, parameters and ids of this step are final from here on
+    const long long id = safe_id(p.ids, b, p.N, nullptr);        // mid_body reports clamped ids
+
+    // ---- phase 1: the GEMMs of this CTA's layers; idle warps fetch the head operands ----
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            const uint64_t pol = l2_policy_evict_first();
+            for (int l = l_begin; l < l_end && !*abort_flag; ++l) {
+                for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
+                    const int s = it % fp.stages;
+                    const uint32_t ph = (it / fp.stages) & 1;
+                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
+                    const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+                    mbar_expect_tx(full0 + 8 * s, stage_bytes);
+                    tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, 0, l, (int)id, pol);
+                    tma_load_4d(dst + a_bytes, &map_w, full0 + 8 * s, 0, kc * KC, 0, l);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(FWD_ROWS, FUSED_N, 0, 1);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int l = l_begin; l < l_end && ok && !*abort_flag; ++l) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)((l - l_begin) * FUSED_N);
+                for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
+                    const int s = it % fp.stages;
+                    const uint32_t ph = (it / fp.stages) & 1;
+                    if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
+                    const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024), bw0 = smem_desc_sw128(b0, KC * 128, 1024);
+#pragma unroll
+                    for (int k = 0; k < KC / 16; ++k)
+                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bw0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
+                    umma_commit(empty0 + 8 * s);
+                }
+            }
+            if (ok && n_layers > 0) umma_commit(accf);          // every accumulator of this CTA is complete
+        }
+    } else {
+        mid_prefetch_head(p, h, q, id, (int)threadIdx.x - 64, (int)blockDim.x - 64);
+    }
+
+    // ---- phase 2: accumulators -> this CTA's shared memory (hi + lo), as [layer][token][r] ----
+    bool have = false;
+    if (n_layers > 0) have = mbar_wait_warp(accf, 0, abort_flag, p.status);     // also: every load has been consumed
+    if (have) tc_fence_after();
+    {
+        const int quad = warp & 3, part = warp >> 2;              // TMEM lane quadrant, 16-column share
+        const int row = quad * 32 + lane;
+        for (int c0 = part * 16; c0 < p.r; c0 += 16 * (nwarps >> 2)) {
+            for (int li = 0; li < n_layers; ++li) {
+                float v[16], w[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) { v[c] = 0.f; w[c] = 0.f; }
+                if (have) {
+                    const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(li * FUSED_N + c0);
+                    tmem_ld16(taddr, v);
+                    tmem_ld16(taddr + 64, w);
+                    tmem_ld_wait();
+                }
+                float4* dst = reinterpret_cast<float4*>(u_loc + ((size_t)li * 128 + row) * p.r);
+                const int g0 = c0 >> 2, sw = row & p.u_swz;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    dst[(g0 + c) ^ sw] = make_float4(v[4 * c] + w[4 * c], v[4 * c + 1] + w[4 * c + 1], v[4 * c + 2] + w[4 * c + 2], v[4 * c + 3] + w[4 * c + 3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    drain_after_abort(abort_flag);
+    if (warp == 1) tmem_dealloc(tmem_base, 512u);
+    cluster.sync();                                               // every CTA's u tiles are in place
+
+    // ---- phase 3: chain, head, loss, reverse chain on the cluster-resident u ----
+    mid_body<ACT, bf16, 1, STATE_CLUSTER>(p, cluster, reinterpret_cast<float4*>(u_loc), h, true);
+}
+
+// Launch geometry: smallest cluster that gives one 4-column group per thread, at most four layers
+// (4 x 128 TMEM columns) per CTA and fits shared memory.
+struct FusedFwdPlan {
+    bool ok = false;
+    MidPlan mp;
+    int layers_per_cta = 0, stages = 0, k_chunks = 0, u_swz = 0;
+    size_t mid_offset = 0, smem = 0;
+};
+
+inline FusedFwdPlan fused_fwd_plan(const Dims& dm, int max_smem) {
+    FusedFwdPlan fp;
+    if (dm.S > FWD_ROWS || dm.r > 64 || dm.r % 16 != 0 || dm.d % 8 != 0 || dm.d < 64 || dm.C > MID_MAX_C || dm.L > MID_MAX_L) return fp;
+    const size_t stage = FWD_ROWS * KC * 2 + 2 * KC * 128;
+    for (int G = 1; G <= 8; G *= 2) {
+        const int Sg = (dm.S + G - 1) / G, dg = (dm.d + G - 1) / G, lpc = (dm.L + G - 1) / G;
+        const long long need = (long long)Sg * (dm.r / 4);
+        if (need > 512 || lpc > 4) continue;
+        int th = (int)((need + 31) / 32 * 32);
+        if (th < 256) th = 256;                                  // producer, MMA, four drain quadrants and prefetch warps
+        int scratch;
+        size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
+        const size_t wup = (size_t)dm.r * dg;
+        const size_t u_tiles = (size_t)lpc * 128 * dm.r * 4;
+        const size_t budget = (size_t)max_smem - 2048;
+        // stage / u-tile region first, head vectors (with the W_up slice when it fits) behind it
+        for (int with_wup = 1; with_wup >= 0; --with_wup) {
+            const size_t mid_bytes = (floats + (with_wup ? wup : 0)) * sizeof(float);
+            if (mid_bytes + u_tiles > budget) continue;
+            int st = (int)((budget - mid_bytes) / stage);
+            if (st > 16) st = 16;
+            if (st < 2 || (size_t)st * stage < u_tiles) continue;
+            fp.mp.ok = true; fp.mp.G = G; fp.mp.Sg = Sg; fp.mp.dg = dg; fp.mp.threads = th; fp.mp.scratch = scratch;
+            fp.mp.gpt = 1; fp.mp.smem_state = 0; fp.mp.wup_smem = with_wup;
+            fp.layers_per_cta = lpc; fp.stages = st; fp.k_chunks = (dm.d + KC - 1) / KC;
+            const int groups = dm.r / 4;
+            fp.u_swz = (groups & (groups - 1)) == 0 ? groups - 1 : 3;      // r is a multiple of 16
+            fp.mid_offset = (size_t)st * stage;
+            fp.smem = fp.mid_offset + mid_bytes + 1024;
+            fp.ok = true;
+            return fp;
+        }
+    }
+    return fp;
+}
+
+template <int ACT>
+inline cudaError_t fused_fwd_launch_act(const FusedFwdPlan& pl, const CUtensorMap& map_cache, const CUtensorMap& map_w,
+                                        const FusedFwdParams& fp, cudaStream_t stream) {
+    static size_t opted_in = 0;                      // dynamic shared memory the kernel has been allowed so far
+    if (pl.smem > opted_in) {
+        cudaError_t e = cudaFuncSetAttribute(fwd_cluster_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+        if (e != cudaSuccess) return e;
+        opted_in = pl.smem;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(fp.mid.B * pl.mp.G), 1, 1);
+    cfg.blockDim = dim3((unsigned)pl.mp.threads, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)pl.mp.G;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, fwd_cluster_kernel<ACT>, map_cache, map_w, fp);
+}
+
+inline cudaError_t fused_fwd_launch(const FusedFwdPlan& pl, const CUtensorMap& map_cache, const CUtensorMap& map_w,
+                                    const FusedFwdParams& fp, int act, cudaStream_t stream) {
+    return act == PAC_ACT_RELU ? fused_fwd_launch_act<PAC_ACT_RELU>(pl, map_cache, map_w, fp, stream)
+                               : fused_fwd_launch_act<PAC_ACT_IDENTITY>(pl, map_cache, map_w, fp, stream);
+}
+
+}  // namespace pac

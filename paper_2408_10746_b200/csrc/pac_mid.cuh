@@ -31,6 +31,7 @@ struct MidParams {
     int scratch;                // floats of block-local reduction scratch
     int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
     int layers_per_cta;         // STATE_CLUSTER: layers whose u tiles each CTA of the cluster holds
+    int u_swz;                  // STATE_CLUSTER: a token row's 4-column groups are stored at (group ^ (row & u_swz))
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
     void* du;                   // [L][max_rows][r] bf16 or fp32
@@ -64,7 +65,8 @@ enum {
     STATE_DU = 1,        // u read from global memory; u_l - a_{l-1} parked, in du's type, in the du slot
                          // that the reverse pass overwrites with du_l once it has consumed it
     STATE_CLUSTER = 2    // u tiles produced by the cluster's own GEMMs: layer l sits in the shared memory
-                         // of CTA l / layers_per_cta as [layer][128 tokens][r] fp32 and is updated in place
+                         // of CTA l / layers_per_cta as [layer][128 tokens][r] fp32 (4-column groups of a row
+                         // permuted by u_swz against bank conflicts of the producer) and is updated in place
                          // through distributed shared memory (every element has exactly one owner thread)
 };
 
@@ -138,7 +140,8 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     auto cluster_slot = [&](int l, int g) -> float4* {      // STATE_CLUSTER: the element's home in the cluster
         const int owner = l / p.layers_per_cta, li = l - owner * p.layers_per_cta;
         float* tile = cluster.map_shared_rank(reinterpret_cast<float*>(u_s), owner);
-        return reinterpret_cast<float4*>(tile + ((size_t)li * 128 + (q * p.Sg + s_local[g])) * r + j4[g]);
+        const int row = q * p.Sg + s_local[g];
+        return reinterpret_cast<float4*>(tile + ((size_t)li * 128 + row) * r + ((((j4[g] >> 2) ^ (row & p.u_swz))) << 2));
     };
     auto load_u = [&](int l, int g) -> float4 {
         if constexpr (STATE == STATE_SMEM) return u_s[((size_t)l * GPT + g) * nt + t];

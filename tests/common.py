@@ -34,12 +34,14 @@ class Case:
             return po.gather(self.cache_np, ids)
         return pi.cache_samples(self.spec, self.seed, list(ids), "cpu").float().numpy()
 
-    def context(self, max_batch=None, act=0, force_simt=False, seed=1):
+    def context(self, max_batch=None, act=0, force_simt=False, seed=1, kernel_path=0):
         import paper_2408_10746_b200 as pac
         s = self.spec
         ctx = pac.PacContext(0)
         if force_simt:
             ctx.set_option(0, 1)
+        elif kernel_path:
+            ctx.set_option(0, kernel_path)
         ctx.cache_register(self.cache, self.labels)
         ctx.adapter_init(r=s.r, n_out=s.n_out, max_batch=max_batch or s.B, act=act,
                          head=pac.PAC_HEAD_FROZEN_LM if s.head == "lm" else pac.PAC_HEAD_MEANPOOL_CLS,

@@ -120,11 +120,11 @@ def test_zero_up_projection_is_head_only(tiny):
 
 
 # ------------------------------------------------------------------ trajectories
-def run_trajectory(case, steps, act=0, force_simt=False, hp=None):
+def run_trajectory(case, steps, act=0, force_simt=False, hp=None, kernel_path=0):
     import paper_2408_10746_b200 as pac
     spec = case.spec
     hp = hp or po.AdamW()
-    ctx = case.context(act=act, force_simt=force_simt)
+    ctx = case.context(act=act, force_simt=force_simt, kernel_path=kernel_path)
     flat0 = ctx.get_params()
     perm = pi.epoch_permutation(spec.N, 2)
     batches = [perm[i * spec.B:(i + 1) * spec.B].tolist() for i in range(steps)]
@@ -254,14 +254,19 @@ TC_SPECS = [
     # per-sample chain state too large for shared memory: 2 and 4 column groups per thread, state parked in du
     (TC_BASE.scaled(name="tc_long_S", S=300, d=128, r=64, L=3, B=2, N=6), 2, 0),
     (TC_BASE.scaled(name="tc_long_S_wide_r", S=500, d=128, r=128, L=2, B=2, N=4), 2, 1),
+    # short sequence, r/4 not a power of two, layers split unevenly over the sample's cluster
+    (TC_BASE.scaled(name="tc_r48_short", S=100, d=200, r=48, L=5, B=3), 3, 0),
 ]
+# shapes that can take the single forward kernel (S <= 128, r <= 64): also run with it switched on
+TC_ONE_KERNEL_FORWARD = [s for s in TC_SPECS if s[0].S <= 128 and s[0].r <= 64]
 
 
-def tc_check(spec, max_batch, act, ids=None, loss_tol=2e-2, chain_tol=1e-2, head_tol=2e-3, case=None):
+def tc_check(spec, max_batch, act, ids=None, loss_tol=2e-2, chain_tol=1e-2, head_tol=2e-3, case=None, kernel_path=0):
     case = case or Case(spec)
     ids = ids or [spec.N - 1, 0, 5, 5][:spec.B]
-    ctx = case.context(max_batch=max_batch, act=act)
-    assert ctx.kernel_path() == "tensor"
+    ctx = case.context(max_batch=max_batch, act=act, kernel_path=kernel_path)
+    one_kernel = spec.head == "cls" and spec.S <= 128 and spec.r <= 64 and kernel_path == 3
+    assert ctx.kernel_path() == ("tensor+fused_forward" if one_kernel else "tensor")
     flat = pi.random_params(spec, 3)
     ctx.set_params(flat)
     loss = ctx.train_step(ids)
@@ -285,6 +290,33 @@ def test_tensor_path_loss_and_gradients(spec, max_batch, act):
     tc_check(spec, max_batch, act)
 
 
+@pytest.mark.parametrize("spec,max_batch,act", TC_ONE_KERNEL_FORWARD, ids=[s[0].name for s in TC_ONE_KERNEL_FORWARD])
+def test_tensor_path_one_kernel_forward(spec, max_batch, act):
+    """The same shapes with the down-projections and the head phase in one launch."""
+    tc_check(spec, max_batch, act, kernel_path=3)
+
+
+@pytest.mark.parametrize("spec,max_batch,act", TC_ONE_KERNEL_FORWARD, ids=[s[0].name for s in TC_ONE_KERNEL_FORWARD])
+def test_one_kernel_forward_matches_separate_kernels(spec, max_batch, act):
+    """Both forward variants do the same arithmetic per element; only the order of a few cross-block
+    sums differs (another cluster size), so loss, logits and gradients agree to fp32 rounding."""
+    case = Case(spec)
+    flat = pi.random_params(spec, 5)
+    ids = [spec.N - 1, 0, 5, 5][:spec.B]
+    res = []
+    for path in (3, 2):
+        ctx = case.context(max_batch=max_batch, act=act, kernel_path=path)
+        ctx.set_params(flat)
+        out = torch.zeros((len(ids), spec.n_out), dtype=torch.float32, device="cuda")
+        ctx.eval_logits(ids, out)
+        loss = ctx.train_step(ids)
+        ctx.sync()
+        res.append((loss, out.cpu().numpy(), ctx.get_grads()))
+    assert abs(res[0][0] - res[1][0]) <= 1e-5 * abs(res[1][0])
+    assert rel_l2(res[0][1], res[1][1]) < 1e-5
+    assert rel_l2(res[0][2], res[1][2]) < 1e-5
+
+
 def test_tensor_path_eval_and_determinism():
     case = Case(TC_BASE)
     flat = pi.random_params(TC_BASE, 4)
@@ -302,13 +334,14 @@ def test_tensor_path_eval_and_determinism():
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(grads[0], grads[1])    # fixed summation orders
 
 
-def test_tensor_path_ten_steps_t5_base_shape():
+@pytest.mark.parametrize("kernel_path", [0, 3], ids=["auto", "one_kernel_forward"])
+def test_tensor_path_ten_steps_t5_base_shape(kernel_path):
     """T5-Base layer shape (L=12, S=128, d=768, r=64) on a short cache: 10 AdamW steps from the
     seeded initial state; loss within 2e-2, parameter vector within 1e-2 relative L2."""
     spec = pi.CONFIGS["t5_base"].scaled(N=96, B=8, name="t5_base_short")
     case = Case(spec, materialize_cpu=False)
-    ctx, losses, ref_losses, p, ref_p, p0 = run_trajectory(case, 10)
-    assert ctx.kernel_path() == "tensor"
+    ctx, losses, ref_losses, p, ref_p, p0 = run_trajectory(case, 10, kernel_path=kernel_path)
+    assert ctx.kernel_path() == ("tensor+fused_forward" if kernel_path == 3 else "tensor")
     assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses))
     assert rel_l2(p, ref_p) < 1e-2
     assert rel_l2(p - p0, ref_p - p0) < 0.1          # the update itself is reproduced, not only the initial values
