@@ -1,14 +1,14 @@
-// Forward-fused sample kernel for short sequences (S <= 128, r <= 64, classifier head):
-// one thread-block cluster per batch sample does, in ONE launch,
-//   1. the down-projections u_l = h_l W_down^l of the sample's 128-token tile, the L layers
-//      split over the cluster's CTAs (each CTA: TMA-fed tcgen05 MMAs into one TMEM accumulator
-//      per layer, weights as bf16 hi|lo side by side along N),
-//   2. the hand-over of u through distributed shared memory - the u tiles never go to global
-//      memory: every CTA parks its layers' tiles in its own shared memory and the chain reads and
-//      updates them in place across the cluster,
-//   3. everything the stand-alone fused kernel does afterwards (mid_body): merge/activation
-//      chain, pooling, head, loss, head gradients, reverse chain -> du_l and dlambda partials.
-// During the GEMM phase the otherwise idle warps prefetch the head operands.
+// One-launch forward for short sequences (S <= 128, r <= 64, classifier head): one thread-block
+// cluster per batch sample does
+//   1. the down-projections u_l = h_l W_down^l (Section IV-A) of the sample's 128-token tile, the
+//      L layers split over the cluster's CTAs (each CTA: TMA-fed tcgen05 MMAs into one TMEM
+//      accumulator per layer, weights as bf16 hi|lo side by side along N); meanwhile the other
+//      warps fetch the head operands and form the head's product matrix (mid_head_products),
+//   2. the hand-over of u through distributed shared memory - u never goes to global memory: the
+//      chain is split by tokens, so every CTA writes each accumulator row straight into the shared
+//      memory of the CTA that owns the token,
+//   3. everything the stand-alone fused kernel does afterwards (mid_body) on the now local tiles:
+//      merge/activation chain, pooling, head, loss, reverse chain -> du_l and dlambda partials.
 #pragma once
 #include "pac_mid.cuh"
 #include "pac_tensor.cuh"
@@ -35,17 +35,18 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     const int b = blockIdx.x / p.G;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const uint32_t a_bytes = FWD_ROWS * KC * 2, b_bytes = 2 * KC * 128, stage_bytes = a_bytes + b_bytes;
-    float* u_loc = reinterpret_cast<float*>(smem);                       // [layers_per_cta][128][r] after the GEMM phase
+    float* u_loc = reinterpret_cast<float*>(smem);                       // [L][Sg][r]: this CTA's tokens, all layers, after the GEMM phase
     const MidShared h = mid_carve(reinterpret_cast<float*>(smem + fp.mid_offset), p);
     __shared__ __align__(8) unsigned long long bars[2 * 16 + 1];
     __shared__ uint32_t tmem_base_sh;
-    __shared__ int abort_sh;
+    __shared__ int abort_sh, have_sh;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]), accf = smem_u32(&bars[32]);
     const int l_begin = q * p.layers_per_cta, l_end = min(p.L, l_begin + p.layers_per_cta);
     const int n_layers = max(0, l_end - l_begin);
 
     if (threadIdx.x == 0) {
         abort_sh = 0;
+        have_sh = 0;
         for (int s = 0; s < fp.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(accf, 1);
         fence_mbar_init();
@@ -62,56 +63,74 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     pdl_wait();                 // weights, parameters and ids of this step are final from here on
     const long long id = safe_id(p.ids, b, p.N, nullptr);        // mid_body reports clamped ids
 
-    // ---- phase 1: the GEMMs of this CTA's layers; idle warps fetch the head operands ----
+    // ---- phase 1: the GEMMs of this CTA's layers; the other warps fetch the head operands.
+    // Both pipeline loops are run by a whole converged warp, one elected lane issues. ----
     if (warp == 0) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            const uint64_t pol = l2_policy_evict_first();
-            for (int l = l_begin; l < l_end && !*abort_flag; ++l) {
-                for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
-                    const int s = it % fp.stages;
-                    const uint32_t ph = (it / fp.stages) & 1;
-                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-                    const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+        uint32_t it = 0;
+        const uint64_t pol = l2_policy_evict_first();
+        bool ok = true;
+        for (int l = l_begin; l < l_end && ok; ++l) {
+            for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
+                const int s = it % fp.stages;
+                const uint32_t ph = (it / fp.stages) & 1;
+                if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+                if (elect_one()) {
                     mbar_expect_tx(full0 + 8 * s, stage_bytes);
                     tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, 0, l, (int)id, pol);
                     tma_load_4d(dst + a_bytes, &map_w, full0 + 8 * s, 0, kc * KC, 0, l);
                 }
+                __syncwarp();
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(FWD_ROWS, FUSED_N, 0, 1);
-            uint32_t it = 0;
-            bool ok = true;
-            for (int l = l_begin; l < l_end && ok && !*abort_flag; ++l) {
-                const uint32_t d_tmem = tmem_base + (uint32_t)((l - l_begin) * FUSED_N);
-                for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
-                    const int s = it % fp.stages;
-                    const uint32_t ph = (it / fp.stages) & 1;
-                    if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
-                    const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024), bw0 = smem_desc_sw128(b0, KC * 128, 1024);
+        const uint32_t idesc = instr_desc_bf16(FWD_ROWS, FUSED_N, 0, 1);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int l = l_begin; l < l_end && ok; ++l) {
+            const uint32_t d_tmem = tmem_base + (uint32_t)((l - l_begin) * FUSED_N);
+            for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
+                const int s = it % fp.stages;
+                const uint32_t ph = (it / fp.stages) & 1;
+                if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
+                const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024), bw0 = smem_desc_sw128(b0, KC * 128, 1024);
+                if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < KC / 16; ++k)
                         umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bw0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
                     umma_commit(empty0 + 8 * s);
                 }
+                __syncwarp();
             }
-            if (ok && n_layers > 0) umma_commit(accf);          // every accumulator of this CTA is complete
+        }
+        if (ok && n_layers > 0) {
+            if (elect_one()) umma_commit(accf);                   // every accumulator of this CTA is complete ...
+            __syncwarp();
+            if (mbar_wait_uniform(accf, 0, abort_flag, p.status)) have_sh = 1;    // ... and every load has been consumed
         }
     } else {
+        // head operands -> shared memory, then this CTA's slice of the head products; the barrier
+        // covers these warps only (ids 2 .. nwarps-1), the two pipeline warps never join it
         mid_prefetch_head(p, h, q, id, (int)threadIdx.x - 64, (int)blockDim.x - 64);
+        cp_async_commit();
+        cp_async_wait_group<0>();
+        asm volatile("bar.sync 1, %0;" ::"r"((int)blockDim.x - 64) : "memory");
+        mid_head_products(p, h, q, warp - 2, nwarps - 2, lane);
     }
 
-    // ---- phase 2: accumulators -> this CTA's shared memory (hi + lo), as [layer][token][r] ----
-    bool have = false;
-    if (n_layers > 0) have = mbar_wait_warp(accf, 0, abort_flag, p.status);     // also: every load has been consumed
-    if (have) tc_fence_after();
+    // ---- phase 2: accumulators (hi + lo) -> shared memory of the CTA that owns the token ----
+    // Only the MMA thread watches the accumulator barrier; everybody else sleeps at the cluster
+    // barrier (threads that poll an mbarrier slow down the pipeline's own barrier traffic).
+    cluster.sync();         // every CTA of the cluster is done with its stage buffers; head products are published
+    const bool have = have_sh != 0;
+    tc_fence_after();
     {
         const int quad = warp & 3, part = warp >> 2;              // TMEM lane quadrant, 16-column share
-        const int row = quad * 32 + lane;
+        const int row = quad * 32 + lane;                         // token
+        const int owner = row / p.Sg, s_loc = row - owner * p.Sg;
+        float* tiles = cluster.map_shared_rank(u_loc, row < p.S ? owner : q);     // [L][Sg][r] in the owner's memory
         for (int c0 = part * 16; c0 < p.r; c0 += 16 * (nwarps >> 2)) {
             for (int li = 0; li < n_layers; ++li) {
                 float v[16], w[16];
@@ -123,11 +142,13 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     tmem_ld16(taddr + 64, w);
                     tmem_ld_wait();
                 }
-                float4* dst = reinterpret_cast<float4*>(u_loc + ((size_t)li * 128 + row) * p.r);
-                const int g0 = c0 >> 2, sw = row & p.u_swz;
+                if (row < p.S) {
+                    float4* dst = reinterpret_cast<float4*>(tiles + ((size_t)(l_begin + li) * p.Sg + s_loc) * p.r);
+                    const int g0 = c0 >> 2, sw = s_loc & p.u_swz;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    dst[(g0 + c) ^ sw] = make_float4(v[4 * c] + w[4 * c], v[4 * c + 1] + w[4 * c + 1], v[4 * c + 2] + w[4 * c + 2], v[4 * c + 3] + w[4 * c + 3]);
+                    for (int c = 0; c < 4; ++c)
+                        dst[(g0 + c) ^ sw] = make_float4(v[4 * c] + w[4 * c], v[4 * c + 1] + w[4 * c + 1], v[4 * c + 2] + w[4 * c + 2], v[4 * c + 3] + w[4 * c + 3]);
+                }
             }
         }
     }
@@ -135,10 +156,10 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     __syncthreads();
     drain_after_abort(abort_flag);
     if (warp == 1) tmem_dealloc(tmem_base, 512u);
-    cluster.sync();                                               // every CTA's u tiles are in place
+    cluster.sync();                                               // every token's u rows have arrived
 
     // ---- phase 3: chain, head, loss, reverse chain on the cluster-resident u ----
-    mid_body<ACT, bf16, 1, STATE_CLUSTER>(p, cluster, reinterpret_cast<float4*>(u_loc), h, true);
+    mid_body<ACT, bf16, 1, STATE_TILES>(p, cluster, reinterpret_cast<float4*>(u_loc), h, true);
 }
 
 // Launch geometry: smallest cluster that gives one 4-column group per thread, at most four layers
@@ -163,7 +184,7 @@ inline FusedFwdPlan fused_fwd_plan(const Dims& dm, int max_smem) {
         int scratch;
         size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
         const size_t wup = (size_t)dm.r * dg;
-        const size_t u_tiles = (size_t)lpc * 128 * dm.r * 4;
+        const size_t u_tiles = (size_t)dm.L * Sg * dm.r * 4;
         const size_t budget = (size_t)max_smem - 2048;
         // stage / u-tile region first, head vectors (with the W_up slice when it fits) behind it
         for (int with_wup = 1; with_wup >= 0; --with_wup) {

@@ -56,16 +56,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
 
+    // Both pipeline loops are run by whole converged warps with one elected lane issuing, so that
+    // addresses, coordinates and descriptors stay warp-uniform values.
     if (warp == 0) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
-                const int m0 = (t % p.m_tiles) * GT_BM, n0 = (t / p.m_tiles) * GT_BN;
-                for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                    const int s = it % GT_STAGES;
-                    const uint32_t ph = (it / GT_STAGES) & 1;
-                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-                    const uint32_t dst = smem_u32(smem + (size_t)s * GT_STAGE);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+            const int m0 = (t % p.m_tiles) * GT_BM, n0 = (t / p.m_tiles) * GT_BN;
+            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+                const int s = it % GT_STAGES;
+                const uint32_t ph = (it / GT_STAGES) & 1;
+                if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                const uint32_t dst = smem_u32(smem + (size_t)s * GT_STAGE);
+                if (elect_one()) {
                     mbar_expect_tx(full0 + 8 * s, GT_STAGE);
                     tma_load_2d(dst, &map_a, full0 + 8 * s, kc * GT_BK, m0);
                     if (p.b_mn_major) {
@@ -75,37 +78,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         tma_load_2d(dst + GT_A_BYTES, &map_b, full0 + 8 * s, kc * GT_BK, n0);
                     }
                 }
+                __syncwarp();
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(GT_BM, GT_BN, 0, p.b_mn_major);
-            uint32_t it = 0, tile_n = 0;
-            for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++tile_n) {
-                const int buf = tile_n & 1;
-                const uint32_t aph = (tile_n >> 1) & 1;
-                if (!mbar_wait(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
+        const uint32_t idesc = instr_desc_bf16(GT_BM, GT_BN, 0, p.b_mn_major);
+        uint32_t it = 0, tile_n = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_n) {
+            const int buf = tile_n & 1;
+            const uint32_t aph = (tile_n >> 1) & 1;
+            if (!mbar_wait_uniform(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GT_BN);
+            bool ok = true;
+            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+                const int s = it % GT_STAGES;
+                const uint32_t ph = (it / GT_STAGES) & 1;
+                if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GT_BN);
-                bool ok = true;
-                for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                    const int s = it % GT_STAGES;
-                    const uint32_t ph = (it / GT_STAGES) & 1;
-                    if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a0 = smem_u32(smem + (size_t)s * GT_STAGE), b0 = a0 + GT_A_BYTES;
-                    const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
-                    // K-major B: 256 rows of 128 B; MN-major B: four [64 k][128 B] blocks 8192 B apart
-                    const uint64_t bd0 = p.b_mn_major ? smem_desc_sw128(b0, 8192, 1024) : smem_desc_sw128(b0, 16, 1024);
-                    const uint64_t bstep = p.b_mn_major ? 128u : 2u;     // 16 K elements further, in 16-byte units
+                const uint32_t a0 = smem_u32(smem + (size_t)s * GT_STAGE), b0 = a0 + GT_A_BYTES;
+                const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
+                // K-major B: 256 rows of 128 B; MN-major B: four [64 k][128 B] blocks 8192 B apart
+                const uint64_t bd0 = p.b_mn_major ? smem_desc_sw128(b0, 8192, 1024) : smem_desc_sw128(b0, 16, 1024);
+                const uint64_t bstep = p.b_mn_major ? 128u : 2u;     // 16 K elements further, in 16-byte units
+                if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < GT_BK / 16; ++k)
                         umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bd0 + bstep * k, idesc, (kc | k) ? 1u : 0u);
                     umma_commit(empty0 + 8 * s);
                 }
-                if (!ok) break;
-                umma_commit(accf0 + 8 * buf);
+                __syncwarp();
             }
+            if (!ok) break;
+            if (elect_one()) umma_commit(accf0 + 8 * buf);
+            __syncwarp();
         }
     } else {
         const int q = warp & 3;

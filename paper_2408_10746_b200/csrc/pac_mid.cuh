@@ -30,8 +30,8 @@ struct MidParams {
     int train;
     int scratch;                // floats of block-local reduction scratch
     int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
-    int layers_per_cta;         // STATE_CLUSTER: layers whose u tiles each CTA of the cluster holds
-    int u_swz;                  // STATE_CLUSTER: a token row's 4-column groups are stored at (group ^ (row & u_swz))
+    int layers_per_cta;         // one-kernel forward: layers whose down-projections each CTA of the cluster computes
+    int u_swz;                  // STATE_TILES: a token row's 4-column groups are stored at (group ^ (token & u_swz))
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
     void* du;                   // [L][max_rows][r] bf16 or fp32
@@ -64,30 +64,28 @@ enum {
     STATE_SMEM = 0,      // this CTA's shared memory, prefetched from the global u buffer with cp.async
     STATE_DU = 1,        // u read from global memory; u_l - a_{l-1} parked, in du's type, in the du slot
                          // that the reverse pass overwrites with du_l once it has consumed it
-    STATE_CLUSTER = 2    // u tiles produced by the cluster's own GEMMs: layer l sits in the shared memory
-                         // of CTA l / layers_per_cta as [layer][128 tokens][r] fp32 (4-column groups of a row
-                         // permuted by u_swz against bank conflicts of the producer) and is updated in place
-                         // through distributed shared memory (every element has exactly one owner thread)
+    STATE_TILES = 2      // this CTA's shared memory, filled by the cluster's own GEMMs before the call:
+                         // [L][Sg tokens][r] fp32, a token row's 4-column groups permuted by u_swz
 };
 
 // The small per-CTA vectors of the head computation, carved from one shared-memory region.
 struct MidShared {
-    float *aL, *colsum, *lpart, *dpart, *pooled, *daL, *py, *gk, *lg, *lam_s, *wh_s, *lred, *wup_s;
+    float *aL, *colsum, *prodq, *prod, *pooled, *daL, *py, *lg, *lam_s, *wh_s, *lred, *wup_s;
 };
 __device__ __forceinline__ MidShared mid_carve(float* sm, const MidParams& p) {
     MidShared h;
+    const size_t rc = (size_t)(p.r + 1) * p.C;
     h.aL = sm;                                        // [Sg][r]   a_L of this CTA's tokens
     h.colsum = h.aL + (size_t)p.Sg * p.r;             // [r]       exchanged through DSMEM
-    h.lpart = h.colsum + p.r;                         // [MID_MAX_C] exchanged
-    h.dpart = h.lpart + MID_MAX_C;                    // [r]       exchanged
-    h.pooled = h.dpart + p.r;                         // [r]
+    h.prodq = h.colsum + p.r;                         // [r+1][C]  this CTA's partial head products, exchanged
+    h.prod = h.prodq + rc;                            // [r+1][C]  their sum over the cluster
+    h.pooled = h.prod + rc;                           // [r]
     h.daL = h.pooled + p.r;                           // [r]
-    h.py = h.daL + p.r;                               // [dg]  hbar slice, then mean_s y
-    h.gk = h.py + p.dg;                               // [dg]
-    h.lg = h.gk + p.dg;                               // [MID_MAX_C] logits, then dlogits
+    h.py = h.daL + p.r;                               // [dg]  slice of mean_s h_L
+    h.lg = h.py + p.dg;                               // [MID_MAX_C] logits, then dlogits
     h.lam_s = h.lg + MID_MAX_C;                       // [MID_MAX_L]
     h.wh_s = h.lam_s + MID_MAX_L;                     // [dg][C] slice of W_head
-    h.lred = h.wh_s + (size_t)p.dg * p.C;             // [nwarps][MID_MAX_L]; also [nwarps][MID_MAX_C] and [parts][r] scratch
+    h.lred = h.wh_s + (size_t)p.dg * p.C;             // [nwarps][MID_MAX_L]; also [parts][r] scratch
     h.wup_s = h.lred + (size_t)p.scratch;             // [r][dg] slice of W_up (when p.wup_smem)
     return h;
 }
@@ -106,21 +104,56 @@ __device__ __forceinline__ void mid_prefetch_head(const MidParams& p, const MidS
     for (int l = t; l < MID_MAX_L; l += nthr) h.lam_s[l] = l < p.L ? p.lam[l] : 0.f;
 }
 
+// The head is linear in mean_s a_L, so both directions through it reduce to one small matrix:
+//   logits = b_head + hbar W_head + (mean_s a_L) (W_up W_head),      d loss / d mean_s a_L = (W_up W_head) dlogits.
+// Each CTA forms the products over its own slice of the hidden width (operands already in shared
+// memory):  prodq[j][c] = sum_k W_up[j][k] W_head[k][c]  (j < r),  prodq[r][c] = sum_k hbar[k] W_head[k][c];
+// the slices are added across the cluster afterwards.  Called by nw whole warps, w = the caller's
+// index among them; none of it depends on u, so it can run while u is still being produced.
+__device__ __forceinline__ void mid_head_products(const MidParams& p, const MidShared& h, int q, int w, int nw, int lane) {
+    const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));
+    for (int j = w; j <= p.r; j += nw) {
+        for (int c0 = 0; c0 < p.C; c0 += 4) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int kk = lane; kk < kn; kk += 32) {
+                const float a = j == p.r ? h.py[kk]
+                              : p.wup_smem ? h.wup_s[(size_t)j * p.dg + kk] : p.W_up[(long long)j * p.d + k0 + kk];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (c0 + c < p.C) acc[c] = fmaf(a, h.wh_s[kk * p.C + c0 + c], acc[c]);
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float v = warp_sum(acc[c]);
+                if (lane == 0 && c0 + c < p.C) h.prodq[j * p.C + c0 + c] = v;
+            }
+        }
+    }
+}
+// After a cluster-wide barrier behind mid_head_products: the sum over the cluster, in rank order.
+__device__ __forceinline__ void mid_sum_products(const MidParams& p, const MidShared& h, cg::cluster_group& cluster, int t, int nthr) {
+    for (int e = t; e < (p.r + 1) * p.C; e += nthr) {
+        float acc = 0.f;
+        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(h.prodq, g)[e];
+        h.prod[e] = acc;
+    }
+}
+
 // Everything after the down-projections for one sample, executed by one CTA (rank q) of the
 // sample's cluster.  GPT: 4-column groups per thread.  u_s: STATE_SMEM: [L][GPT][nt] float4 state;
-// STATE_CLUSTER: this CTA's [layers_per_cta][128][r] fp32 u tiles.  head_prefetched: the caller has
-// already issued mid_prefetch_head (its threads still have to wait for their copies here).
+// STATE_TILES: [L][Sg][r] fp32 u tiles.  products_ready: the caller has already prefetched the head
+// operands, run mid_head_products and passed a cluster barrier.
 template <int ACT, typename DU, int GPT, int STATE>
 __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& cluster, float4* u_s, const MidShared& h,
-                                         bool head_prefetched) {
+                                         bool products_ready) {
     constexpr int LT = MID_MAX_L;
     const int q = (int)cluster.block_rank();
     const int b = blockIdx.x / p.G;
     const int t = threadIdx.x, nt = blockDim.x;
     const int r = p.r, L = p.L, C = p.C;
     const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
-    float *aL = h.aL, *colsum = h.colsum, *lpart = h.lpart, *dpart = h.dpart, *pooled = h.pooled, *daL = h.daL, *py = h.py,
-          *gk = h.gk, *lg = h.lg, *lam_s = h.lam_s, *wh_s = h.wh_s, *lred = h.lred, *wup_s = h.wup_s;
+    float *aL = h.aL, *colsum = h.colsum, *prod = h.prod, *pooled = h.pooled, *daL = h.daL, *py = h.py,
+          *lg = h.lg, *lam_s = h.lam_s, *wh_s = h.wh_s, *lred = h.lred, *wup_s = h.wup_s;
 
     const int groups_per_tok = r >> 2;
     int s_local[GPT], j4[GPT];
@@ -137,22 +170,20 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     }
     DU* du = reinterpret_cast<DU*>(p.du);
     // layer l of group g: read u, park / fetch the reverse-pass state
-    auto cluster_slot = [&](int l, int g) -> float4* {      // STATE_CLUSTER: the element's home in the cluster
-        const int owner = l / p.layers_per_cta, li = l - owner * p.layers_per_cta;
-        float* tile = cluster.map_shared_rank(reinterpret_cast<float*>(u_s), owner);
-        const int row = q * p.Sg + s_local[g];
-        return reinterpret_cast<float4*>(tile + ((size_t)li * 128 + row) * r + ((((j4[g] >> 2) ^ (row & p.u_swz))) << 2));
+    auto tile_slot = [&](int l, int g) -> float4* {          // STATE_TILES
+        float* row = reinterpret_cast<float*>(u_s) + ((size_t)l * p.Sg + s_local[g]) * r;
+        return reinterpret_cast<float4*>(row + (((j4[g] >> 2) ^ (s_local[g] & p.u_swz)) << 2));
     };
     auto load_u = [&](int l, int g) -> float4 {
         if constexpr (STATE == STATE_SMEM) return u_s[((size_t)l * GPT + g) * nt + t];
-        else if constexpr (STATE == STATE_CLUSTER) return *cluster_slot(l, g);
+        else if constexpr (STATE == STATE_TILES) return *tile_slot(l, g);
         else return *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base[g]);
     };
     auto store_w = [&](int l, int g, const float* wv) {
         if constexpr (STATE == STATE_SMEM) {
             u_s[((size_t)l * GPT + g) * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
-        } else if constexpr (STATE == STATE_CLUSTER) {
-            *cluster_slot(l, g) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+        } else if constexpr (STATE == STATE_TILES) {
+            *tile_slot(l, g) = make_float4(wv[0], wv[1], wv[2], wv[3]);
         } else if constexpr (sizeof(DU) == 2) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]), hi = __floats2bfloat162_rn(wv[2], wv[3]);
             uint2 pk;
@@ -166,8 +197,8 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     auto load_w = [&](int l, int g) -> float4 {
         if constexpr (STATE == STATE_SMEM) {
             return u_s[((size_t)l * GPT + g) * nt + t];
-        } else if constexpr (STATE == STATE_CLUSTER) {
-            return *cluster_slot(l, g);
+        } else if constexpr (STATE == STATE_TILES) {
+            return *tile_slot(l, g);
         } else if constexpr (sizeof(DU) == 2) {
             const uint2 pk = *reinterpret_cast<const uint2*>(du + (long long)l * p.lstride + base[g]);
             const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
@@ -177,6 +208,10 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             return *reinterpret_cast<const float4*>(du + (long long)l * p.lstride + base[g]);
         }
     };
+    const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
+    const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
+    if (!products_ready) mid_prefetch_head(p, h, q, id, t, nt);
+    cp_async_commit();                                                          // group: head operands
     if constexpr (STATE == STATE_SMEM) {
 #pragma unroll
         for (int g = 0; g < GPT; ++g)
@@ -184,13 +219,15 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 for (int l = 0; l < L; ++l) cp_async_16(u_s + ((size_t)l * GPT + g) * nt + t, p.u + (long long)l * p.lstride + base[g]);
     }
     cp_async_commit();                                                          // group: u
-    const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
-    const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
-    if (!head_prefetched) mid_prefetch_head(p, h, q, id, t, nt);
-    cp_async_commit();                                                          // group: head operands
     const int label = p.train ? p.labels[id] : 0;
-    __syncthreads();
-    cp_async_wait_group<1>();                                                   // own u values have landed
+    if (!products_ready) {
+        cp_async_wait_group<1>();                                               // head operands have landed ...
+        __syncthreads();                                                        // ... those of every thread
+        mid_head_products(p, h, q, warp, nwarps, lane);                         // overlaps the u copies in flight
+        cluster.sync();
+    }
+    mid_sum_products(p, h, cluster, t, nt);              // read after the block barriers below
+    cp_async_wait_group<0>();                            // own u values have landed
 
     // ---- forward chain over each group of 4 adapter columns of one token.  The slot that held
     // u_l is overwritten with u_l - a_{l-1} (= d z_l / d lambda_l) for the reverse pass; the ReLU
@@ -264,37 +301,12 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(colsum, g)[j];
         pooled[j] = acc / (float)p.S;                     // mean_s a_L
     }
-    cp_async_wait_group<0>();
     __syncthreads();
 
-    // ---- head on this CTA's slice of the hidden width ----
-    for (int kk = t; kk < kn; kk += nt) {
-        float acc = 0.f;
-        if (p.wup_smem) {
-#pragma unroll 8
-            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], wup_s[(size_t)j * p.dg + kk], acc);
-        } else {
-            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], p.W_up[(long long)j * p.d + k0 + kk], acc);
-        }
-        py[kk] += acc;                                    // mean_s y = mean_s h_L + (mean_s a_L) W_up
-    }
-    __syncthreads();
-    for (int c = 0; c < C; ++c) {
-        float part = 0.f;
-        for (int kk = t; kk < kn; kk += nt) part = fmaf(py[kk], wh_s[kk * C + c], part);
-        part = warp_sum(part);
-        if (lane == 0) lred[warp * MID_MAX_C + c] = part;
-    }
-    __syncthreads();
+    // ---- head: logits, loss, dlogits and d loss / d a_L, the same in every CTA of the cluster ----
     if (t < C) {
-        float acc = 0.f;
-        for (int wv = 0; wv < nwarps; ++wv) acc += lred[wv * MID_MAX_C + t];
-        lpart[t] = acc;
-    }
-    cluster.sync();
-    if (t < C) {
-        float acc = p.b_head[t];
-        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(lpart, g)[t];
+        float acc = p.b_head[t] + prod[r * C + t];        // b_head + (mean_s h_L) W_head
+        for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], prod[j * C + t], acc);
         lg[t] = acc;
         if (q == 0) p.logits_out[(long long)b * C + t] = acc;
     }
@@ -317,31 +329,9 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         }
         __syncthreads();
     }
-    for (int kk = t; kk < kn; kk += nt) {
-        const int k = k0 + kk;
-        float acc = 0.f;
-        for (int c = 0; c < C; ++c) acc = fmaf(wh_s[kk * C + c], lg[c], acc);
-        gk[kk] = acc;                                     // d loss / d mean_s y
-        p.gvec[(long long)b * p.d + k] = acc;
-        p.pooled_y[(long long)b * p.d + k] = py[kk];
-    }
-    if (q == 0)
-        for (int j = t; j < r; j += nt) p.pooled_a[(long long)b * r + j] = pooled[j];
-    __syncthreads();
-    for (int j = warp; j < r; j += nwarps) {
-        float part = 0.f;
-        if (p.wup_smem) {
-            for (int kk = lane; kk < kn; kk += 32) part = fmaf(wup_s[(size_t)j * p.dg + kk], gk[kk], part);
-        } else {
-            for (int kk = lane; kk < kn; kk += 32) part = fmaf(p.W_up[(long long)j * p.d + k0 + kk], gk[kk], part);
-        }
-        part = warp_sum(part);
-        if (lane == 0) dpart[j] = part;
-    }
-    cluster.sync();
     for (int j = t; j < r; j += nt) {
         float acc = 0.f;
-        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(dpart, g)[j];
+        for (int c = 0; c < C; ++c) acc = fmaf(prod[j * C + c], lg[c], acc);
         daL[j] = acc / (float)p.S;                         // da_L, the same for every token of the sample
     }
     __syncthreads();
@@ -395,6 +385,24 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             }
         }
     }
+    // ---- per-sample vectors the gradient finalisation needs, for this CTA's slice of the hidden
+    // width: mean_s y = mean_s h_L + (mean_s a_L) W_up  and  g = d loss / d mean_s y = W_head dlogits ----
+    for (int kk = t; kk < kn; kk += nt) {
+        const int k = k0 + kk;
+        float acc = 0.f;
+        if (p.wup_smem) {
+#pragma unroll 8
+            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], wup_s[(size_t)j * p.dg + kk], acc);
+        } else {
+            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], p.W_up[(long long)j * p.d + k], acc);
+        }
+        float gv = 0.f;
+        for (int c = 0; c < C; ++c) gv = fmaf(wh_s[kk * C + c], lg[c], gv);
+        p.pooled_y[(long long)b * p.d + k] = py[kk] + acc;
+        p.gvec[(long long)b * p.d + k] = gv;
+    }
+    if (q == 0)
+        for (int j = t; j < r; j += nt) p.pooled_a[(long long)b * r + j] = pooled[j];
     __syncthreads();
     if (t < L) {
         float acc = 0.f;
@@ -521,11 +529,11 @@ struct MidPlan {
 inline size_t mid_base_floats(const Dims& dm, int Sg, int dg, int th, int* scratch_out) {
     const int nw = th / 32;
     int scratch = nw * MID_MAX_L;
-    if (nw * MID_MAX_C > scratch) scratch = nw * MID_MAX_C;
     const int parts = th / dm.r > 0 ? th / dm.r : 1;
     if (parts * dm.r > scratch) scratch = parts * dm.r;
     *scratch_out = scratch;
-    return (size_t)Sg * dm.r + 4 * (size_t)dm.r + 2 * (size_t)dg + 2 * MID_MAX_C + MID_MAX_L + scratch + (size_t)dg * dm.C + 4;
+    return (size_t)Sg * dm.r + 3 * (size_t)dm.r + 2 * (size_t)(dm.r + 1) * dm.C + (size_t)dg + MID_MAX_C + MID_MAX_L + scratch +
+           (size_t)dg * dm.C + 4;
 }
 
 inline MidPlan mid_plan(const Dims& dm) {

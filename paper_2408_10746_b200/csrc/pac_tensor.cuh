@@ -83,6 +83,19 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
 }
+// The same with every lane of a converged warp waiting; all lanes get the same answer.  Loops that
+// issue TMA copies or MMAs are run by the whole warp with one elected lane issuing, so that
+// addresses and descriptors stay warp-uniform values for the compiler.
+__device__ __forceinline__ bool mbar_wait_uniform(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status);
+    return __all_sync(0xffffffffu, ok) != 0;
+}
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xffffffff;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+    return pred != 0;
+}
 // After a wait gave up: give copies that are still in flight time to land before the CTA ends.
 __device__ __forceinline__ void drain_after_abort(volatile int* abort_flag) {
     if (*abort_flag)
@@ -240,50 +253,54 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     volatile int* abort_flag = &abort_sh;
     pdl_wait();            // everything above overlapped the previous kernel; its results are needed from here on
 
+    // The two pipeline loops are run by whole converged warps with one elected lane issuing, so that
+    // addresses, coordinates and descriptors stay warp-uniform values.
     if (warp == 0) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            // cache tiles are read once per pass: evict them first, so that u, du, the weight shadow and
-            // the optimizer state stay L2-resident
-            const uint64_t pol = l2_policy_evict_first();
-            for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
-                const int sc = t % p.s_chunks, b = (t / p.s_chunks) % p.B, l = t / (p.s_chunks * p.B);
-                const int id = (int)safe_id(p.ids, b, p.N, nullptr);
-                for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (it / p.stages) & 1;
-                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-                    const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+        uint32_t it = 0;
+        // cache tiles are read once per pass: evict them first, so that u, du, the weight shadow and
+        // the optimizer state stay L2-resident
+        const uint64_t pol = l2_policy_evict_first();
+        bool ok = true;
+        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+            const int sc = t % p.s_chunks, b = (t / p.s_chunks) % p.B, l = t / (p.s_chunks * p.B);
+            const int id = (int)safe_id(p.ids, b, p.N, nullptr);
+            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+                const int s = it % p.stages;
+                const uint32_t ph = (it / p.stages) & 1;
+                if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+                if (elect_one()) {
                     mbar_expect_tx(full0 + 8 * s, a_bytes + b_bytes);
                     tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, sc * FWD_ROWS, l, id, pol);
                     for (int rb = 0; rb < r_blocks; ++rb)
                         tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full0 + 8 * s, rb * 64, kc * KC, 0, l);
                 }
+                __syncwarp();
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // wide_n: the hi and lo blocks lie next to each other along N ([r block][hi|lo] in 64-column
-            // blocks), so one MMA of N = 128 * r_blocks yields u_hi | u_lo side by side in TMEM
-            const uint32_t idesc = p.wide_n ? instr_desc_bf16(FWD_ROWS, 128 * r_blocks, 0, 1) : instr_desc_bf16(FWD_ROWS, r_pad, 0, 1);
-            uint32_t it = 0, tile_n = 0;
-            for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++tile_n) {
-                const int buf = tile_n & 1;
-                const uint32_t aph = (tile_n >> 1) & 1;
-                if (!mbar_wait(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
+        // wide_n: the hi and lo blocks lie next to each other along N ([r block][hi|lo] in 64-column
+        // blocks), so one MMA of N = 128 * r_blocks yields u_hi | u_lo side by side in TMEM
+        const uint32_t idesc = p.wide_n ? instr_desc_bf16(FWD_ROWS, 128 * r_blocks, 0, 1) : instr_desc_bf16(FWD_ROWS, r_pad, 0, 1);
+        uint32_t it = 0, tile_n = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_n) {
+            const int buf = tile_n & 1;
+            const uint32_t aph = (tile_n >> 1) & 1;
+            if (!mbar_wait_uniform(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_stride);
+            bool ok = true;
+            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+                const int s = it % p.stages;
+                const uint32_t ph = (it / p.stages) & 1;
+                if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_stride);
-                bool ok = true;
-                for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (it / p.stages) & 1;
-                    if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + b_off;
-                    // descriptors of the first 16-wide K step; later steps only move the start address
-                    // (field in 16-byte units): +32 B per step in the K-major A tile, +2048 B (16 rows) in B
-                    const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
-                    const uint64_t bh0 = smem_desc_sw128(b0, 2 * b_box, 1024), bl0 = smem_desc_sw128(b0 + b_box, 2 * b_box, 1024);
+                const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + b_off;
+                // descriptors of the first 16-wide K step; later steps only move the start address
+                // (field in 16-byte units): +32 B per step in the K-major A tile, +2048 B (16 rows) in B
+                const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
+                const uint64_t bh0 = smem_desc_sw128(b0, 2 * b_box, 1024), bl0 = smem_desc_sw128(b0 + b_box, 2 * b_box, 1024);
+                if (elect_one()) {
                     if (p.wide_n) {
                         const uint64_t bw0 = smem_desc_sw128(b0, b_box, 1024);
 #pragma unroll
@@ -298,9 +315,11 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     }
                     umma_commit(empty0 + 8 * s);          // frees the smem slot once these MMAs are done
                 }
-                if (!ok) break;
-                umma_commit(accf0 + 8 * buf);             // accumulator complete
+                __syncwarp();
             }
+            if (!ok) break;
+            if (elect_one()) umma_commit(accf0 + 8 * buf);    // accumulator complete
+            __syncwarp();
         }
     } else {
         const int q = warp & 3;                           // TMEM lane quadrant this warp may read
@@ -407,45 +426,50 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     pdl_wait();
 
     if (warp == 0) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            const uint64_t pol = l2_policy_evict_first();
-            for (int rt = rt0; rt < rt1; ++rt, ++it) {
-                const int sc = rt % p.s_chunks, b = rt / p.s_chunks;
-                const int id = (int)safe_id(p.ids, b, p.N, nullptr);
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+        uint32_t it = 0;
+        const uint64_t pol = l2_policy_evict_first();
+        for (int rt = rt0; rt < rt1; ++rt, ++it) {
+            const int sc = rt % p.s_chunks, b = rt / p.s_chunks;
+            const int id = (int)safe_id(p.ids, b, p.N, nullptr);
+            const int s = it % p.stages;
+            const uint32_t ph = (it / p.stages) & 1;
+            if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
+            const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+            if (elect_one()) {
                 mbar_expect_tx(full0 + 8 * s, stage_bytes);
                 for (int q = 0; q < 2 * p.chunks; ++q)
                     tma_load_4d_hint(dst + q * box_bytes, &map_cache, full0 + 8 * s, col0 + q * 64, sc * BWD_KR, l, id, pol);
                 for (int q = 0; q < p.r_blocks; ++q)
                     tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full0 + 8 * s, q * 64, b * p.S + sc * BWD_KR, l);
             }
+            __syncwarp();
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(128, r_pad, 1, 1);
-            uint32_t it = 0;
-            bool ok = true;
-            for (int rt = rt0; rt < rt1 && ok; ++rt, ++it) {
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
-                const uint64_t bd0 = smem_desc_sw128(b0, box_bytes, 1024);
-                for (int c = 0; c < p.chunks; ++c) {
-                    const uint64_t ad0 = smem_desc_sw128(a0 + c * 2 * box_bytes, box_bytes, 1024);
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(c * r_pad);
+        const uint32_t idesc = instr_desc_bf16(128, r_pad, 1, 1);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int rt = rt0; rt < rt1 && ok; ++rt, ++it) {
+            const int s = it % p.stages;
+            const uint32_t ph = (it / p.stages) & 1;
+            if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
+            const uint64_t bd0 = smem_desc_sw128(b0, box_bytes, 1024);
+            if (elect_one()) {
+                // consecutive MMAs alternate between the column blocks' accumulators: an MMA that adds to
+                // the result of the one before it would have to wait for that one to finish
 #pragma unroll
-                    for (int k = 0; k < BWD_KR / 16; ++k)      // 16 tokens = 2048 B further along K in both operands
-                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 128), bd0 + (uint64_t)(k * 128), idesc, (it | (uint32_t)k) ? 1u : 0u);
-                }
+                for (int k = 0; k < BWD_KR / 16; ++k)          // 16 tokens = 2048 B further along K in both operands
+                    for (int c = 0; c < p.chunks; ++c)
+                        umma_bf16(tmem_base + (uint32_t)(c * r_pad), smem_desc_sw128(a0 + c * 2 * box_bytes, box_bytes, 1024) + (uint64_t)(k * 128),
+                                  bd0 + (uint64_t)(k * 128), idesc, (it | (uint32_t)k) ? 1u : 0u);
                 umma_commit(empty0 + 8 * s);
             }
-            if (ok) umma_commit(accf);
+            __syncwarp();
+        }
+        if (ok) {
+            if (elect_one()) umma_commit(accf);
+            __syncwarp();
         }
     } else {
         const int q = warp & 3;
