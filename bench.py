@@ -270,8 +270,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--force-simt", action="store_true", help="use the plain fp32-FMA kernels")
-    ap.add_argument("--one-kernel-forward", action="store_true",
-                    help="tensor-core path with the down-projections and the head phase in one kernel")
+    ap.add_argument("--forward", choices=["auto", "split", "one-kernel"], default="auto",
+                    help="tensor-core path: down-projections and head phase as one kernel or two (default: library's choice)")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "dp"],
                     help="N > 1: independent replicas (default) or data parallel with a per-step all-reduce of "
                          "the adapter gradients (paper Section V-B)")
@@ -322,8 +322,8 @@ def main():
     ctx = pac.PacContext(local, stream.cuda_stream)
     if args.force_simt:
         ctx.set_option(binding.PAC_OPT_KERNEL_PATH, 1)
-    elif args.one_kernel_forward:
-        ctx.set_option(binding.PAC_OPT_KERNEL_PATH, 3)
+    elif args.forward != "auto":
+        ctx.set_option(binding.PAC_OPT_KERNEL_PATH, 3 if args.forward == "one-kernel" else 2)
     ctx.cache_register(cache, labels)
     ctx.adapter_init(r=spec.r, n_out=spec.n_out, max_batch=spec.B,
                      head=pac.PAC_HEAD_FROZEN_LM if spec.head == "lm" else pac.PAC_HEAD_MEANPOOL_CLS, lm_head=lm)

@@ -71,13 +71,15 @@ typedef struct { float lr, beta1, beta2, eps, weight_decay; } pac_adamw;
 
 /* Options for pac_set_option. */
 typedef enum {
-    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic (tensor-core path when the shape allows; currently the
-                                     same kernels as 2),
+    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic: tensor-core path when the shape allows; its forward half
+                                     (down-projections + classifier-head phase) runs as ONE launch per
+                                     step when the shape allows it (bf16 cache, classifier head, S <= 128,
+                                     r <= 64) and the batch's clusters all fit on the device at once,
+                                     otherwise as two launches,
                                  1 = force the plain fp32-FMA kernels,
-                                 2 = tensor-core path with the down-projections and the classifier-head
-                                     kernel as separate launches,
-                                 3 = tensor-core path with both in ONE launch per step where the shape
-                                     allows (bf16 cache, classifier head, S <= 128, r <= 64), else as 2;
+                                 2 = tensor-core path, forward half always as two launches,
+                                 3 = tensor-core path, forward half as one launch whenever the shape
+                                     allows it, whatever the batch size;
                                  set before adapter_init */
     PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events */
 } pac_option;
@@ -173,8 +175,8 @@ pac_status pac_launch_count(pac_ctx* ctx, long long* n);
 pac_status pac_sync(pac_ctx* ctx);
 const char* pac_last_error(const pac_ctx* ctx);
 /* Which kernels the next train step will use (valid after adapter_init): "simt", "tensor", or
- * "tensor+fused_forward" when the down-projections (Section IV-A) and the whole classifier-head
- * phase run as one launch per step (bf16 cache, S <= 128, r <= 64). */
+ * "tensor+fused_forward" when a batch of max_batch samples runs the down-projections
+ * (Section IV-A) and the whole classifier-head phase as one launch per step. */
 const char* pac_kernel_path(const pac_ctx* ctx);
 
 /* Block-wise absmax INT8 quantisation, Section IV-D, Eq. 1 (the paper applies it to the frozen

@@ -91,7 +91,7 @@ struct pac_ctx {
     TensorPlan tplan{};
     MidPlan mplan{};               // fused classifier-head kernel (when the shape allows)
     FusedFwdPlan fplan{};          // down-projections + classifier-head kernel in one launch (short sequences)
-    int one_kernel_forward = 0;    // 1: down-projections and head phase as one launch when the shape allows
+    int forward_mode = 0;          // 0: one-launch forward when a batch's clusters fit the device at once, 2: never, 3: whenever the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
     bool lm_tensor = false;
     std::string err;
@@ -363,8 +363,13 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
 }
 
 bool use_fused_cls(const pac_ctx* c) { return c->cfg.head == PAC_HEAD_MEANPOOL_CLS && c->mplan.ok; }
-bool use_fused_fwd(const pac_ctx* c) { return use_fused_cls(c) && use_tensor(c) && c->fplan.ok; }
-int cls_cluster_size(const pac_ctx* c) { return use_fused_fwd(c) ? c->fplan.mp.G : c->mplan.G; }
+// The one-launch forward pays off when all of the batch's clusters run at the same time (its GEMM
+// and chain phases do not overlap across waves); larger batches keep the two separate kernels.
+bool use_fused_fwd(const pac_ctx* c, int B) {
+    if (!use_fused_cls(c) || !use_tensor(c) || !c->fplan.ok) return false;
+    return c->forward_mode == 3 || B <= c->fplan.max_clusters;
+}
+int cls_cluster_size(const pac_ctx* c, int B) { return use_fused_fwd(c, B) ? c->fplan.mp.G : c->mplan.G; }
 
 pac_status down_projection(pac_ctx* c, const int* d_ids, int B) {
     pac_status st;
@@ -439,7 +444,7 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
 // Forward half of a classifier-head step (everything up to du and the per-sample head vectors).
 pac_status cls_forward_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
     pac_status st;
-    if (use_fused_fwd(c)) {
+    if (use_fused_fwd(c, B)) {
         time_mark(c, 0, false);
         st = fused_fwd_enqueue(c, d_ids, B, train, d_logits_out);
         time_mark(c, 0, true);
@@ -465,7 +470,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
     f.dw_part = sc.dw_part;
     f.splits = use_tensor(c) ? tensor_splits(c->tplan, B) : 1;
     f.dw_elems = (long long)dm.L * dm.d * dm.r;
-    f.lam_part = sc.lam_part; f.lam_blocks = B * cls_cluster_size(c);
+    f.lam_part = sc.lam_part; f.lam_blocks = B * cls_cluster_size(c, B);
     f.pooled_a = sc.pooled_a; f.gvec = sc.gvec; f.pooled_y = sc.pooled_y; f.dlogits = sc.dlogits; f.loss_b = sc.loss_b;
     f.grads = c->grads; f.loss_out = d_loss;
     f.adam = hp ? 1 : 0;
@@ -641,7 +646,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     c->mplan = cls ? mid_plan(dm) : MidPlan{};
     if (c->mplan.ok && cfg->max_batch * c->mplan.G > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * c->mplan.G;
     FusedFwdPlan fwd_plan{};
-    if (c->mplan.ok && c->dtype == PAC_BF16 && tensor_shape_supported(dm) && !c->force_simt && c->one_kernel_forward) {
+    if (c->mplan.ok && c->dtype == PAC_BF16 && tensor_shape_supported(dm) && !c->force_simt && c->forward_mode != 2) {
         int max_smem = 0;
         CU_OK(c, cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device));
         fwd_plan = fused_fwd_plan(dm, max_smem);
@@ -700,7 +705,10 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             if (ts == PAC_OK) {
                 A(dmalloc(c, &s.dw_part, part_floats));
                 c->tensor_ok = (st == PAC_OK);
-                if (c->tensor_ok) c->fplan = fwd_plan;
+                if (c->tensor_ok && fwd_plan.ok) {
+                    fwd_plan.max_clusters = fused_fwd_max_clusters(fwd_plan, cfg->act);
+                    if (fwd_plan.max_clusters > 0) c->fplan = fwd_plan;
+                }
             } else if (ts != PAC_ERR_UNSUPPORTED) {
                 st = fail(c, ts, "tensor path set-up failed: %s", tensor_last_error());
             }
@@ -902,7 +910,7 @@ pac_status pac_set_option(pac_ctx* c, int option, int value) {
         if (value < 0 || value > 3) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0, 1, 2 or 3");
         if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_set_option: set the kernel path before pac_adapter_init");
         c->force_simt = value == 1;
-        c->one_kernel_forward = value == 3;
+        c->forward_mode = value >= 2 ? value : 0;
         return PAC_OK;
     }
     if (option == PAC_OPT_KERNEL_TIMING) {
@@ -955,7 +963,7 @@ const char* pac_last_error(const pac_ctx* c) { return c ? c->err.c_str() : "null
 
 const char* pac_kernel_path(const pac_ctx* c) {
     if (!c || !c->inited || !use_tensor(c)) return "simt";
-    return use_fused_fwd(c) ? "tensor+fused_forward" : "tensor";
+    return use_fused_fwd(c, c->cfg.max_batch) ? "tensor+fused_forward" : "tensor";
 }
 
 }  // extern "C"

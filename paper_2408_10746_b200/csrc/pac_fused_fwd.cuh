@@ -168,6 +168,7 @@ struct FusedFwdPlan {
     bool ok = false;
     MidPlan mp;
     int layers_per_cta = 0, stages = 0, k_chunks = 0, u_swz = 0;
+    int max_clusters = 0;          // clusters of this shape the device runs at the same time
     size_t mid_offset = 0, smem = 0;
 };
 
@@ -205,6 +206,35 @@ inline FusedFwdPlan fused_fwd_plan(const Dims& dm, int max_smem) {
         }
     }
     return fp;
+}
+
+// How many of the plan's clusters can be resident at once (0 when the query fails).
+template <int ACT>
+inline int fused_fwd_max_clusters_act(const FusedFwdPlan& pl) {
+    if (cudaFuncSetAttribute(fwd_cluster_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(pl.mp.G * 1024), 1, 1);
+    cfg.blockDim = dim3((unsigned)pl.mp.threads, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)pl.mp.G;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, fwd_cluster_kernel<ACT>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+inline int fused_fwd_max_clusters(const FusedFwdPlan& pl, int act) {
+    return act == PAC_ACT_RELU ? fused_fwd_max_clusters_act<PAC_ACT_RELU>(pl) : fused_fwd_max_clusters_act<PAC_ACT_IDENTITY>(pl);
 }
 
 template <int ACT>

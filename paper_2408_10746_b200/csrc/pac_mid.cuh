@@ -499,13 +499,13 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         const long long e = i - lay.w_up;
         const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
         g = 0.f;
-#pragma unroll 8
+#pragma unroll 16
         for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], f.gvec[(long long)b * f.d + k], g);
     } else if (i < lay.b_head) {
         const long long e = i - lay.w_head;
         const int k = (int)(e / f.C), c = (int)(e - (long long)k * f.C);
         g = 0.f;
-#pragma unroll 8
+#pragma unroll 16
         for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_y[(long long)b * f.d + k], f.dlogits[(long long)b * f.C + c], g);
     } else {
         const int c = (int)(i - lay.b_head);
