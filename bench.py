@@ -7,7 +7,7 @@ One "step" is one pass of the whole hot path over one minibatch: gather of the c
 states, adapter forward, head and loss, adapter-only backward, AdamW.  `value` is
 samples/s with the cache, the shuffled ids and the losses resident in HBM (one
 pac_train_epoch_dev call over K*B ids); `e2e` is the same metric through
-pac_train_step/pac_adam_step with host ids in and the host loss out every step.
+pac_train_step_async with host ids in and the host loss out every step.
 Prints ONE JSON line (rank 0).
 """
 from __future__ import annotations
@@ -364,22 +364,30 @@ def main():
     if not np.isfinite(losses).all():
         raise SystemExit("non-finite loss in the timed region")
 
-    # ---------------- end to end through the public per-step calls ----------------
-    for i in range(3):
-        ctx.train_step(ids_host[i * B:(i + 1) * B]); ctx.adam_step(hp)
+    # ---------------- end to end through the public per-step call ----------------
+    # every step: B ids from page-locked host memory in (H2D), the step's loss out to page-locked
+    # host memory (D2H); one wait at the end, then every loss is checked on the host
     Ke = min(K, 512)
+    h_ids = torch.from_numpy(ids_host[:Ke * B].copy()).pin_memory()
+    h_losses = torch.zeros(Ke, dtype=torch.float32).pin_memory()
+    ids_view, loss_ptr = h_ids.numpy(), h_losses.data_ptr()
+    for i in range(3):
+        ctx.train_step_async(ids_view[i * B:(i + 1) * B], hp, loss_ptr + 4 * i)
+    ctx.sync()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t0 = time.perf_counter()
     with torch.cuda.stream(stream):
         e0.record(stream)
         for i in range(Ke):
-            ctx.train_step(ids_host[i * B:(i + 1) * B], want_loss=True)
-            ctx.adam_step(hp)
+            ctx.train_step_async(ids_view[i * B:(i + 1) * B], hp, loss_ptr + 4 * i)
         e1.record(stream)
+    ctx.sync()
     barrier()
     wall_ms = 1e3 * (time.perf_counter() - t0)
     e2e_ms = max(e0.elapsed_time(e1), wall_ms)
+    if not np.isfinite(h_losses.numpy()).all():
+        raise SystemExit("non-finite loss in the end-to-end region")
 
     # ---------------- per-kernel times of the two cache-stream kernels ----------------
     ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 1)
@@ -387,6 +395,11 @@ def main():
     Kt = min(K, 256)
     ctx.train_epoch_dev(d_ids[:Kt * B], B, hp, None)
     kt = ctx.kernel_times()
+    # the same steps once more with device-side timestamps of the passes' stream phases; no event
+    # brackets, so the kernels overlap as in the timed region
+    ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 2)
+    ctx.train_epoch_dev(d_ids[:Kt * B], B, hp, None)
+    pt = ctx.stream_phase_times()
     ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 0)
 
     if dist is not None:
@@ -403,6 +416,12 @@ def main():
             kern[name] = {"avg_ms": avg, "launches": cnt}
             if name in ("down_projection", "dw_down"):      # the two passes over the cached activations
                 kern[name]["gbs"] = pass_bytes / (avg * 1e-3) / 1e9
+    phases = {}
+    for name, (tot_ms, cnt) in pt.items():
+        if cnt:
+            avg = tot_ms / cnt
+            phases[name] = {"avg_ms": avg, "launches": cnt, "gbs": pass_bytes / (avg * 1e-3) / 1e9,
+                            "frac": pass_bytes / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     stream_k = [k for k in kern if "gbs" in kern[k]]
     dominant = max(stream_k, key=lambda k: kern[k]["avg_ms"]) if stream_k else None
     roofline = None
@@ -411,7 +430,10 @@ def main():
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"],
                     "traffic": ncu_traffic(spec, ctx.kernel_path(), dominant), "algorithmic_bytes_per_launch": pass_bytes,
-                    "kernels": kern}
+                    "kernels": kern,
+                    # first cache copy issued -> last accumulator complete, over all CTAs of a launch (device
+                    # timestamps): the part of each pass that streams the minibatch's slabs
+                    "stream_phase": phases}
     step_s = ms * 1e-3 / K
     stream_gbs = 2 * pass_bytes / step_s / 1e9
 

@@ -81,7 +81,9 @@ typedef enum {
                                  3 = tensor-core path, forward half as one launch whenever the shape
                                      allows it, whatever the batch size;
                                  set before adapter_init */
-    PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events */
+    PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events
+                                 (pac_kernel_times), 2 = device-side timestamps of the two passes' stream
+                                 phases on the tensor-core path (pac_stream_phase_times) */
 } pac_option;
 
 /* Creates a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t to
@@ -111,6 +113,17 @@ pac_status pac_adapter_init(pac_ctx* ctx, const pac_adapter_cfg* cfg, unsigned l
  * parameters.  If loss_out (host) is non-NULL the call waits for the stream and stores
  * the mean loss; if NULL the call returns as soon as the work is enqueued. */
 pac_status pac_train_step(pac_ctx* ctx, const int* sample_ids, int B, float* loss_out);
+
+/* One whole training step without waiting: pac_train_step on sample_ids (host, B ints) followed by
+ * the AdamW update of pac_adam_step with `hp`, all enqueued on the context's stream; the call
+ * returns as soon as that is done (it waits only when more than 8 earlier steps' ids are still in
+ * flight).  If loss_out is non-NULL the step's mean loss is copied there once the step has run:
+ * loss_out is HOST memory that must stay valid until the next pac_sync (page-locked memory keeps
+ * the copy asynchronous); read it after pac_sync.  Errors of the arguments are reported at once,
+ * device-side errors by the next pac_sync.  The step a caller loops over when the minibatches
+ * are chosen on the host one at a time (Section IV-B: from the second epoch on a step needs
+ * nothing but the cached activations of its samples). */
+pac_status pac_train_step_async(pac_ctx* ctx, const int* sample_ids, int B, const pac_adamw* hp, float* loss_out);
 
 /* AdamW on the adapter parameters (and the classifier head) from the current gradients:
  * decoupled decay on W_down, W_up, W_head; none on lambda and b_head; bias-corrected
@@ -168,6 +181,17 @@ pac_status pac_set_option(pac_ctx* ctx, int option, int value);
  * bracketed launches since the last call in out_ms[4] and out_count[4] (host arrays).
  * At most 4096 brackets per group are kept between two calls. */
 pac_status pac_kernel_times(pac_ctx* ctx, double* out_ms, long long* out_count);
+/* Stream phases of the two passes over the cached activations (Section IV-B), timed on the device.
+ * With PAC_OPT_KERNEL_TIMING = 2 every later launch of a tensor-core cache pass records, through
+ * %globaltimer, the earliest time any of its CTAs issued its first cache copy and the latest time
+ * any of its CTAs saw its last accumulator complete.  The difference is the time the minibatch's
+ * slabs took to stream from memory through the tensor cores, without the kernel's launch, set-up
+ * and (for the one-launch forward) its chain / head phase; the launch overlap between the kernels
+ * of a step stays as it is without timing.  This call waits for the stream, then stores the summed
+ * milliseconds and the number of timed launches since the last call in out_ms[2] / out_count[2]
+ * (host arrays): [0] first pass (down-projections), [1] second pass (dW_down).  At most 1024
+ * launches per pass are kept between two calls. */
+pac_status pac_stream_phase_times(pac_ctx* ctx, double* out_ms, long long* out_count);
 /* Number of kernels this context has launched so far. */
 pac_status pac_launch_count(pac_ctx* ctx, long long* n);
 /* Waits for the context's stream; reports device-side status words (bounded waits that

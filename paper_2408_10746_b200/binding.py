@@ -22,10 +22,10 @@ STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_S
                 "PAC_ERR_UNSUPPORTED", "PAC_ERR_NOMEM", "PAC_ERR_CUDA", "PAC_ERR_TIMEOUT"]
 
 # every symbol include/pac.h declares
-EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init", "pac_train_step",
+EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init", "pac_train_step", "pac_train_step_async",
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
-           "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_launch_count", "pac_sync", "pac_last_error",
+           "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_stream_phase_times", "pac_launch_count", "pac_sync", "pac_last_error",
            "pac_kernel_path", "pac_eval_logits_static", "pac_quantize_absmax", "pac_dequantize_absmax"]
 
 
@@ -80,7 +80,7 @@ def load_library() -> C.CDLL:
         "pac_create": [C.POINTER(P), I, P], "pac_destroy": [P],
         "pac_cache_register": [P, P, I, LL, I, I, I, P, I],
         "pac_adapter_init": [P, C.POINTER(_AdapterCfg), C.c_ulonglong],
-        "pac_train_step": [P, P, I, C.POINTER(F)], "pac_adam_step": [P, C.POINTER(_AdamW)],
+        "pac_train_step": [P, P, I, C.POINTER(F)], "pac_train_step_async": [P, P, I, C.POINTER(_AdamW), P], "pac_adam_step": [P, C.POINTER(_AdamW)],
         "pac_eval_logits": [P, P, I, P], "pac_gather": [P, P, I, P],
         "pac_train_epoch": [P, P, LL, I, C.POINTER(_AdamW), P],
         "pac_train_epoch_dev": [P, P, LL, I, C.POINTER(_AdamW), P],
@@ -89,6 +89,7 @@ def load_library() -> C.CDLL:
         "pac_set_opt_state": [P, P, P, LL], "pac_set_option": [P, I, I],
         "pac_launch_count": [P, C.POINTER(LL)], "pac_sync": [P],
         "pac_kernel_times": [P, C.POINTER(C.c_double), C.POINTER(LL)],
+        "pac_stream_phase_times": [P, C.POINTER(C.c_double), C.POINTER(LL)],
         "pac_device_buffers": [P, C.POINTER(P), C.POINTER(P)], "pac_params_changed": [P],
     }
     for name, args in sig.items():
@@ -185,6 +186,13 @@ class PacContext:
         self._ck(self._lib.pac_train_step(self._h, ids.ctypes.data, ids.size, C.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
 
+    def train_step_async(self, sample_ids, hp: AdamW, loss_out_ptr: int = 0):
+        """Enqueues one whole step (forward, backward, AdamW) and returns at once.  loss_out_ptr: address
+        of one host float (page-locked for a truly asynchronous copy) that receives the loss, or 0."""
+        ids = _ids(sample_ids)
+        self._ck(self._lib.pac_train_step_async(self._h, ids.ctypes.data, ids.size, C.byref(hp._c()),
+                                                C.c_void_p(loss_out_ptr) if loss_out_ptr else None))
+
     def adam_step(self, hp: AdamW):
         self._ck(self._lib.pac_adam_step(self._h, C.byref(hp._c())))
 
@@ -252,6 +260,13 @@ class PacContext:
         self._ck(self._lib.pac_kernel_times(self._h, ms, cnt))
         names = ["down_projection", "chain_head", "dw_down", "finalize"]
         return {n: (ms[i], cnt[i]) for i, n in enumerate(names)}
+
+    def stream_phase_times(self):
+        """(ms_total, launches) of the two cache passes' stream phases (device timestamps) since the last call."""
+        ms = (C.c_double * 2)()
+        cnt = (C.c_longlong * 2)()
+        self._ck(self._lib.pac_stream_phase_times(self._h, ms, cnt))
+        return {"first_pass": (ms[0], cnt[0]), "second_pass": (ms[1], cnt[1])}
 
     def device_buffers(self):
         """Zero-copy torch views (CUDA, fp32) of the context's parameter and gradient vectors."""

@@ -86,6 +86,9 @@ struct pac_ctx {
     int timing = 0;
     std::vector<cudaEvent_t> tev[4];   // start/stop pairs per bracketed kernel group
     size_t tev_used[4] = {0, 0, 0, 0};
+    // device-side stream-phase timestamps (timing == 2): [pass][slot]{earliest first copy, latest accumulator complete}
+    unsigned long long* d_stamps = nullptr;
+    size_t stamps_used[2] = {0, 0};
     bool tensor_ok = false;
     long long launches = 0;
     TensorPlan tplan{};
@@ -172,8 +175,24 @@ void fill_initial_params(const pac_ctx* c, unsigned long long seed, std::vector<
 
 // ---- optional event brackets around the two cache-stream kernels ----
 constexpr size_t MAX_TIMED = 4096;
+constexpr size_t STAMP_SLOTS = 1024;
+// Slot for the next launch of pass `which` (0: first pass over the cache, 1: second), or null.
+unsigned long long* next_stamp(pac_ctx* c, int which) {
+    if (c->timing != 2 || !c->d_stamps || c->stamps_used[which] >= STAMP_SLOTS) return nullptr;
+    return c->d_stamps + ((size_t)which * STAMP_SLOTS + c->stamps_used[which]++) * 2;
+}
+pac_status reset_stamps(pac_ctx* c) {
+    std::vector<unsigned long long> init(2 * STAMP_SLOTS * 2);
+    for (size_t i = 0; i < init.size(); i += 2) { init[i] = ~0ull; init[i + 1] = 0ull; }
+    if (!c->d_stamps) CU_OK(c, cudaMalloc((void**)&c->d_stamps, sizeof(unsigned long long) * init.size()));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    CU_OK(c, cudaMemcpy(c->d_stamps, init.data(), sizeof(unsigned long long) * init.size(), cudaMemcpyHostToDevice));
+    c->stamps_used[0] = c->stamps_used[1] = 0;
+    return PAC_OK;
+}
+
 void time_mark(pac_ctx* c, int which, bool stop) {
-    if (!c->timing) return;
+    if (c->timing != 1) return;
     size_t pair = c->tev_used[which] / 2;
     if (pair >= MAX_TIMED) return;
     if (c->tev[which].size() < 2 * (pair + 1)) {
@@ -375,7 +394,7 @@ pac_status down_projection(pac_ctx* c, const int* d_ids, int B) {
     pac_status st;
     time_mark(c, 0, false);
     if (use_tensor(c)) {
-        st = tensor_down_projection(c->tplan, c->stream, d_ids, B, c->sc.u, c->status, &c->launches);
+        st = tensor_down_projection(c->tplan, c->stream, d_ids, B, c->sc.u, c->status, &c->launches, next_stamp(c, 0));
         if (st != PAC_OK) return fail(c, st, "tensor-core down-projection launch failed: %s", tensor_last_error());
     } else {
         st = c->dtype == PAC_F32 ? down_projection_simt<float>(c, d_ids, B) : down_projection_simt<bf16>(c, d_ids, B);
@@ -390,7 +409,7 @@ pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     time_mark(c, 2, false);
     if (use_tensor(c)) {
         st = tensor_dw_down(c->tplan, c->stream, d_ids, B, c->sc.du16, c->grads + c->lay.w_down, c->sc.dw_part,
-                            reduce_splits, c->status, &c->launches);
+                            reduce_splits, c->status, &c->launches, next_stamp(c, 1));
         if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
     } else {
         st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
@@ -435,6 +454,7 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     fp.mid.layers_per_cta = pl.layers_per_cta;
     fp.mid.u_swz = pl.u_swz;
     fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset;
+    fp.stamp = next_stamp(c, 0);
     cudaError_t e = fused_fwd_launch(pl, c->tplan.map_cache_fwd, c->tplan.map_w, fp, c->cfg.act, c->stream);
     c->launches++;
     if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "fused forward kernel launch failed: %s", cudaGetErrorString(e));
@@ -540,7 +560,7 @@ void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
                     s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.dw_part, c->params, c->grads,
-                    c->m, c->v, c->status, c->d_perm, c->d_losses};
+                    c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->h_ids) cudaFreeHost(c->h_ids);
@@ -754,6 +774,16 @@ pac_status pac_train_step(pac_ctx* c, const int* sample_ids, int B, float* loss_
     return PAC_OK;
 }
 
+pac_status pac_train_step_async(pac_ctx* c, const int* sample_ids, int B, const pac_adamw* hp, float* loss_out) {
+    NEED_INIT(c, "pac_train_step_async");
+    pac_status st = check_hp(c, hp);
+    if (st != PAC_OK) return st;
+    if ((st = stage_ids(c, sample_ids, B, "pac_train_step_async")) != PAC_OK) return st;
+    if ((st = train_enqueue(c, c->sc.ids, B, c->sc.loss, hp)) != PAC_OK) return st;
+    if (loss_out) CU_OK(c, cudaMemcpyAsync(loss_out, c->sc.loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    return PAC_OK;
+}
+
 pac_status pac_adam_step(pac_ctx* c, const pac_adamw* hp) {
     NEED_INIT(c, "pac_adam_step");
     pac_status st = check_hp(c, hp);
@@ -914,11 +944,34 @@ pac_status pac_set_option(pac_ctx* c, int option, int value) {
         return PAC_OK;
     }
     if (option == PAC_OPT_KERNEL_TIMING) {
-        if (value != 0 && value != 1) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: timing must be 0 or 1");
+        if (value < 0 || value > 2) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: timing must be 0, 1 or 2");
+        if (value == 2) {
+            CU_OK(c, cudaSetDevice(c->device));
+            pac_status st = reset_stamps(c);
+            if (st != PAC_OK) return st;
+        }
         c->timing = value;
         return PAC_OK;
     }
     return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: unknown option %d", option);
+}
+
+pac_status pac_stream_phase_times(pac_ctx* c, double* out_ms, long long* out_count) {
+    NEED_CTX(c);
+    if (!out_ms || !out_count) return fail(c, PAC_ERR_INVALID_ARG, "pac_stream_phase_times: NULL argument");
+    out_ms[0] = out_ms[1] = 0.0;
+    out_count[0] = out_count[1] = 0;
+    if (!c->d_stamps) return PAC_OK;
+    CU_OK(c, cudaSetDevice(c->device));
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    std::vector<unsigned long long> h(2 * STAMP_SLOTS * 2);
+    CU_OK(c, cudaMemcpy(h.data(), c->d_stamps, sizeof(unsigned long long) * h.size(), cudaMemcpyDeviceToHost));
+    for (int w = 0; w < 2; ++w)
+        for (size_t i = 0; i < c->stamps_used[w]; ++i) {
+            const unsigned long long t0 = h[((size_t)w * STAMP_SLOTS + i) * 2], t1 = h[((size_t)w * STAMP_SLOTS + i) * 2 + 1];
+            if (t1 > t0) { out_ms[w] += (double)(t1 - t0) * 1e-6; out_count[w]++; }
+        }
+    return reset_stamps(c);
 }
 
 pac_status pac_kernel_times(pac_ctx* c, double* out_ms, long long* out_count) {

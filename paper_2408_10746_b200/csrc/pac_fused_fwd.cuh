@@ -20,6 +20,7 @@ struct FusedFwdParams {
     int k_chunks;              // ceil(d / 64)
     int stages;                // pipeline depth of the GEMM phase
     size_t mid_offset;         // byte offset of the head vectors behind the stage / u-tile region
+    unsigned long long* stamp; // optional stream-phase timestamps (see stamp_begin)
 };
 
 constexpr int FUSED_N = 128;   // MMA N: 64 hi columns | 64 lo columns
@@ -69,6 +70,7 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
         uint32_t it = 0;
         const uint64_t pol = l2_policy_evict_first();
         bool ok = true;
+        if (lane == 0 && n_layers > 0) stamp_begin(fp.stamp);
         for (int l = l_begin; l < l_end && ok; ++l) {
             for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
                 const int s = it % fp.stages;
@@ -109,6 +111,7 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
             if (elect_one()) umma_commit(accf);                   // every accumulator of this CTA is complete ...
             __syncwarp();
             if (mbar_wait_uniform(accf, 0, abort_flag, p.status)) have_sh = 1;    // ... and every load has been consumed
+            if (lane == 0) stamp_end(fp.stamp);
         }
     } else {
         // head operands -> shared memory, then this CTA's slice of the head products; the barrier

@@ -96,6 +96,16 @@ __device__ __forceinline__ bool elect_one() {
     asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xffffffff;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
     return pred != 0;
 }
+// Optional device-side timing of a pass's stream phase: stamp[0] receives the earliest first-copy
+// time over the grid's CTAs, stamp[1] the latest accumulator-complete time (%globaltimer, ns).
+// The host presets {all ones, 0}.  Unlike event brackets this leaves the launch overlap between the
+// kernels of a step untouched.
+__device__ __forceinline__ void stamp_begin(unsigned long long* stamp) {
+    if (stamp) atomicMin(&stamp[0], global_ns());
+}
+__device__ __forceinline__ void stamp_end(unsigned long long* stamp) {
+    if (stamp) atomicMax(&stamp[1], global_ns());
+}
 // After a wait gave up: give copies that are still in flight time to land before the CTA ends.
 __device__ __forceinline__ void drain_after_abort(volatile int* abort_flag) {
     if (*abort_flag)
@@ -207,6 +217,7 @@ struct FwdParams {
     int wide_n;                            // 1: hi and lo blocks form one N = 128*r_blocks MMA, summed in the epilogue
     float* u; long long layer_stride;      // u[l][m][j], layer_stride = max_rows * r
     unsigned* status;
+    unsigned long long* stamp;             // optional stream-phase timestamps (see stamp_begin)
 };
 
 // ---------------------------------------------------------------------------
@@ -261,6 +272,7 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
         // the optimizer state stay L2-resident
         const uint64_t pol = l2_policy_evict_first();
         bool ok = true;
+        if (lane == 0) stamp_begin(p.stamp);
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
             const int sc = t % p.s_chunks, b = (t / p.s_chunks) % p.B, l = t / (p.s_chunks * p.B);
             const int id = (int)safe_id(p.ids, b, p.N, nullptr);
@@ -330,6 +342,7 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
             const uint32_t aph = (tile_n >> 1) & 1;
             if (!mbar_wait_warp(accf0 + 8 * buf, aph, abort_flag, p.status)) break;
             tc_fence_after();
+            if (threadIdx.x == 64 && t + (int)gridDim.x >= n_tiles) stamp_end(p.stamp);      // this CTA's last tile
             const int srow = sc * FWD_ROWS + q * 32 + lane;          // token index inside the sample
             const long long m = (long long)b * p.S + srow;
             float* dst = p.u + (long long)l * p.layer_stride + m * p.r;
@@ -378,6 +391,7 @@ struct BwdParams {
     int tmem_cols;
     float* out;                            // splits == 1: dW_down [L][d][r]; else partials [J][L][d][r]
     unsigned* status;
+    unsigned long long* stamp;             // optional stream-phase timestamps (see stamp_begin)
 };
 
 // ---------------------------------------------------------------------------
@@ -428,6 +442,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     if (warp == 0) {
         uint32_t it = 0;
         const uint64_t pol = l2_policy_evict_first();
+        if (lane == 0 && rt1 > rt0) stamp_begin(p.stamp);
         for (int rt = rt0; rt < rt1; ++rt, ++it) {
             const int sc = rt % p.s_chunks, b = rt / p.s_chunks;
             const int id = (int)safe_id(p.ids, b, p.N, nullptr);
@@ -476,6 +491,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
         if (rt1 > rt0) {
             if (mbar_wait_warp(accf, 0, abort_flag, p.status)) {
                 tc_fence_after();
+                if (threadIdx.x == 64) stamp_end(p.stamp);
                 for (int c = 0; c < p.chunks; ++c) {
                     const int k = col0 + c * 128 + q * 32 + lane;             // column of h = row of dW_down
                     float* dst = p.out + (((long long)j * p.L + l) * p.d + k) * p.r;
@@ -691,9 +707,9 @@ inline pac_status tensor_plan_create(TensorPlan& tp, int device, const bf16* cac
 inline void tensor_plan_destroy(TensorPlan& tp) { tp.ready = false; }
 
 inline pac_status tensor_down_projection(TensorPlan& tp, cudaStream_t stream, const int* d_ids, int B, float* u,
-                                         unsigned* status, long long* launches) {
+                                         unsigned* status, long long* launches, unsigned long long* stamp = nullptr) {
     FwdParams p = tp.fp;
-    p.ids = d_ids; p.B = B; p.u = u; p.status = status;
+    p.ids = d_ids; p.B = B; p.u = u; p.status = status; p.stamp = stamp;
     const int tiles = p.L * B * p.s_chunks;
     const int grid = tiles < tp.sms ? tiles : tp.sms;
     cudaLaunchConfig_t cfg = {};
@@ -715,9 +731,10 @@ inline int tensor_splits(const TensorPlan& tp, int B) {
 // With reduce_splits == false and more than one split the partial sums stay in `part`
 // ([J][L][d][r]) for the caller's own reduction.
 inline pac_status tensor_dw_down(TensorPlan& tp, cudaStream_t stream, const int* d_ids, int B, const bf16* /*du16*/,
-                                 float* dW, float* part, bool reduce_splits, unsigned* status, long long* launches) {
+                                 float* dW, float* part, bool reduce_splits, unsigned* status, long long* launches,
+                                 unsigned long long* stamp = nullptr) {
     BwdParams p = tp.bp;
-    p.ids = d_ids; p.B = B; p.status = status;
+    p.ids = d_ids; p.B = B; p.status = status; p.stamp = stamp;
     const int J = tensor_splits(tp, B);
     p.splits = J;
     p.out = J > 1 ? part : dW;

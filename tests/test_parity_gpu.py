@@ -454,6 +454,42 @@ def test_tensor_path_epoch_equals_step_loop():
     assert sa == sb == 6 and np.array_equal(ma, mb) and np.array_equal(va, vb)
 
 
+@pytest.mark.parametrize("which", ["tensor", "plain_fp32"])
+def test_async_step_equals_step_then_adam(which, tiny):
+    """pac_train_step_async (no wait, loss copied to page-locked host memory) gives the same bits
+    as pac_train_step followed by pac_adam_step, and reports bad arguments at once."""
+    import paper_2408_10746_b200 as pac
+    if which == "tensor":
+        spec = TC_BASE.scaled(N=32, name="tc_async")
+        case = Case(spec, materialize_cpu=False)
+    else:
+        spec, case = TINY, tiny
+    hp = pac.AdamW()
+    n_steps = 12                                   # more than the 8 id-staging slots
+    perm = np.concatenate([pi.epoch_permutation(spec.N, 2, epoch=e) for e in range(4)])[:n_steps * spec.B]
+    a = case.context()
+    a.set_params(pi.random_params(spec, 3))
+    losses = torch.zeros(n_steps, dtype=torch.float32).pin_memory()
+    for i in range(n_steps):
+        a.train_step_async(perm[i * spec.B:(i + 1) * spec.B], hp, losses.data_ptr() + 4 * i)
+    a.sync()
+    b = case.context()
+    b.set_params(pi.random_params(spec, 3))
+    ref = []
+    for i in range(n_steps):
+        ref.append(b.train_step(perm[i * spec.B:(i + 1) * spec.B]))
+        b.adam_step(hp)
+    assert np.array_equal(losses.numpy(), np.array(ref, dtype=np.float32))
+    assert np.array_equal(a.get_params(), b.get_params())
+    assert a.get_opt_state()[2] == n_steps
+    before = a.get_params()
+    with pytest.raises(pac.PacError) as e:
+        a.train_step_async([0, spec.N], hp)
+    assert e.value.status_name == "PAC_ERR_SAMPLE_ID_RANGE"
+    a.sync()
+    assert np.array_equal(a.get_params(), before) and a.get_opt_state()[2] == n_steps
+
+
 def test_device_buffer_views_and_single_rank_data_parallel(tiny):
     """The zero-copy views alias the library's buffers (what an in-place all-reduce needs), and
     the data-parallel wrapper with one rank is the plain trainer."""
