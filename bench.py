@@ -31,15 +31,14 @@ METRIC = "adapter_epoch_samples_per_sec"
 UNIT = "samples/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
 # capture summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES = {"t5_base": {"down_projection": 80058880, "dw_down": 83782912}}
+NCU_TRAFFIC_BYTES = {"t5_base": {"tensor+fused_forward": {"down_projection": 79930368, "dw_down": 84020480},
+                                 "tensor": {"dw_down": 84020480}}}
 
 
 def ncu_traffic(spec, kernel_path, kernel):
-    """DRAM bytes per launch from the committed ncu capture; None for kernels it does not cover
-    (the counters were taken on the separate down-projection kernel, not the one-kernel forward)."""
-    if kernel == "down_projection" and kernel_path != "tensor":
-        return None
-    return (NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]) or {}).get(kernel)
+    """DRAM bytes per launch from the committed ncu capture (profiles/); None for kernels it does
+    not cover."""
+    return ((NCU_TRAFFIC_BYTES.get(spec.name.split("[")[0]) or {}).get(kernel_path) or {}).get(kernel)
 
 
 def load_peaks():
