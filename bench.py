@@ -259,6 +259,73 @@ def run_codec(args):
                       "data": "synthetic", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "results": res}))
 
 
+def run_host_cache(args, spec):
+    """The cache in page-locked host memory, reloaded per minibatch (paper Section V-B, storage cost
+    analysis): whole epochs through pac_train_epoch with host ids in and host losses out.  The reload
+    is bound by the host link, so the roofline is the measured host-to-device copy bandwidth."""
+    import torch
+    import paper_2408_10746_b200 as pac
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    h_cache = torch.empty((spec.N, spec.L, spec.S, spec.d), dtype=torch.bfloat16 if spec.dtype == "bf16" else torch.float32,
+                          pin_memory=True)
+    chunk = max(1, min(spec.N, (1 << 30) // max(1, spec.cache_bytes // spec.N)))
+    for n0 in range(0, spec.N, chunk):                       # generated on the device, kept on the host only
+        ids = list(range(n0, min(spec.N, n0 + chunk)))
+        h_cache[n0:n0 + len(ids)].copy_(pi.cache_samples(spec, 0, ids, dev))
+    h_labels = pi.labels(spec, 0, "cpu").pin_memory()
+    # host-to-device copy bandwidth of this box: 1 GiB page-locked -> device, best of 5
+    src = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+    best = 1e9
+    for _ in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); dst.copy_(src, non_blocking=True); e1.record(); torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    h2d_gbs = (1 << 30) / (best * 1e-3) / 1e9
+    del src, dst
+    stream = torch.cuda.Stream(device=dev)
+    ctx = pac.PacContext(0, stream.cuda_stream)
+    ctx.cache_register_host(h_cache, h_labels)
+    ctx.adapter_init(r=spec.r, n_out=spec.n_out, max_batch=spec.B)
+    hp = pac.AdamW()
+    K, W, B = args.steps, args.warmup, spec.B
+    ids_host = epoch_ids(spec, K)
+    ctx.train_epoch(epoch_ids(spec, W), B, hp, want_losses=False)
+    sampler = ClockSampler(0)
+    launches0 = ctx.launch_count()
+    torch.cuda.synchronize()
+    sampler.start()
+    t0 = time.perf_counter()
+    losses = ctx.train_epoch(ids_host, B, hp)
+    torch.cuda.synchronize()
+    ms = 1e3 * (time.perf_counter() - t0)
+    clocks = sampler.finish()
+    if not np.isfinite(losses).all():
+        raise SystemExit("non-finite loss in the timed region")
+    pass_bytes = B * spec.L * spec.S * spec.d * spec.elem_bytes
+    ach = pass_bytes / (ms * 1e-3 / K) / 1e9
+    value = K * B / (ms * 1e-3)
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": ms / K,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if spec.dtype == "bf16" else "f32",
+           "data": "synthetic",
+           "config": {"workload": workload_name(spec), "cache": "page-locked host memory, reloaded per minibatch into two device "
+                      "staging slots (one copy per sample on a copy stream, overlapped with the previous step)",
+                      "kernel_path": ctx.kernel_path(), "parallelism": "1 GPU"},
+           "clocks": clocks,
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": pass_bytes + 4 * B * (spec.S if spec.head == "lm" else 1),
+                   "d2h_bytes_per_step": 4, "steps": K},
+           "gpu_launches": int(ctx.launch_count() - launches0),
+           "roofline": {"bound": "host_link", "achieved": ach, "peak": h2d_gbs, "unit": "GB/s", "frac": ach / h2d_gbs,
+                        "peak_source": "1 GiB page-locked host-to-device copy timed in this run", "traffic": None,
+                        "algorithmic_bytes_per_step": pass_bytes},
+           "final_loss": float(losses[-1]), "cpu_baseline": None}
+    ctx.close()
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -276,6 +343,8 @@ def main():
                          "the adapter gradients (paper Section V-B)")
     ap.add_argument("--codec", action="store_true",
                     help="measure the block-wise absmax INT8 codec (paper Eq. 1-2) instead of the train step")
+    ap.add_argument("--cache", choices=["device", "host"], default="device",
+                    help="host: keep the cache in page-locked host memory and reload every minibatch (N defaults to 1024)")
     ap.add_argument("--n-samples", type=int, default=0,
                     help="profiling aid: shrink the cache to this many samples (same per-step shapes); "
                          "the JSON line then names the reduced workload")
@@ -289,6 +358,12 @@ def main():
         return run_reference(args, spec)
     if args.codec:
         return run_codec(args)
+    if args.cache == "host":
+        if not args.n_samples:
+            spec = spec.scaled(N=min(spec.N, 1024), name=f"{spec.name}[N={min(spec.N, 1024)}]")
+        if args.steps == 2560:
+            args.steps, args.warmup = 256, 16
+        return run_host_cache(args, spec)
 
     import torch
     import paper_2408_10746_b200 as pac

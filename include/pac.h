@@ -99,6 +99,22 @@ pac_status pac_destroy(pac_ctx* ctx);
 pac_status pac_cache_register(pac_ctx* ctx, const void* dev_cache, int dtype, long long N, int L, int S, int d,
                               const int* dev_labels, int labels_per_sample);
 
+/* The same for a cache that does not fit (or should not occupy) device memory (Section V-B,
+ * storage cost analysis: the cache is kept on storage and reloaded per micro-batch).  host_cache is
+ * HOST memory, [N][L][S][d] of `dtype`, 16-byte aligned; host_labels is HOST int32 memory, [N] or
+ * [N][S]; both borrowed and read-only until pac_destroy.  Page-locked memory (cudaHostAlloc /
+ * cudaHostRegister) lets the reload overlap the computation; pageable memory works but every copy
+ * then waits for the host.  pac_adapter_init allocates two device staging slots of max_batch
+ * samples each (2 * max_batch * L*S*d elements).  Every call that takes host sample ids
+ * (pac_train_step, pac_train_step_async, pac_train_epoch, pac_eval_logits, pac_gather) first copies
+ * the slabs and labels of its ids into a slot, one contiguous copy per sample on a copy stream of
+ * the context's own, and runs the same kernels on the slot; the copies of a step overlap the
+ * kernels of the step before it, and the host runs at most two steps ahead of the copies.  Results
+ * are bit-identical to those on a device-resident cache.  pac_train_epoch_dev (ids on the device)
+ * returns PAC_ERR_UNSUPPORTED in this mode. */
+pac_status pac_cache_register_host(pac_ctx* ctx, const void* host_cache, int dtype, long long N, int L, int S, int d,
+                                   const int* host_labels, int labels_per_sample);
+
 /* Allocates parameters, gradients, AdamW moments and scratch for batches up to
  * cfg->max_batch and fills the parameters from `seed`:
  * W_down ~ N(0, 1/d), lambda = lambda_init, W_up = 0, W_head ~ N(0, 1/d), b_head = 0

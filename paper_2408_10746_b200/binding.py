@@ -22,7 +22,7 @@ STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_S
                 "PAC_ERR_UNSUPPORTED", "PAC_ERR_NOMEM", "PAC_ERR_CUDA", "PAC_ERR_TIMEOUT"]
 
 # every symbol include/pac.h declares
-EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_adapter_init", "pac_train_step", "pac_train_step_async",
+EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_cache_register_host", "pac_adapter_init", "pac_train_step", "pac_train_step_async",
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
            "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_stream_phase_times", "pac_launch_count", "pac_sync", "pac_last_error",
@@ -79,6 +79,7 @@ def load_library() -> C.CDLL:
     sig = {
         "pac_create": [C.POINTER(P), I, P], "pac_destroy": [P],
         "pac_cache_register": [P, P, I, LL, I, I, I, P, I],
+        "pac_cache_register_host": [P, P, I, LL, I, I, I, P, I],
         "pac_adapter_init": [P, C.POINTER(_AdapterCfg), C.c_ulonglong],
         "pac_train_step": [P, P, I, C.POINTER(F)], "pac_train_step_async": [P, P, I, C.POINTER(_AdamW), P], "pac_adam_step": [P, C.POINTER(_AdamW)],
         "pac_eval_logits": [P, P, I, P], "pac_gather": [P, P, I, P],
@@ -165,6 +166,20 @@ class PacContext:
         dt = {torch.float32: PAC_F32, torch.bfloat16: PAC_BF16}[cache.dtype]
         per = 1 if labels.dim() == 1 else labels.shape[1]
         self._ck(self._lib.pac_cache_register(self._h, cache.data_ptr(), dt, N, L, S, d, labels.data_ptr(), per))
+        self._keep += [cache, labels]
+        self.shape = (N, L, S, d)
+        self.cache_dtype = cache.dtype
+
+    def cache_register_host(self, cache, labels):
+        """cache: CPU tensor [N][L][S][d] (float32 or bfloat16), ideally page-locked; labels: CPU int32
+        [N] or [N][S].  The cache stays in host memory; every step reloads its minibatch."""
+        import torch
+        assert not cache.is_cuda and not labels.is_cuda and cache.is_contiguous() and labels.is_contiguous()
+        assert labels.dtype == torch.int32
+        N, L, S, d = cache.shape
+        dt = {torch.float32: PAC_F32, torch.bfloat16: PAC_BF16}[cache.dtype]
+        per = 1 if labels.dim() == 1 else labels.shape[1]
+        self._ck(self._lib.pac_cache_register_host(self._h, cache.data_ptr(), dt, N, L, S, d, labels.data_ptr(), per))
         self._keep += [cache, labels]
         self.shape = (N, L, S, d)
         self.cache_dtype = cache.dtype

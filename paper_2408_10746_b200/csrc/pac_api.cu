@@ -49,6 +49,29 @@ struct Scratch {
     float* dw_part = nullptr;      // split partials of dW_down
 };
 
+// A cache that lives in host memory (Section V-B, storage cost analysis: the cache is kept on
+// storage and reloaded per micro-batch).  The device holds two staging slots of max_batch samples;
+// a step's slabs are copied into a slot by the copy engine on a stream of their own while the step
+// before it computes on the other slot.  The kernels see a slot as a cache of max_batch samples and
+// the ids 0 .. B-1.
+struct HostCache {
+    bool on = false;
+    const unsigned char* host = nullptr;    // [N][L][S][d], host memory (page-locked for asynchronous copies)
+    const int* host_labels = nullptr;       // [N][labels_per_sample], host memory
+    long long N = 0;                        // samples in the host cache
+    long long sample_bytes = 0;             // L * S * d * element size
+    int cur = 0;                            // slot the next step uses
+    unsigned char* stage[2] = {nullptr, nullptr};   // device [max_batch][L][S][d]
+    int* lab_stage[2] = {nullptr, nullptr};         // device [max_batch][labels_per_sample]
+    int* h_lab[2] = {nullptr, nullptr};             // page-locked staging of the labels
+    float* hbar_stage[2] = {nullptr, nullptr};      // device [max_batch][d]
+    int* iota = nullptr;                            // device 0 .. max_batch-1
+    TensorPlan tplan[2];
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ready[2] = {nullptr, nullptr};      // slot filled (copy stream)
+    cudaEvent_t freed[2] = {nullptr, nullptr};      // slot's step enqueued and done (compute stream)
+};
+
 }  // namespace
 
 struct pac_ctx {
@@ -97,6 +120,7 @@ struct pac_ctx {
     int forward_mode = 0;          // 0: one-launch forward when a batch's clusters fit the device at once, 2: never, 3: whenever the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
     bool lm_tensor = false;
+    HostCache hc;                  // out-of-core mode (pac_cache_register_host)
     std::string err;
 };
 
@@ -558,11 +582,22 @@ pac_status refresh_shadow(pac_ctx* c) {
 
 void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
+    if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
                     s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.dw_part, c->params, c->grads,
                     c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
+    for (int k = 0; k < 2; ++k) {
+        if (c->hc.stage[k]) cudaFree(c->hc.stage[k]);
+        if (c->hc.lab_stage[k]) cudaFree(c->hc.lab_stage[k]);
+        if (c->hc.hbar_stage[k]) cudaFree(c->hc.hbar_stage[k]);
+        if (c->hc.h_lab[k]) cudaFreeHost(c->hc.h_lab[k]);
+        if (c->hc.ready[k]) cudaEventDestroy(c->hc.ready[k]);
+        if (c->hc.freed[k]) cudaEventDestroy(c->hc.freed[k]);
+    }
+    if (c->hc.iota) cudaFree(c->hc.iota);
+    if (c->hc.copy_stream) cudaStreamDestroy(c->hc.copy_stream);
     if (c->h_ids) cudaFreeHost(c->h_ids);
     if (c->h_loss) cudaFreeHost(c->h_loss);
     if (c->h_status) cudaFreeHost(c->h_status);
@@ -641,6 +676,22 @@ pac_status pac_cache_register(pac_ctx* c, const void* dev_cache, int dtype, long
     return PAC_OK;
 }
 
+pac_status pac_cache_register_host(pac_ctx* c, const void* host_cache, int dtype, long long N, int L, int S, int d,
+                                   const int* host_labels, int labels_per_sample) {
+    NEED_CTX(c);
+    // same checks as for a device-resident cache; the pointers are host memory here
+    pac_status st = pac_cache_register(c, host_cache, dtype, N, L, S, d, host_labels, labels_per_sample);
+    if (st != PAC_OK) return st;
+    c->hc.on = true;
+    c->hc.host = (const unsigned char*)host_cache;
+    c->hc.host_labels = host_labels;
+    c->hc.N = N;
+    c->hc.sample_bytes = (long long)L * S * d * (dtype == PAC_F32 ? 4 : 2);
+    c->cache = nullptr;                  // bound to a staging slot before every use
+    c->labels = nullptr;
+    return PAC_OK;
+}
+
 pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned long long seed) {
     NEED_CTX(c);
     if (!c->registered) return fail(c, PAC_ERR_BAD_STATE, "pac_adapter_init: call pac_cache_register first");
@@ -658,6 +709,27 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     CU_OK(c, cudaSetDevice(c->device));
     c->cfg = *cfg;
     c->dm.r = cfg->r; c->dm.C = cfg->n_out;
+    if (c->hc.on) {
+        // the kernels see a staging slot: a cache of max_batch samples
+        HostCache& h = c->hc;
+        c->dm.N = cfg->max_batch;
+        const size_t lab_n = (size_t)cfg->max_batch * c->labels_per_sample;
+        CU_OK(c, cudaStreamCreateWithFlags(&h.copy_stream, cudaStreamNonBlocking));
+        for (int k = 0; k < 2; ++k) {
+            CU_OK(c, cudaMalloc((void**)&h.stage[k], (size_t)cfg->max_batch * h.sample_bytes));
+            CU_OK(c, cudaMalloc((void**)&h.lab_stage[k], sizeof(int) * lab_n));
+            CU_OK(c, cudaMalloc((void**)&h.hbar_stage[k], sizeof(float) * (size_t)cfg->max_batch * c->dm.d));
+            CU_OK(c, cudaMallocHost((void**)&h.h_lab[k], sizeof(int) * lab_n));
+            CU_OK(c, cudaEventCreateWithFlags(&h.ready[k], cudaEventDisableTiming));
+            CU_OK(c, cudaEventCreateWithFlags(&h.freed[k], cudaEventDisableTiming));
+        }
+        std::vector<int> iota(cfg->max_batch);
+        for (int b = 0; b < cfg->max_batch; ++b) iota[b] = b;
+        CU_OK(c, cudaMalloc((void**)&h.iota, sizeof(int) * cfg->max_batch));
+        CU_OK(c, cudaMemcpy(h.iota, iota.data(), sizeof(int) * cfg->max_batch, cudaMemcpyHostToDevice));
+        c->cache = h.stage[0];
+        c->labels = h.lab_stage[0];
+    }
     const Dims& dm = c->dm;
     c->lay = ParamLayout::make(dm.L, dm.d, dm.r, dm.C, cls);
     c->max_rows = cfg->max_batch * dm.S;
@@ -683,7 +755,8 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     A(dmalloc(c, &s.lam_part, (long long)dm.L * c->chain_blocks_max));
     A(dmalloc(c, &s.loss, 1));
     if (cls) {
-        A(dmalloc(c, &s.hbar, dm.N * dm.d));
+        if (c->hc.on) s.hbar = c->hc.hbar_stage[0];
+        else A(dmalloc(c, &s.hbar, dm.N * dm.d));
         A(dmalloc(c, &s.pooled_a, (long long)cfg->max_batch * dm.r));
         A(dmalloc(c, &s.pooled_y, (long long)cfg->max_batch * dm.d));
         A(dmalloc(c, &s.logits, (long long)cfg->max_batch * dm.C));
@@ -722,6 +795,12 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
         if (st == PAC_OK) {
             pac_status ts = tensor_plan_create(c->tplan, c->device, (const bf16*)c->cache, dm, cfg->max_batch, s.wdT,
                                                s.du16, &part_floats);
+            if (ts == PAC_OK && c->hc.on) {
+                // one set of tensor maps per staging slot
+                c->hc.tplan[0] = c->tplan;
+                long long pf2 = 0;
+                ts = tensor_plan_create(c->hc.tplan[1], c->device, (const bf16*)c->hc.stage[1], dm, cfg->max_batch, s.wdT, s.du16, &pf2);
+            }
             if (ts == PAC_OK) {
                 A(dmalloc(c, &s.dw_part, part_floats));
                 c->tensor_ok = (st == PAC_OK);
@@ -749,7 +828,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     CU_OK(c, cudaStreamSynchronize(c->stream));
     c->step = 0;
     if ((st = refresh_shadow(c)) != PAC_OK) return st;
-    if (cls) {
+    if (cls && !c->hc.on) {
         if (c->dtype == PAC_F32)
             pool_last_layer_kernel<float><<<(unsigned)dm.N, 256, 0, c->stream>>>((const float*)c->cache, s.hbar, dm.L, dm.S, dm.d);
         else
@@ -761,11 +840,77 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     return PAC_OK;
 }
 
+// ---- out-of-core cache: bring a minibatch's slabs into a staging slot and point the context at it ----
+namespace {
+
+// Validates host ids against the host cache, copies their slabs and labels into the next slot on
+// the copy stream, makes the compute stream wait for them and binds the slot: afterwards the
+// kernels run on ids 0 .. B-1 of a cache of max_batch samples.  *ids_out receives those ids.
+pac_status host_cache_stage(pac_ctx* c, const int* ids, int B, const char* who, const int** ids_out) {
+    HostCache& h = c->hc;
+    if (!ids) return fail(c, PAC_ERR_INVALID_ARG, "%s: sample_ids is NULL", who);
+    if (B < 1 || B > c->cfg.max_batch)
+        return fail(c, PAC_ERR_INVALID_ARG, "%s: B=%d outside [1, max_batch=%d]", who, B, c->cfg.max_batch);
+    for (int b = 0; b < B; ++b)
+        if (ids[b] < 0 || ids[b] >= h.N)
+            return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "%s: sample_ids[%d]=%d outside [0, %lld)", who, b, ids[b], h.N);
+    const int k = h.cur;
+    h.cur ^= 1;
+    const int lps = c->labels_per_sample;
+    // the slot's previous contents: its copies must have run before the label staging is rewritten,
+    // its step must have finished before the slabs are overwritten
+    CU_OK(c, cudaEventSynchronize(h.ready[k]));
+    CU_OK(c, cudaStreamWaitEvent(h.copy_stream, h.freed[k], 0));
+    for (int b = 0; b < B; ++b) {
+        CU_OK(c, cudaMemcpyAsync(h.stage[k] + (size_t)b * h.sample_bytes, h.host + (size_t)ids[b] * h.sample_bytes,
+                                 (size_t)h.sample_bytes, cudaMemcpyHostToDevice, h.copy_stream));
+        std::memcpy(h.h_lab[k] + (size_t)b * lps, h.host_labels + (size_t)ids[b] * lps, sizeof(int) * lps);
+    }
+    CU_OK(c, cudaMemcpyAsync(h.lab_stage[k], h.h_lab[k], sizeof(int) * (size_t)B * lps, cudaMemcpyHostToDevice, h.copy_stream));
+    CU_OK(c, cudaEventRecord(h.ready[k], h.copy_stream));
+    CU_OK(c, cudaStreamWaitEvent(c->stream, h.ready[k], 0));
+    // bind
+    c->cache = h.stage[k];
+    c->labels = h.lab_stage[k];
+    c->sc.hbar = h.hbar_stage[k];
+    if (c->tensor_ok) c->tplan = h.tplan[k];
+    if (c->cfg.head == PAC_HEAD_MEANPOOL_CLS) {
+        // token mean of the last cached layer of the staged samples (computed once at set-up for a resident cache)
+        if (c->dtype == PAC_F32)
+            pool_last_layer_kernel<float><<<(unsigned)B, 256, 0, c->stream>>>((const float*)c->cache, c->sc.hbar, c->dm.L, c->dm.S, c->dm.d);
+        else
+            pool_last_layer_kernel<bf16><<<(unsigned)B, 256, 0, c->stream>>>((const bf16*)c->cache, c->sc.hbar, c->dm.L, c->dm.S, c->dm.d);
+        LAUNCH_CHECK(c);
+    }
+    *ids_out = h.iota;
+    return PAC_OK;
+}
+
+// After the step that uses the bound slot has been enqueued.
+pac_status host_cache_release(pac_ctx* c) {
+    HostCache& h = c->hc;
+    const int k = h.cur ^ 1;               // the slot host_cache_stage bound last
+    CU_OK(c, cudaEventRecord(h.freed[k], c->stream));
+    return PAC_OK;
+}
+
+// Ids of a step, wherever the cache lives: device ids the kernels index the (staged) cache with.
+pac_status prepare_ids(pac_ctx* c, const int* sample_ids, int B, const char* who, const int** d_ids) {
+    if (c->hc.on) return host_cache_stage(c, sample_ids, B, who, d_ids);
+    *d_ids = c->sc.ids;
+    return stage_ids(c, sample_ids, B, who);
+}
+pac_status finish_ids(pac_ctx* c) { return c->hc.on ? host_cache_release(c) : PAC_OK; }
+
+}  // namespace
+
 pac_status pac_train_step(pac_ctx* c, const int* sample_ids, int B, float* loss_out) {
     NEED_INIT(c, "pac_train_step");
-    pac_status st = stage_ids(c, sample_ids, B, "pac_train_step");
+    const int* d_ids = nullptr;
+    pac_status st = prepare_ids(c, sample_ids, B, "pac_train_step", &d_ids);
     if (st != PAC_OK) return st;
-    if ((st = train_enqueue(c, c->sc.ids, B, c->sc.loss, nullptr)) != PAC_OK) return st;
+    if ((st = train_enqueue(c, d_ids, B, c->sc.loss, nullptr)) != PAC_OK) return st;
+    if ((st = finish_ids(c)) != PAC_OK) return st;
     if (loss_out) {
         CU_OK(c, cudaMemcpyAsync(c->h_loss, c->sc.loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
         CU_OK(c, cudaStreamSynchronize(c->stream));
@@ -778,8 +923,10 @@ pac_status pac_train_step_async(pac_ctx* c, const int* sample_ids, int B, const 
     NEED_INIT(c, "pac_train_step_async");
     pac_status st = check_hp(c, hp);
     if (st != PAC_OK) return st;
-    if ((st = stage_ids(c, sample_ids, B, "pac_train_step_async")) != PAC_OK) return st;
-    if ((st = train_enqueue(c, c->sc.ids, B, c->sc.loss, hp)) != PAC_OK) return st;
+    const int* d_ids = nullptr;
+    if ((st = prepare_ids(c, sample_ids, B, "pac_train_step_async", &d_ids)) != PAC_OK) return st;
+    if ((st = train_enqueue(c, d_ids, B, c->sc.loss, hp)) != PAC_OK) return st;
+    if ((st = finish_ids(c)) != PAC_OK) return st;
     if (loss_out) CU_OK(c, cudaMemcpyAsync(loss_out, c->sc.loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
     return PAC_OK;
 }
@@ -794,26 +941,29 @@ pac_status pac_adam_step(pac_ctx* c, const pac_adamw* hp) {
 pac_status pac_eval_logits(pac_ctx* c, const int* sample_ids, int B, float* dev_out) {
     NEED_INIT(c, "pac_eval_logits");
     if (!dev_out) return fail(c, PAC_ERR_INVALID_ARG, "pac_eval_logits: dev_out is NULL");
-    pac_status st = stage_ids(c, sample_ids, B, "pac_eval_logits");
+    const int* d_ids = nullptr;
+    pac_status st = prepare_ids(c, sample_ids, B, "pac_eval_logits", &d_ids);
     if (st != PAC_OK) return st;
-    if (use_fused_cls(c)) return cls_forward_enqueue(c, c->sc.ids, B, false, dev_out);
-    return forward(c, c->sc.ids, B, false, dev_out);
+    st = use_fused_cls(c) ? cls_forward_enqueue(c, d_ids, B, false, dev_out) : forward(c, d_ids, B, false, dev_out);
+    if (st != PAC_OK) return st;
+    return finish_ids(c);
 }
 
 pac_status pac_gather(pac_ctx* c, const int* sample_ids, int B, void* dev_out) {
     NEED_INIT(c, "pac_gather");
     if (!dev_out) return fail(c, PAC_ERR_INVALID_ARG, "pac_gather: dev_out is NULL");
-    pac_status st = stage_ids(c, sample_ids, B, "pac_gather");
+    const int* d_ids = nullptr;
+    pac_status st = prepare_ids(c, sample_ids, B, "pac_gather", &d_ids);
     if (st != PAC_OK) return st;
     const Dims& dm = c->dm;
     const long long slab = (long long)dm.S * dm.d * (c->dtype == PAC_F32 ? 4 : 2);
     const int vec16 = (slab % 16 == 0) && (((uintptr_t)dev_out & 15) == 0);
     unsigned chunks = (unsigned)std::min<long long>(64, std::max<long long>(1, slab / (16 * 256 * 4)));
     dim3 grid((unsigned)(B * dm.L), chunks, 1);
-    gather_kernel<<<grid, 256, 0, c->stream>>>((const unsigned char*)c->cache, c->sc.ids, dm.N, dm.L, B, slab,
+    gather_kernel<<<grid, 256, 0, c->stream>>>((const unsigned char*)c->cache, d_ids, dm.N, dm.L, B, slab,
                                                (unsigned char*)dev_out, vec16, c->status);
     LAUNCH_CHECK(c);
-    return PAC_OK;
+    return finish_ids(c);
 }
 
 static pac_status epoch_common(pac_ctx* c, const int* d_perm, long long n, int B, const pac_adamw* hp, float* d_losses) {
@@ -832,9 +982,30 @@ pac_status pac_train_epoch(pac_ctx* c, const int* perm, long long n, int B, cons
     if (!perm) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch: perm is NULL");
     if (B < 1 || B > c->cfg.max_batch) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch: B=%d outside [1, max_batch]", B);
     if (n < B || n % B != 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch: n=%lld is not a positive multiple of B=%d", n, B);
+    const long long n_cache = c->hc.on ? c->hc.N : c->dm.N;
     for (long long i = 0; i < n; ++i)
-        if (perm[i] < 0 || perm[i] >= c->dm.N)
-            return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "pac_train_epoch: perm[%lld]=%d outside [0, %lld)", i, perm[i], c->dm.N);
+        if (perm[i] < 0 || perm[i] >= n_cache)
+            return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "pac_train_epoch: perm[%lld]=%d outside [0, %lld)", i, perm[i], n_cache);
+    if (c->hc.on && n / B > c->losses_cap) {
+        CU_OK(c, cudaStreamSynchronize(c->stream));
+        if (c->d_losses) cudaFree(c->d_losses);
+        c->d_losses = nullptr; c->losses_cap = 0;
+        if ((st = dmalloc(c, &c->d_losses, n / B)) != PAC_OK) return st;
+        c->losses_cap = n / B;
+    }
+    if (c->hc.on) {
+        // host-resident cache: the slabs of step s+1 travel to their staging slot while step s computes
+        for (long long s = 0; s < n / B; ++s) {
+            const int* d_ids = nullptr;
+            if ((st = host_cache_stage(c, perm + s * B, B, "pac_train_epoch", &d_ids)) != PAC_OK) return st;
+            if ((st = train_enqueue(c, d_ids, B, c->d_losses + s, hp)) != PAC_OK) return st;
+            if ((st = host_cache_release(c)) != PAC_OK) return st;
+        }
+        if (losses_out)
+            CU_OK(c, cudaMemcpyAsync(losses_out, c->d_losses, sizeof(float) * (n / B), cudaMemcpyDeviceToHost, c->stream));
+        CU_OK(c, cudaStreamSynchronize(c->stream));
+        return PAC_OK;
+    }
     if (n > c->perm_cap) {
         CU_OK(c, cudaStreamSynchronize(c->stream));
         if (c->d_perm) cudaFree(c->d_perm);
@@ -862,6 +1033,8 @@ pac_status pac_train_epoch_dev(pac_ctx* c, const int* dev_perm, long long n, int
     NEED_INIT(c, "pac_train_epoch_dev");
     pac_status st = check_hp(c, hp);
     if (st != PAC_OK) return st;
+    if (c->hc.on)
+        return fail(c, PAC_ERR_UNSUPPORTED, "pac_train_epoch_dev: a host-resident cache needs the ids on the host (use pac_train_epoch)");
     if (!dev_perm) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch_dev: dev_perm is NULL");
     if (B < 1 || B > c->cfg.max_batch) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch_dev: B=%d outside [1, max_batch]", B);
     if (n < B || n % B != 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_epoch_dev: n=%lld is not a positive multiple of B=%d", n, B);
