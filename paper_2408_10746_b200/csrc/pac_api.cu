@@ -120,6 +120,8 @@ struct pac_ctx {
     int forward_mode = 0;          // 0: one-launch forward when a batch's clusters fit the device at once, 2: never, 3: whenever the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
     bool lm_tensor = false;
+    int sms = 0;                   // multiprocessors of the device
+    bool lm_ce_stream = false;     // LM cross-entropy as a register-resident stream over the logits (V <= 32768, V % 4 == 0)
     HostCache hc;                  // out-of-core mode (pac_cache_register_host)
     std::string err;
 };
@@ -318,7 +320,13 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
             gemm_simt<<<g2, 256, 0, c->stream>>>(M, dm.C, dm.d, Ay, Bw, El);
             LAUNCH_CHECK(c);
         }
-        if (train) {
+        if (train && c->lm_tensor && c->lm_ce_stream) {
+            // logits read once, dlogits written as bf16: a stream bound by HBM
+            cudaError_t e = lm_ce_stream_launch(c->stream, c->sms, lg, d_ids, dm.N, c->labels, dm.S, dm.C, M, sc.loss_b,
+                                                sc.dlog16, c->status);
+            c->launches++;
+            if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "LM cross-entropy launch failed: %s", cudaGetErrorString(e));
+        } else if (train) {
             lm_ce_kernel<<<M, 256, 0, c->stream>>>(lg, d_ids, dm.N, c->labels, dm.S, dm.C, M, 1, sc.loss_b, c->status,
                                                    c->lm_tensor ? sc.dlog16 : nullptr);
             LAUNCH_CHECK(c);
@@ -631,6 +639,7 @@ pac_status pac_create(pac_ctx** out, int device, void* cuda_stream) {
     pac_ctx* c = new (std::nothrow) pac_ctx();
     if (!c) return PAC_ERR_NOMEM;
     c->device = device;
+    if (cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->sms < 1) c->sms = 1;
     if (cuda_stream) {
         c->stream = (cudaStream_t)cuda_stream;
     } else {
@@ -777,7 +786,12 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             if (st == PAC_OK) {
                 pac_status g1 = gemm_plan_create(c->g_logits, c->device, s.y16, c->max_rows, (const bf16*)cfg->lm_head, dm.C, dm.d, 0);
                 pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_dy, c->device, s.dlog16, c->max_rows, (const bf16*)cfg->lm_head, dm.d, dm.C, 1) : g1;
-                if (g1 == PAC_OK && g2 == PAC_OK) c->lm_tensor = true;
+                if (g1 == PAC_OK && g2 == PAC_OK) {
+                    c->lm_tensor = true;
+                    int max_smem = 0;
+                    c->lm_ce_stream = cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) == cudaSuccess &&
+                                      lm_ce_stream_supported(dm.C, max_smem);
+                }
                 else if ((g1 != PAC_OK && g1 != PAC_ERR_UNSUPPORTED) || (g2 != PAC_OK && g2 != PAC_ERR_UNSUPPORTED))
                     st = fail(c, PAC_ERR_CUDA, "LM-head GEMM set-up failed: %s", tensor_last_error());
             }

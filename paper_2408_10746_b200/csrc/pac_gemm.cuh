@@ -152,6 +152,125 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 1) tmem_dealloc(tmem_base, 512u);
 }
 
+// ---------------------------------------------------------------------------
+// Cross-entropy of the LM head as a stream over the logits: rows of [M][V] fp32 in, loss per row
+// and dlogits = (softmax - onehot) / M as bf16 out (the A operand of dy = dlogits W_lm).
+// Persistent CTAs of 512 threads, one row at a time: the row (V <= 32768, V % 4 == 0) is held in
+// registers, 16 float4 per thread, while the NEXT row is already on its way into shared memory
+// as bulk asynchronous copies, so the logits are read from HBM exactly once and the read of one
+// row overlaps the arithmetic and the write of the row before it.  All sums have a fixed order.
+// ---------------------------------------------------------------------------
+constexpr int CE_THREADS = 512, CE_V4_PER_THREAD = 16, CE_MAX_V = CE_THREADS * CE_V4_PER_THREAD * 4;
+constexpr uint32_t CE_COPY_BYTES = 32768;                 // size of one bulk copy
+
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(CE_THREADS, 1)
+lm_ce_stream_kernel(const float* __restrict__ logits, const int* __restrict__ ids, long long N, const int* __restrict__ targets,
+                    int S, int V, int M, float* __restrict__ loss_row, bf16* __restrict__ dlog16, unsigned* status) {
+    extern __shared__ __align__(128) unsigned char ce_smem[];
+    float4* row_s = reinterpret_cast<float4*>(ce_smem);
+    __shared__ __align__(8) unsigned long long bar_sh;
+    __shared__ float red[32];
+    __shared__ int abort_sh;
+    const uint32_t bar = smem_u32(&bar_sh);
+    const int t = threadIdx.x;
+    const uint32_t row_bytes = (uint32_t)V * 4u;
+    const int n4 = V >> 2;
+    volatile int* abort_flag = &abort_sh;
+    if (t == 0) {
+        abort_sh = 0;
+        mbar_init(bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    auto issue = [&](int m) {                              // thread 0: the whole row as 32 KB pieces
+        mbar_expect_tx(bar, row_bytes);
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(logits + (long long)m * V);
+        for (uint32_t off = 0; off < row_bytes; off += CE_COPY_BYTES)
+            bulk_load_1d(smem_u32(ce_smem) + off, src + off, min(CE_COPY_BYTES, row_bytes - off), bar);
+    };
+    int m = blockIdx.x;
+    if (t == 0 && m < M) issue(m);
+    uint32_t phase = 0;
+    for (; m < M; m += gridDim.x, phase ^= 1) {
+        // the row has landed -> registers; then the buffer is free for the next row
+        int ok = 1;
+        if ((t & 31) == 0) ok = mbar_wait(bar, phase, abort_flag, status) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!__syncthreads_and(ok)) break;
+        float4 v[CE_V4_PER_THREAD];
+#pragma unroll
+        for (int i = 0; i < CE_V4_PER_THREAD; ++i) {
+            const int e = i * CE_THREADS + t;
+            v[i] = e < n4 ? row_s[e] : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        }
+        __syncthreads();
+        const int m_next = m + gridDim.x;
+        if (t == 0 && m_next < M) { fence_proxy_async(); issue(m_next); }
+
+        const int b = m / S, s = m - b * S;
+        const long long id = safe_id(ids, b, N, (t == 0 && s == 0) ? status : nullptr);
+        const int tgt = targets[id * S + s];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < CE_V4_PER_THREAD; ++i) mx = fmaxf(mx, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+        mx = block_max(mx, red);
+        float se = 0.f, tl = 0.f;                          // sum of exponentials; the target's logit (one thread has it)
+#pragma unroll
+        for (int i = 0; i < CE_V4_PER_THREAD; ++i) {
+            const int e0 = (i * CE_THREADS + t) * 4;
+            if (tgt >= e0 && tgt < e0 + 4) tl = tgt == e0 ? v[i].x : tgt == e0 + 1 ? v[i].y : tgt == e0 + 2 ? v[i].z : v[i].w;
+            v[i].x = expf(v[i].x - mx); v[i].y = expf(v[i].y - mx); v[i].z = expf(v[i].z - mx); v[i].w = expf(v[i].w - mx);
+            se += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+        }
+        se = block_sum(se, red);
+        tl = block_sum(tl, red);                           // every other thread contributes 0
+        if (t == 0) loss_row[m] = mx + logf(se) - tl;
+        if (dlog16) {
+            const float inv = 1.f / se, invM = 1.f / (float)M;
+            bf16* out = dlog16 + (long long)m * V;
+#pragma unroll
+            for (int i = 0; i < CE_V4_PER_THREAD; ++i) {
+                const int e = i * CE_THREADS + t, e0 = e * 4;
+                if (e < n4) {
+                    const float g0 = (v[i].x * inv - (tgt == e0 ? 1.f : 0.f)) * invM, g1 = (v[i].y * inv - (tgt == e0 + 1 ? 1.f : 0.f)) * invM;
+                    const float g2 = (v[i].z * inv - (tgt == e0 + 2 ? 1.f : 0.f)) * invM, g3 = (v[i].w * inv - (tgt == e0 + 3 ? 1.f : 0.f)) * invM;
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(g0, g1), hi = __floats2bfloat162_rn(g2, g3);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<unsigned*>(&lo);
+                    pk.y = *reinterpret_cast<unsigned*>(&hi);
+                    *reinterpret_cast<uint2*>(out + e0) = pk;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    drain_after_abort(abort_flag);
+}
+
+inline bool lm_ce_stream_supported(int V, int max_smem) {
+    return V % 4 == 0 && V <= CE_MAX_V && (size_t)V * 4 + 1024 <= (size_t)max_smem;
+}
+
+// rows [M][V] fp32 -> loss_row [M], dlog16 [M][V] (may be null: loss only)
+inline cudaError_t lm_ce_stream_launch(cudaStream_t stream, int sms, const float* logits, const int* ids, long long N,
+                                       const int* targets, int S, int V, int M, float* loss_row, bf16* dlog16, unsigned* status) {
+    static size_t opted_in = 0;
+    const size_t smem = (size_t)V * 4;
+    if (smem > opted_in) {
+        cudaError_t e = cudaFuncSetAttribute(lm_ce_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        opted_in = smem;
+    }
+    const int grid = M < sms ? M : sms;
+    lm_ce_stream_kernel<<<grid, CE_THREADS, smem, stream>>>(logits, ids, N, targets, S, V, M, loss_row, dlog16, status);
+    return cudaGetLastError();
+}
+
 // Host side: tensor maps and launch for one GEMM shape.
 struct GemmPlan {
     bool ready = false;
