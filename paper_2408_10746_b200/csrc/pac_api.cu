@@ -19,6 +19,7 @@ using namespace pac;
 namespace {
 
 constexpr int STAGE_SLOTS = 8;
+constexpr int LM_MAX_K_SLICES = 8;
 
 struct Scratch {
     // per-step state, sized for max_batch
@@ -46,6 +47,7 @@ struct Scratch {
     bf16* dlog16 = nullptr;        // [M][V] bf16 dlogits (tensor-core LM head)
     // tensor path
     bf16* wdT = nullptr;           // [L][2][d][r] bf16 hi/lo shadow of W_down
+    float* lm_part = nullptr;      // [slices][...] partial sums of the LM path's two skinny products (dW_up, da_L)
     float* dw_part = nullptr;      // split partials of dW_down
 };
 
@@ -379,19 +381,49 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
             gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.C, Ad, Bw, Ed);
             LAUNCH_CHECK(c);
         }
+        // Both products below have few output tiles and a long reduction: the reduction is cut into
+        // slices when that fills the device (partial sums added in slice order).
+        auto k_slices = [&](long long tiles, int K, long long out_elems) {
+            if (!sc.lm_part || out_elems % 4 != 0) return 1;
+            long long s = (2LL * c->sms + tiles - 1) / tiles;
+            s = std::min<long long>(s, std::min<long long>(LM_MAX_K_SLICES, K / 256));
+            return (int)std::max<long long>(1, s);
+        };
         // dW_up = a_L^T dy
         dim3 g2(cdiv(dm.d, SG_BN), cdiv(dm.r, SG_BM), 1);
         MatA_ColMajor At{{aL, 0, dm.r}};
         MatB_RowMajor Bd{{sc.dy, 0, dm.d}};
-        StoreRowMajor Eu{c->grads + c->lay.w_up, 0, dm.d};
-        gemm_simt<<<g2, 256, 0, c->stream>>>(dm.r, dm.d, M, At, Bd, Eu);
+        const int s2 = k_slices((long long)g2.x * g2.y, M, (long long)dm.r * dm.d);
+        if (s2 > 1) {
+            const int k_slice = (int)cdiv(cdiv(M, s2), SG_BK) * SG_BK;
+            g2.z = cdiv(M, k_slice);
+            gemm_simt_ksplit<<<g2, 256, 0, c->stream>>>(dm.r, dm.d, M, k_slice, At, Bd, sc.lm_part);
+            LAUNCH_CHECK(c);
+            const long long ne = (long long)dm.r * dm.d;
+            reduce_splits_kernel<<<cdiv(ne / 4, 256), 256, 0, c->stream>>>(sc.lm_part, (int)g2.z, ne, c->grads + c->lay.w_up);
+            c->launches++;
+        } else {
+            StoreRowMajor Eu{c->grads + c->lay.w_up, 0, dm.d};
+            gemm_simt<<<g2, 256, 0, c->stream>>>(dm.r, dm.d, M, At, Bd, Eu);
+        }
         LAUNCH_CHECK(c);
         // da_L = dy W_up^T
         dim3 g3(cdiv(dm.r, SG_BN), cdiv(M, SG_BM), 1);
         MatA_RowMajor Ady{{sc.dy, 0, dm.d}};
         MatB_ColMajor But{{W_up, 0, dm.d}};
-        StoreRowMajor Ea{sc.daL, 0, dm.r};
-        gemm_simt<<<g3, 256, 0, c->stream>>>(M, dm.r, dm.d, Ady, But, Ea);
+        const int s3 = k_slices((long long)g3.x * g3.y, dm.d, (long long)M * dm.r);
+        if (s3 > 1) {
+            const int k_slice = (int)cdiv(cdiv(dm.d, s3), SG_BK) * SG_BK;
+            g3.z = cdiv(dm.d, k_slice);
+            gemm_simt_ksplit<<<g3, 256, 0, c->stream>>>(M, dm.r, dm.d, k_slice, Ady, But, sc.lm_part);
+            LAUNCH_CHECK(c);
+            const long long ne = (long long)M * dm.r;
+            reduce_splits_kernel<<<cdiv(ne / 4, 256), 256, 0, c->stream>>>(sc.lm_part, (int)g3.z, ne, sc.daL);
+            c->launches++;
+        } else {
+            StoreRowMajor Ea{sc.daL, 0, dm.r};
+            gemm_simt<<<g3, 256, 0, c->stream>>>(M, dm.r, dm.d, Ady, But, Ea);
+        }
         LAUNCH_CHECK(c);
         per_sample = 0;
     }
@@ -592,7 +624,7 @@ void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
-                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.dw_part, c->params, c->grads,
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.lm_part, s.dw_part, c->params, c->grads,
                     c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -778,6 +810,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
         A(dmalloc(c, &s.daL, Mr));
         A(dmalloc(c, &s.lm_logits, (long long)c->max_rows * dm.C));
         A(dmalloc(c, &s.dy, (long long)c->max_rows * dm.d));
+        A(dmalloc(c, &s.lm_part, LM_MAX_K_SLICES * std::max((long long)dm.r * dm.d, Mr)));
         // the two dense LM-head GEMMs go to the tensor cores for bf16 caches with 16-byte operand rows
         c->lm_tensor = false;
         if (st == PAC_OK && c->dtype == PAC_BF16 && !c->force_simt && dm.d % 8 == 0 && dm.C % 8 == 0) {

@@ -40,25 +40,22 @@ __global__ void gather_kernel(const unsigned char* __restrict__ cache, const int
 // ---------------------------------------------------------------------------
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16;
 
-template <class AF, class BF, class EF>
-__global__ void __launch_bounds__(256) gemm_simt(int M, int N, int K, AF A, BF B, EF E) {
-    __shared__ float As[SG_BK][SG_BM + 4];
-    __shared__ float Bs[SG_BK][SG_BN + 4];
-    const int z = blockIdx.z;
-    const int i0 = blockIdx.y * SG_BM, j0 = blockIdx.x * SG_BN;
+// The k loop of one 64x64 output tile over [k_begin, k_end): 4x4 partial sums per thread.
+template <class AF, class BF>
+__device__ __forceinline__ void gemm_simt_tile(int M, int N, int K, int k_begin, int k_end, const AF& A, const BF& B, int z,
+                                               int i0, int j0, float (&acc)[4][4], float (*As)[SG_BM + 4], float (*Bs)[SG_BN + 4]) {
     const int t = threadIdx.x, ty = t / 16, tx = t % 16;
-    float acc[4][4] = {};
-    for (int k0 = 0; k0 < K; k0 += SG_BK) {
+    for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             int i, k;
             if (AF::k_contiguous) { k = t % 16; i = t / 16 + 16 * q; } else { i = t % 64; k = t / 64 + 4 * q; }
             int gi = i0 + i, gk = k0 + k;
-            As[k][i] = (gi < M && gk < K) ? A(z, gi, gk) : 0.f;
+            As[k][i] = (gi < M && gk < k_end && gk < K) ? A(z, gi, gk) : 0.f;
             int j;
             if (BF::k_contiguous) { k = t % 16; j = t / 16 + 16 * q; } else { j = t % 64; k = t / 64 + 4 * q; }
             int gj = j0 + j; gk = k0 + k;
-            Bs[k][j] = (gj < N && gk < K) ? B(z, gk, gj) : 0.f;
+            Bs[k][j] = (gj < N && gk < k_end && gk < K) ? B(z, gk, gj) : 0.f;
         }
         __syncthreads();
 #pragma unroll
@@ -73,12 +70,46 @@ __global__ void __launch_bounds__(256) gemm_simt(int M, int N, int K, AF A, BF B
         }
         __syncthreads();
     }
+}
+
+template <class AF, class BF, class EF>
+__global__ void __launch_bounds__(256) gemm_simt(int M, int N, int K, AF A, BF B, EF E) {
+    __shared__ float As[SG_BK][SG_BM + 4];
+    __shared__ float Bs[SG_BK][SG_BN + 4];
+    const int z = blockIdx.z;
+    const int i0 = blockIdx.y * SG_BM, j0 = blockIdx.x * SG_BN;
+    const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+    float acc[4][4] = {};
+    gemm_simt_tile(M, N, K, 0, K, A, B, z, i0, j0, acc, As, Bs);
 #pragma unroll
     for (int p = 0; p < 4; ++p)
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             int gi = i0 + ty * 4 + p, gj = j0 + tx * 4 + q;
             if (gi < M && gj < N) E(z, gi, gj, acc[p][q]);
+        }
+}
+
+// The same product with the k range cut into gridDim.z slices (a multiple of 16 each) for shapes
+// with few output tiles and a long reduction: slice s writes its partial sums to part[s][M][N];
+// the caller adds the slices up in slice order (reduce_splits_kernel), so the result is still
+// independent of timing.
+template <class AF, class BF>
+__global__ void __launch_bounds__(256) gemm_simt_ksplit(int M, int N, int K, int k_slice, AF A, BF B, float* __restrict__ part) {
+    __shared__ float As[SG_BK][SG_BM + 4];
+    __shared__ float Bs[SG_BK][SG_BN + 4];
+    const int i0 = blockIdx.y * SG_BM, j0 = blockIdx.x * SG_BN;
+    const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+    const int k_begin = blockIdx.z * k_slice, k_end = min(K, k_begin + k_slice);
+    float acc[4][4] = {};
+    gemm_simt_tile(M, N, K, k_begin, k_end, A, B, 0, i0, j0, acc, As, Bs);
+    float* out = part + (long long)blockIdx.z * M * N;
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int gi = i0 + ty * 4 + p, gj = j0 + tx * 4 + q;
+            if (gi < M && gj < N) out[(long long)gi * N + gj] = acc[p][q];
         }
 }
 
