@@ -496,6 +496,13 @@ def main():
             avg = tot_ms / cnt
             phases[name] = {"avg_ms": avg, "launches": cnt, "gbs": pass_bytes / (avg * 1e-3) / 1e9,
                             "frac": pass_bytes / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    if spec.head == "lm":
+        # the two dense contractions of the frozen LM head: tensor-core bound
+        gemm_flop = 2.0 * B * spec.S * spec.n_out * spec.d
+        for old, new in (("chain_head", "lm_logits_gemm"), ("finalize", "lm_dy_gemm")):
+            if old in kern:
+                kern[new] = kern.pop(old)
+                kern[new]["tflops"] = gemm_flop / (kern[new]["avg_ms"] * 1e-3) / 1e12
     stream_k = [k for k in kern if "gbs" in kern[k]]
     dominant = max(stream_k, key=lambda k: kern[k]["avg_ms"]) if stream_k else None
     roofline = None
@@ -508,6 +515,20 @@ def main():
                     # first cache copy issued -> last accumulator complete, over all CTAs of a launch (device
                     # timestamps): the part of each pass that streams the minibatch's slabs
                     "stream_phase": phases}
+    gemm_k = [k for k in kern if "tflops" in kern[k]]
+    if gemm_k and max(kern[k]["avg_ms"] for k in gemm_k) > (kern[dominant]["avg_ms"] if dominant else 0.0):
+        # the dominant kernel is a dense contraction: report it against the measured bf16 GEMM peak
+        # (the sustained figure: the kernel runs inside a long step)
+        gk = max(gemm_k, key=lambda k: kern[k]["avg_ms"])
+        tf_peak, tf_src = 1400.0, "fallback"
+        try:
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                tf_peak, tf_src = float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+        except Exception:
+            pass
+        roofline = {"bound": "tensor", "kernel": gk, "achieved": kern[gk]["tflops"], "peak": tf_peak, "unit": "TFLOP/s",
+                    "frac": kern[gk]["tflops"] / tf_peak, "peak_source": tf_src, "traffic": None,
+                    "flop_per_launch": 2.0 * B * spec.S * spec.n_out * spec.d, "kernels": kern, "stream_phase": phases}
     step_s = ms * 1e-3 / K
     stream_gbs = 2 * pass_bytes / step_s / 1e9
 

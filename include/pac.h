@@ -192,7 +192,9 @@ pac_status pac_set_option(pac_ctx* ctx, int option, int value);
  *   [2] dW_down = h_l^T du_l over all layers (second pass over the cache)
  *   [3] gradient finalisation (+ AdamW when fused into the step)
  * When the forward half runs as one kernel (pac_kernel_path() == "tensor+fused_forward") that
- * kernel is counted in group [0] and group [1] stays empty.
+ * kernel is counted in group [0] and group [1] stays empty.  With the frozen LM head on the tensor
+ * cores, group [1] is the logits GEMM (logits = y W_lm^T) and group [3] the dy GEMM
+ * (dy = dlogits W_lm), each 2*B*S*V*d flop.
  * This call waits for the stream, then stores the summed milliseconds and the number of
  * bracketed launches since the last call in out_ms[4] and out_count[4] (host arrays).
  * At most 4096 brackets per group are kept between two calls. */

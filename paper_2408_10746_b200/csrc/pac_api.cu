@@ -312,7 +312,9 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
         // logits = y W_lm^T
         float* lg = train ? sc.lm_logits : d_logits_out;
         if (c->lm_tensor) {
+            time_mark(c, 1, false);
             st = gemm_launch(c->g_logits, c->stream, M, lg, dm.C, c->status, &c->launches);
+            time_mark(c, 1, true);
             if (st != PAC_OK) return fail(c, st, "tensor-core logits GEMM launch failed: %s", tensor_last_error());
         } else {
             dim3 g2(cdiv(dm.C, SG_BN), cdiv(M, SG_BM), 1);
@@ -371,7 +373,9 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
         LAUNCH_CHECK(c);
         // dy = dlogits W_lm   (the head is frozen: it receives no gradient)
         if (c->lm_tensor) {
+            time_mark(c, 3, false);
             pac_status gs = gemm_launch(c->g_dy, c->stream, M, sc.dy, dm.d, c->status, &c->launches);
+            time_mark(c, 3, true);
             if (gs != PAC_OK) return fail(c, gs, "tensor-core dy GEMM launch failed: %s", tensor_last_error());
         } else {
             dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
