@@ -456,6 +456,7 @@ def main():
         for i in range(Ke):
             ctx.train_step_async(ids_view[i * B:(i + 1) * B], hp, loss_ptr + 4 * i)
         e1.record(stream)
+    enqueue_ms = 1e3 * (time.perf_counter() - t0)           # host time to enqueue the Ke steps
     ctx.sync()
     barrier()
     wall_ms = 1e3 * (time.perf_counter() - t0)
@@ -542,7 +543,7 @@ def main():
                    "notes": note},
         "clocks": clocks,
         "e2e": {"value": world * Ke * B / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * B,
-                "d2h_bytes_per_step": 4, "steps": Ke},
+                "d2h_bytes_per_step": 4, "steps": Ke, "host_enqueue_us_per_step": 1e3 * enqueue_ms / Ke},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "cache_stream": {"gbs_two_reads": stream_gbs, "frac_of_peak": stream_gbs / peaks["hbm_gbs"],

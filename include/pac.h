@@ -132,10 +132,13 @@ pac_status pac_train_step(pac_ctx* ctx, const int* sample_ids, int B, float* los
 
 /* One whole training step without waiting: pac_train_step on sample_ids (host, B ints) followed by
  * the AdamW update of pac_adam_step with `hp`, all enqueued on the context's stream; the call
- * returns as soon as that is done (it waits only when more than 8 earlier steps' ids are still in
- * flight).  If loss_out is non-NULL the step's mean loss is copied there once the step has run:
- * loss_out is HOST memory that must stay valid until the next pac_sync (page-locked memory keeps
- * the copy asynchronous); read it after pac_sync.  Errors of the arguments are reported at once,
+ * returns as soon as that is done (it waits only when too many earlier steps' ids are still in
+ * flight: 8, or 32 to 64 with the one-launch forward).  If loss_out is non-NULL the step's mean loss
+ * arrives there once the step has run: loss_out is HOST memory that must stay valid until the next
+ * pac_sync; read it after pac_sync.  Page-locked memory (cudaHostAlloc / cudaHostRegister) is written
+ * by the last kernel of the step itself; other memory gets a copy behind the step.  With the one-launch
+ * forward the ids are likewise read by the kernel from a page-locked ring inside the library, so a
+ * step is three kernels back to back and consecutive steps overlap as in pac_train_epoch_dev.  Errors of the arguments are reported at once,
  * device-side errors by the next pac_sync.  The step a caller loops over when the minibatches
  * are chosen on the host one at a time (Section IV-B: from the second epoch on a step needs
  * nothing but the cached activations of its samples). */

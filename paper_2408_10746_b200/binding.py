@@ -205,8 +205,11 @@ class PacContext:
         """Enqueues one whole step (forward, backward, AdamW) and returns at once.  loss_out_ptr: address
         of one host float (page-locked for a truly asynchronous copy) that receives the loss, or 0."""
         ids = _ids(sample_ids)
-        self._ck(self._lib.pac_train_step_async(self._h, ids.ctypes.data, ids.size, C.byref(hp._c()),
-                                                C.c_void_p(loss_out_ptr) if loss_out_ptr else None))
+        if getattr(self, "_hp_src", None) is not hp:                   # marshal the hyper-parameters once per object
+            self._hp_src, self._hp_c = hp, hp._c()
+        st = self._lib.pac_train_step_async(self._h, ids.ctypes.data, ids.size, self._hp_c, loss_out_ptr or None)
+        if st != 0:
+            self._ck(st)
 
     def adam_step(self, hp: AdamW):
         self._ck(self._lib.pac_adam_step(self._h, C.byref(hp._c())))

@@ -20,6 +20,7 @@ namespace {
 
 constexpr int STAGE_SLOTS = 8;
 constexpr int LM_MAX_K_SLICES = 8;
+constexpr int ZC_SLOTS = 64;
 
 struct Scratch {
     // per-step state, sized for max_batch
@@ -125,6 +126,12 @@ struct pac_ctx {
     int sms = 0;                   // multiprocessors of the device
     bool lm_ce_stream = false;     // LM cross-entropy as a register-resident stream over the logits (V <= 32768, V % 4 == 0)
     HostCache hc;                  // out-of-core mode (pac_cache_register_host)
+    // pac_train_step_async without copy nodes in the stream: a ring of id slots in page-locked host memory that
+    // the forward kernel reads directly (two halves, an event per half orders the reuse)
+    int* zc_ids = nullptr;         // [ZC_SLOTS][max_batch]
+    cudaEvent_t zc_ev[2] = {nullptr, nullptr};
+    unsigned long long zc_count = 0;
+    bool step_host_ids = false;    // the step being enqueued reads its ids from the ring
     std::string err;
 };
 
@@ -520,6 +527,7 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     fp.mid = mid_params(c, pl.mp, d_ids, B, train, d_logits_out);
     fp.mid.u = nullptr;
     fp.mid.layers_per_cta = pl.layers_per_cta;
+    if (c->step_host_ids) { fp.mid.host_ids = 1; fp.mid.ids_copy = c->sc.ids; }
     fp.mid.u_swz = pl.u_swz;
     fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset;
     fp.stamp = next_stamp(c, 0);
@@ -584,6 +592,7 @@ pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, con
     pac_status st;
     if (use_fused_cls(c)) {
         if ((st = cls_forward_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
+        if (c->step_host_ids) d_ids = c->sc.ids;          // the forward kernel left a device copy for the later kernels
         if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
         time_mark(c, 3, false);
         st = finalize_enqueue(c, B, d_loss, hp);
@@ -642,6 +651,9 @@ void free_all(pac_ctx* c) {
     }
     if (c->hc.iota) cudaFree(c->hc.iota);
     if (c->hc.copy_stream) cudaStreamDestroy(c->hc.copy_stream);
+    if (c->zc_ids) cudaFreeHost(c->zc_ids);
+    for (auto& e : c->zc_ev)
+        if (e) cudaEventDestroy(e);
     if (c->h_ids) cudaFreeHost(c->h_ids);
     if (c->h_loss) cudaFreeHost(c->h_loss);
     if (c->h_status) cudaFreeHost(c->h_status);
@@ -837,6 +849,13 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     }
     if (st == PAC_OK && cudaMallocHost((void**)&c->h_ids, sizeof(int) * STAGE_SLOTS * cfg->max_batch) != cudaSuccess)
         st = fail(c, PAC_ERR_NOMEM, "pinned id staging allocation failed");
+    if (st == PAC_OK && fwd_plan.ok) {
+        // id ring of pac_train_step_async (only the one-launch forward reads ids from host memory)
+        if (cudaMallocHost((void**)&c->zc_ids, sizeof(int) * ZC_SLOTS * cfg->max_batch) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->zc_ev[0], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->zc_ev[1], cudaEventDisableTiming) != cudaSuccess)
+            st = fail(c, PAC_ERR_NOMEM, "pinned id ring allocation failed");
+    }
     // tensor-core path: bf16 cache with TMA/UMMA-compatible sizes
     c->tensor_ok = false;
     if (st == PAC_OK && c->dtype == PAC_BF16 && tensor_shape_supported(dm)) {
@@ -974,11 +993,44 @@ pac_status pac_train_step_async(pac_ctx* c, const int* sample_ids, int B, const 
     NEED_INIT(c, "pac_train_step_async");
     pac_status st = check_hp(c, hp);
     if (st != PAC_OK) return st;
+    // where the device can write the loss itself (page-locked host memory): no copy node behind the step
+    float* d_loss = c->sc.loss;
+    bool copy_loss = loss_out != nullptr;
+    if (loss_out) {
+        cudaPointerAttributes pa;
+        if (cudaPointerGetAttributes(&pa, loss_out) == cudaSuccess && pa.type == cudaMemoryTypeHost && pa.devicePointer) {
+            d_loss = (float*)pa.devicePointer;
+            copy_loss = false;
+        } else {
+            cudaGetLastError();
+        }
+    }
     const int* d_ids = nullptr;
-    if ((st = prepare_ids(c, sample_ids, B, "pac_train_step_async", &d_ids)) != PAC_OK) return st;
-    if ((st = train_enqueue(c, d_ids, B, c->sc.loss, hp)) != PAC_OK) return st;
-    if ((st = finish_ids(c)) != PAC_OK) return st;
-    if (loss_out) CU_OK(c, cudaMemcpyAsync(loss_out, c->sc.loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    if (!c->hc.on && c->zc_ids && c->timing == 0 && use_fused_fwd(c, B)) {
+        // one-launch forward: it reads the ids straight from a page-locked ring slot, so the step is three
+        // kernels back to back with nothing between them and the steps overlap as in pac_train_epoch_dev
+        if (!sample_ids) return fail(c, PAC_ERR_INVALID_ARG, "pac_train_step_async: sample_ids is NULL");
+        if (B < 1 || B > c->cfg.max_batch)
+            return fail(c, PAC_ERR_INVALID_ARG, "pac_train_step_async: B=%d outside [1, max_batch=%d]", B, c->cfg.max_batch);
+        for (int b = 0; b < B; ++b)
+            if (sample_ids[b] < 0 || sample_ids[b] >= c->dm.N)
+                return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "pac_train_step_async: sample_ids[%d]=%d outside [0, %lld)", b, sample_ids[b], c->dm.N);
+        const int slot = (int)(c->zc_count % ZC_SLOTS), half = slot / (ZC_SLOTS / 2);
+        if (slot % (ZC_SLOTS / 2) == 0) CU_OK(c, cudaEventSynchronize(c->zc_ev[half]));     // the half's previous steps have run
+        int* h = c->zc_ids + (size_t)slot * c->cfg.max_batch;
+        std::memcpy(h, sample_ids, sizeof(int) * B);
+        c->step_host_ids = true;
+        st = train_enqueue(c, h, B, d_loss, hp);
+        c->step_host_ids = false;
+        if (st != PAC_OK) return st;
+        c->zc_count++;
+        if (slot % (ZC_SLOTS / 2) == ZC_SLOTS / 2 - 1) CU_OK(c, cudaEventRecord(c->zc_ev[half], c->stream));
+    } else {
+        if ((st = prepare_ids(c, sample_ids, B, "pac_train_step_async", &d_ids)) != PAC_OK) return st;
+        if ((st = train_enqueue(c, d_ids, B, d_loss, hp)) != PAC_OK) return st;
+        if ((st = finish_ids(c)) != PAC_OK) return st;
+    }
+    if (copy_loss) CU_OK(c, cudaMemcpyAsync(loss_out, d_loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
     return PAC_OK;
 }
 

@@ -61,8 +61,11 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
-    pdl_wait();                 // weights, parameters and ids of this step are final from here on
-    const long long id = safe_id(p.ids, b, p.N, nullptr);        // mid_body reports clamped ids
+    // ids the host wrote before the launch can be fetched across the host link while the predecessor drains
+    long long id = p.host_ids ? safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr) : -1;
+    pdl_wait();                 // weights, parameters and (device) ids of this step are final from here on
+    if (!p.host_ids) id = safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr);
+    if (p.ids_copy && q == 0 && threadIdx.x == 0) p.ids_copy[b] = (int)id;
 
     // ---- phase 1: the GEMMs of this CTA's layers; the other warps fetch the head operands.
     // Both pipeline loops are run by a whole converged warp, one elected lane issues. ----
@@ -162,7 +165,7 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     cluster.sync();                                               // every token's u rows have arrived
 
     // ---- phase 3: chain, head, loss, reverse chain on the cluster-resident u ----
-    mid_body<ACT, bf16, 1, STATE_TILES>(p, cluster, reinterpret_cast<float4*>(u_loc), h, true);
+    mid_body<ACT, bf16, 1, STATE_TILES>(p, cluster, reinterpret_cast<float4*>(u_loc), h, true, id);
 }
 
 // Launch geometry: smallest cluster that gives one 4-column group per thread, at most four layers

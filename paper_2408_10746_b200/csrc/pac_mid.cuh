@@ -31,6 +31,9 @@ struct MidParams {
     int scratch;                // floats of block-local reduction scratch
     int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
     int layers_per_cta;         // one-kernel forward: layers whose down-projections each CTA of the cluster computes
+    int host_ids;               // 1: ids points at host memory the device can read (written before the launch, so
+                                // it may be read ahead of the predecessor's completion); read once per CTA
+    int* ids_copy;              // one-kernel forward: device copy of the batch's (clamped) ids for the later kernels, or null
     int u_swz;                  // STATE_TILES: a token row's 4-column groups are stored at (group ^ (token & u_swz))
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
@@ -145,7 +148,7 @@ __device__ __forceinline__ void mid_sum_products(const MidParams& p, const MidSh
 // operands, run mid_head_products and passed a cluster barrier.
 template <int ACT, typename DU, int GPT, int STATE>
 __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& cluster, float4* u_s, const MidShared& h,
-                                         bool products_ready) {
+                                         bool products_ready, long long known_id = -1) {
     constexpr int LT = MID_MAX_L;
     const int q = (int)cluster.block_rank();
     const int b = blockIdx.x / p.G;
@@ -208,7 +211,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             return *reinterpret_cast<const float4*>(du + (long long)l * p.lstride + base[g]);
         }
     };
-    const long long id = safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
+    const long long id = known_id >= 0 ? known_id : safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
     const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
     if (!products_ready) mid_prefetch_head(p, h, q, id, t, nt);
     cp_async_commit();                                                          // group: head operands

@@ -465,8 +465,8 @@ def test_async_step_equals_step_then_adam(which, tiny):
     else:
         spec, case = TINY, tiny
     hp = pac.AdamW()
-    n_steps = 12                                   # more than the 8 id-staging slots
-    perm = np.concatenate([pi.epoch_permutation(spec.N, 2, epoch=e) for e in range(4)])[:n_steps * spec.B]
+    n_steps = 150 if which == "tensor" else 12     # more than the id-staging slots (64-slot ring / 8 slots)
+    perm = np.concatenate([pi.epoch_permutation(spec.N, 2, epoch=e) for e in range(1 + n_steps * spec.B // spec.N)])[:n_steps * spec.B]
     a = case.context()
     a.set_params(pi.random_params(spec, 3))
     losses = torch.zeros(n_steps, dtype=torch.float32).pin_memory()
