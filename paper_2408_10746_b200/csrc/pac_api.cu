@@ -132,6 +132,7 @@ struct pac_ctx {
     cudaEvent_t zc_ev[2] = {nullptr, nullptr};
     unsigned long long zc_count = 0;
     bool step_host_ids = false;    // the step being enqueued reads its ids from the ring
+    bool step_early_ids = false;   // the step's device ids were final before any kernel still in flight was launched
     std::string err;
 };
 
@@ -528,6 +529,7 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     fp.mid.u = nullptr;
     fp.mid.layers_per_cta = pl.layers_per_cta;
     if (c->step_host_ids) { fp.mid.host_ids = 1; fp.mid.ids_copy = c->sc.ids; }
+    fp.mid.early_ids = c->step_early_ids ? 1 : 0;
     fp.mid.u_swz = pl.u_swz;
     fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset;
     fp.stamp = next_stamp(c, 0);
@@ -1072,7 +1074,10 @@ pac_status pac_gather(pac_ctx* c, const int* sample_ids, int B, void* dev_out) {
 static pac_status epoch_common(pac_ctx* c, const int* d_perm, long long n, int B, const pac_adamw* hp, float* d_losses) {
     for (long long s = 0; s < n / B; ++s) {
         const int* ids = d_perm + s * B;
+        // from the second step on the kernel ahead is this library's own, which does not write ids
+        c->step_early_ids = s > 0;
         pac_status st = train_enqueue(c, ids, B, d_losses ? d_losses + s : c->sc.loss, hp);
+        c->step_early_ids = false;
         if (st != PAC_OK) return st;
     }
     return PAC_OK;

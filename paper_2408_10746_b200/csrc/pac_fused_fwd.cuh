@@ -61,25 +61,46 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
-    // ids the host wrote before the launch can be fetched across the host link while the predecessor drains
-    long long id = p.host_ids ? safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr) : -1;
+    // Ids that were final before this launch (written by the host, or device ids no kernel ahead of this one
+    // touches) are read while the predecessor still drains, and so are the first cache tiles: the cache never
+    // changes, only the weights (updated by the predecessor) have to wait.
+    const bool early = p.host_ids || p.early_ids;
+    long long id = early ? safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr) : -1;
+    const uint64_t pol = l2_policy_evict_first();
+    uint32_t pre = 0;                                            // stages whose cache tile is already on its way
+    if (early && warp == 0 && n_layers > 0) {
+        pre = (uint32_t)min(n_layers * fp.k_chunks, fp.stages);
+        if (elect_one()) {
+            for (uint32_t s = 0; s < pre; ++s) {
+                mbar_expect_tx(full0 + 8 * s, stage_bytes);
+                tma_load_4d_hint(smem_u32(smem + (size_t)s * stage_bytes), &map_cache, full0 + 8 * s,
+                                 (int)(s % fp.k_chunks) * KC, 0, l_begin + (int)(s / fp.k_chunks), (int)id, pol);
+            }
+        }
+        __syncwarp();
+    }
     pdl_wait();                 // weights, parameters and (device) ids of this step are final from here on
-    if (!p.host_ids) id = safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr);
+    if (!early) id = safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr);
     if (p.ids_copy && q == 0 && threadIdx.x == 0) p.ids_copy[b] = (int)id;
 
     // ---- phase 1: the GEMMs of this CTA's layers; the other warps fetch the head operands.
     // Both pipeline loops are run by a whole converged warp, one elected lane issues. ----
     if (warp == 0) {
         uint32_t it = 0;
-        const uint64_t pol = l2_policy_evict_first();
         bool ok = true;
-        if (lane == 0 && n_layers > 0) stamp_begin(fp.stamp);
+        if (lane == 0 && n_layers > 0) stamp_begin(fp.stamp);      // first copy after the predecessor has finished
         for (int l = l_begin; l < l_end && ok; ++l) {
             for (int kc = 0; kc < fp.k_chunks; ++kc, ++it) {
                 const int s = it % fp.stages;
+                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+                if (it < pre) {
+                    // first round: the cache tile was requested before the wait above, the weight tile follows
+                    if (elect_one()) tma_load_4d(dst + a_bytes, &map_w, full0 + 8 * s, 0, kc * KC, 0, l);
+                    __syncwarp();
+                    continue;
+                }
                 const uint32_t ph = (it / fp.stages) & 1;
                 if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
                 if (elect_one()) {
                     mbar_expect_tx(full0 + 8 * s, stage_bytes);
                     tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, 0, l, (int)id, pol);

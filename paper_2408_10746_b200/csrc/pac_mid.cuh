@@ -33,6 +33,7 @@ struct MidParams {
     int layers_per_cta;         // one-kernel forward: layers whose down-projections each CTA of the cluster computes
     int host_ids;               // 1: ids points at host memory the device can read (written before the launch, so
                                 // it may be read ahead of the predecessor's completion); read once per CTA
+    int early_ids;              // 1: no kernel ahead of this one in the stream writes the ids (device memory)
     int* ids_copy;              // one-kernel forward: device copy of the batch's (clamped) ids for the later kernels, or null
     int u_swz;                  // STATE_TILES: a token row's 4-column groups are stored at (group ^ (token & u_swz))
     const float* u; long long lstride;
