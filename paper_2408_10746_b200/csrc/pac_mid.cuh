@@ -453,8 +453,20 @@ struct FinalizeParams {
 
 __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     pdl_trigger();
-    pdl_wait();
     const ParamLayout& lay = f.lay;
+    // W_down blocks fetch the old parameter and moments while the predecessor still runs: nothing since the
+    // previous finalisation writes them, and that one was over before the predecessor's own predecessor
+    // finished (every kernel of a step lets its successor start only after its own wait has returned or
+    // does not touch these arrays before its wait)
+    const long long i_wd = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    const bool wd_thread = (int)blockIdx.x < f.wd_blocks && blockIdx.x != gridDim.x - 1 && i_wd < lay.lam;
+    float4 p4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = p4, v4 = p4;
+    if (wd_thread && f.adam) {
+        p4 = *reinterpret_cast<const float4*>(f.params + i_wd);
+        m4 = *reinterpret_cast<const float4*>(f.m + i_wd);
+        v4 = *reinterpret_cast<const float4*>(f.v + i_wd);
+    }
+    pdl_wait();
     if (blockIdx.x == gridDim.x - 1) {
         // the last block: dlambda_l (one warp per layer, lanes over the per-block partials, fixed
         // shuffle order) and the mean loss
@@ -492,7 +504,7 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         } else {
             g4 = *reinterpret_cast<const float4*>(f.grads + i);
         }
-        if (f.adam) adamw_w_down4(f.params, f.m, f.v, i, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        if (f.adam) adamw_w_down4_loaded(f.params, f.m, f.v, i, p4, m4, v4, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
         return;
     }
     const long long i = lay.lam + (long long)(blockIdx.x - f.wd_blocks) * blockDim.x + threadIdx.x;

@@ -494,10 +494,19 @@ __device__ __forceinline__ void adamw_element(float* __restrict__ p, float* __re
 
 // Four consecutive elements of the W_down block (i a multiple of 4; d*r is a multiple of 4, so
 // the four share a layer): vector loads and stores, the same arithmetic per element.
+// The same with the old parameter and moments already in registers (a caller may fetch them early).
+__device__ __forceinline__ void adamw_w_down4_loaded(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
+                                                     long long i, float4 p4, float4 m4, float4 v4, float4 g4, const pac_adamw& hp,
+                                                     float bc1, float bc2, bf16* __restrict__ wdT, int d, int r);
 __device__ __forceinline__ void adamw_w_down4(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
                                               long long i, float4 g4, const pac_adamw& hp, float bc1, float bc2,
                                               bf16* __restrict__ wdT, int d, int r) {
-    float4 p4 = *reinterpret_cast<float4*>(p + i), m4 = *reinterpret_cast<float4*>(m + i), v4 = *reinterpret_cast<float4*>(v + i);
+    const float4 p4 = *reinterpret_cast<float4*>(p + i), m4 = *reinterpret_cast<float4*>(m + i), v4 = *reinterpret_cast<float4*>(v + i);
+    adamw_w_down4_loaded(p, m, v, i, p4, m4, v4, g4, hp, bc1, bc2, wdT, d, r);
+}
+__device__ __forceinline__ void adamw_w_down4_loaded(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
+                                                     long long i, float4 p4, float4 m4, float4 v4, float4 g4, const pac_adamw& hp,
+                                                     float bc1, float bc2, bf16* __restrict__ wdT, int d, int r) {
     p4.x = adamw_math(p4.x, m4.x, v4.x, g4.x, true, hp, bc1, bc2);
     p4.y = adamw_math(p4.y, m4.y, v4.y, g4.y, true, hp, bc1, bc2);
     p4.z = adamw_math(p4.z, m4.z, v4.z, g4.z, true, hp, bc1, bc2);

@@ -431,13 +431,15 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
         tma_prefetch_desc(&map_du);
     }
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), (uint32_t)p.tmem_cols); tmem_relinquish(); }
-    pdl_trigger();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
     pdl_wait();
+    // the successor may start only now: when it runs, the forward half of this step (and with it the
+    // previous step's parameter update) is known to be complete
+    pdl_trigger();
 
     if (warp == 0) {
         uint32_t it = 0;
