@@ -582,7 +582,7 @@ def main():
         "aux": aux,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = oracle_baseline(spec, args.cpu_budget, 16)
+        out["cpu_baseline"] = oracle_baseline(spec, args.cpu_budget, 256)
     elif rank == 0:
         out["cpu_baseline"] = None
     ctx.close()
