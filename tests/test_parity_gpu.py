@@ -490,6 +490,35 @@ def test_async_step_equals_step_then_adam(which, tiny):
     assert np.array_equal(a.get_params(), before) and a.get_opt_state()[2] == n_steps
 
 
+def test_stream_phase_and_kernel_timers():
+    """Both timing modes count every launch of the two cache passes, report plausible durations and
+    leave the results of the steps untouched."""
+    import paper_2408_10746_b200 as pac
+    from paper_2408_10746_b200 import binding
+    spec = TC_BASE.scaled(N=32, name="tc_timers")
+    case = Case(spec, materialize_cpu=False)
+    hp = pac.AdamW()
+    perm = torch.from_numpy(pi.epoch_permutation(spec.N, 2)[:4 * spec.B].astype(np.int32)).cuda()
+    ref = case.context()
+    ref.set_params(pi.random_params(spec, 3))
+    ref.train_epoch_dev(perm, spec.B, hp, None)
+    ref.sync()
+    for mode in (1, 2):
+        ctx = case.context()
+        ctx.set_params(pi.random_params(spec, 3))
+        ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, mode)
+        ctx.train_epoch_dev(perm, spec.B, hp, None)
+        times = ctx.kernel_times() if mode == 1 else ctx.stream_phase_times()
+        names = ("down_projection", "dw_down") if mode == 1 else ("first_pass", "second_pass")
+        for n in names:
+            ms, cnt = times[n]
+            assert cnt == 4 and 0.0 < ms / cnt < 5.0, (mode, n, ms, cnt)
+        again = ctx.kernel_times() if mode == 1 else ctx.stream_phase_times()
+        assert all(cnt == 0 for _, cnt in again.values())          # the call resets the counters
+        ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 0)
+        assert np.array_equal(ctx.get_params(), ref.get_params())
+
+
 def test_device_buffer_views_and_single_rank_data_parallel(tiny):
     """The zero-copy views alias the library's buffers (what an in-place all-reduce needs), and
     the data-parallel wrapper with one rank is the plain trainer."""
