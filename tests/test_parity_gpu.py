@@ -205,6 +205,14 @@ def test_frozen_inputs_untouched_and_errors_leave_state_alone(tiny):
     with pytest.raises(pac.PacError) as e:
         ctx.train_step(list(range(TINY.B + 1)))
     assert e.value.status_name == "PAC_ERR_INVALID_ARG"
+    # an empty minibatch is an argument error for every call that takes ids
+    scratch = torch.zeros((TINY.L, 1, TINY.S, TINY.d), device="cuda")
+    for call in (lambda: ctx.train_step([]), lambda: ctx.train_step_async([], pac.AdamW()),
+                 lambda: ctx.eval_logits([], torch.zeros((1, 2), device="cuda")), lambda: ctx.gather([], scratch),
+                 lambda: ctx.train_epoch(np.zeros(0, dtype=np.int32), 8, pac.AdamW())):
+        with pytest.raises(pac.PacError) as e:
+            call()
+        assert e.value.status_name == "PAC_ERR_INVALID_ARG"
     with pytest.raises(pac.PacError):
         ctx.train_epoch(np.arange(12, dtype=np.int32), 8, pac.AdamW())
     with pytest.raises(pac.PacError):
