@@ -41,6 +41,7 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     __shared__ __align__(8) unsigned long long bars[2 * 16 + 1];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh, have_sh;
+    __shared__ long long id_sh;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]), accf = smem_u32(&bars[32]);
     const int l_begin = q * p.layers_per_cta, l_end = min(p.L, l_begin + p.layers_per_cta);
     const int n_layers = max(0, l_end - l_begin);
@@ -56,16 +57,18 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     }
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), 512u); tmem_relinquish(); }
     pdl_trigger();
+    // Ids that were final before this launch (written by the host, or device ids no kernel ahead of this one
+    // touches) are read while the predecessor still drains, and so are the first cache tiles: the cache never
+    // changes, only the weights (updated by the predecessor) have to wait.  One thread fetches the id for the
+    // whole CTA: with ids in host memory every reading warp would be a transaction on the host link.
+    const bool early = p.host_ids || p.early_ids;
+    if (early && threadIdx.x == 64) id_sh = safe_id(p.ids, b, p.N, q == 0 ? p.status : nullptr);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
-    // Ids that were final before this launch (written by the host, or device ids no kernel ahead of this one
-    // touches) are read while the predecessor still drains, and so are the first cache tiles: the cache never
-    // changes, only the weights (updated by the predecessor) have to wait.
-    const bool early = p.host_ids || p.early_ids;
-    long long id = early ? safe_id(p.ids, b, p.N, (threadIdx.x == 0 && q == 0) ? p.status : nullptr) : -1;
+    long long id = early ? id_sh : -1;
     const uint64_t pol = l2_policy_evict_first();
     uint32_t pre = 0;                                            // stages whose cache tile is already on its way
     if (early && warp == 0 && n_layers > 0) {
