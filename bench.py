@@ -443,7 +443,7 @@ def main():
     # ---------------- end to end through the public per-step call ----------------
     # every step: B ids from page-locked host memory in (H2D), the step's loss out to page-locked
     # host memory (D2H); one wait at the end, then every loss is checked on the host
-    Ke = min(K, 512)
+    Ke = K
     h_ids = torch.from_numpy(ids_host[:Ke * B].copy()).pin_memory()
     h_losses = torch.zeros(Ke, dtype=torch.float32).pin_memory()
     ids_view, loss_ptr = h_ids.numpy(), h_losses.data_ptr()
