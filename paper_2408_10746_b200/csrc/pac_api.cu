@@ -129,6 +129,9 @@ struct pac_ctx {
     // pac_train_step_async without copy nodes in the stream: a ring of id slots in page-locked host memory that
     // the forward kernel reads directly (two halves, an event per half orders the reuse)
     int* zc_ids = nullptr;         // [ZC_SLOTS][max_batch]
+    unsigned* zc_tags = nullptr;   // [ZC_SLOTS] page-locked: sequence number of the step whose ids the slot holds (written last)
+    int* zc_dev_ids = nullptr;     // [2][max_batch] device: ids a finalisation kernel fetched for the step after it
+    unsigned* zc_dev_tag = nullptr;// [2] device: sequence number those ids belong to
     cudaEvent_t zc_ev[2] = {nullptr, nullptr};
     unsigned long long zc_count = 0;
     bool step_host_ids = false;    // the step being enqueued reads its ids from the ring
@@ -528,7 +531,13 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     fp.mid = mid_params(c, pl.mp, d_ids, B, train, d_logits_out);
     fp.mid.u = nullptr;
     fp.mid.layers_per_cta = pl.layers_per_cta;
-    if (c->step_host_ids) { fp.mid.host_ids = 1; fp.mid.ids_copy = c->sc.ids; }
+    if (c->step_host_ids) {
+        fp.mid.host_ids = 1; fp.mid.ids_copy = c->sc.ids;
+        const unsigned seq = (unsigned)(c->zc_count + 1);
+        fp.mid.pref_ids = c->zc_dev_ids + (size_t)(seq & 1u) * c->cfg.max_batch;
+        fp.mid.pref_tag = c->zc_dev_tag + (seq & 1u);
+        fp.mid.pref_seq = seq;
+    }
     fp.mid.early_ids = c->step_early_ids ? 1 : 0;
     fp.mid.u_swz = pl.u_swz;
     fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset;
@@ -579,6 +588,16 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         f.wdT = sc.wdT;
     }
     f.wd_blocks = (int)cdiv(c->lay.lam / 4, 256);
+    if (c->step_host_ids) {
+        // the step after this one will look for its ids under sequence number zc_count + 2 in the next ring slot
+        const unsigned next_seq = (unsigned)(c->zc_count + 2);
+        const int next_slot = (int)((c->zc_count + 1) % ZC_SLOTS);
+        f.next_host_ids = c->zc_ids + (size_t)next_slot * c->cfg.max_batch;
+        f.next_host_tag = c->zc_tags + next_slot;
+        f.next_seq = next_seq; f.next_n = c->cfg.max_batch;
+        f.next_dev_ids = c->zc_dev_ids + (size_t)(next_seq & 1u) * c->cfg.max_batch;
+        f.next_dev_tag = c->zc_dev_tag + (next_seq & 1u);
+    }
     const unsigned rest_blocks = cdiv(c->lay.total - c->lay.lam, 256);
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -654,6 +673,9 @@ void free_all(pac_ctx* c) {
     if (c->hc.iota) cudaFree(c->hc.iota);
     if (c->hc.copy_stream) cudaStreamDestroy(c->hc.copy_stream);
     if (c->zc_ids) cudaFreeHost(c->zc_ids);
+    if (c->zc_tags) cudaFreeHost(c->zc_tags);
+    if (c->zc_dev_ids) cudaFree(c->zc_dev_ids);
+    if (c->zc_dev_tag) cudaFree(c->zc_dev_tag);
     for (auto& e : c->zc_ev)
         if (e) cudaEventDestroy(e);
     if (c->h_ids) cudaFreeHost(c->h_ids);
@@ -854,9 +876,15 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     if (st == PAC_OK && fwd_plan.ok) {
         // id ring of pac_train_step_async (only the one-launch forward reads ids from host memory)
         if (cudaMallocHost((void**)&c->zc_ids, sizeof(int) * ZC_SLOTS * cfg->max_batch) != cudaSuccess ||
+            cudaMallocHost((void**)&c->zc_tags, sizeof(unsigned) * ZC_SLOTS) != cudaSuccess ||
+            cudaMalloc((void**)&c->zc_dev_ids, sizeof(int) * 2 * cfg->max_batch) != cudaSuccess ||
+            cudaMalloc((void**)&c->zc_dev_tag, sizeof(unsigned) * 2) != cudaSuccess ||
+            cudaMemset(c->zc_dev_tag, 0, sizeof(unsigned) * 2) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->zc_ev[0], cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->zc_ev[1], cudaEventDisableTiming) != cudaSuccess)
             st = fail(c, PAC_ERR_NOMEM, "pinned id ring allocation failed");
+        else
+            std::memset(c->zc_tags, 0, sizeof(unsigned) * ZC_SLOTS);      // sequence numbers start at 1
     }
     // tensor-core path: bf16 cache with TMA/UMMA-compatible sizes
     c->tensor_ok = false;
@@ -1021,6 +1049,8 @@ pac_status pac_train_step_async(pac_ctx* c, const int* sample_ids, int B, const 
         if (slot % (ZC_SLOTS / 2) == 0) CU_OK(c, cudaEventSynchronize(c->zc_ev[half]));     // the half's previous steps have run
         int* h = c->zc_ids + (size_t)slot * c->cfg.max_batch;
         std::memcpy(h, sample_ids, sizeof(int) * B);
+        // publish: ids first, then the step's sequence number (the kernel of the step before may be looking)
+        __atomic_store_n(&c->zc_tags[slot], (unsigned)(c->zc_count + 1), __ATOMIC_RELEASE);
         c->step_host_ids = true;
         st = train_enqueue(c, h, B, d_loss, hp);
         c->step_host_ids = false;

@@ -62,7 +62,10 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
     // changes, only the weights (updated by the predecessor) have to wait.  One thread fetches the id for the
     // whole CTA: with ids in host memory every reading warp would be a transaction on the host link.
     const bool early = p.host_ids || p.early_ids;
-    if (early && threadIdx.x == 64) id_sh = safe_id(p.ids, b, p.N, q == 0 ? p.status : nullptr);
+    if (early && threadIdx.x == 64) {
+        const bool pref = p.host_ids && p.pref_tag && ld_acquire_gpu(p.pref_tag) == p.pref_seq;
+        id_sh = safe_id(pref ? p.pref_ids : p.ids, b, p.N, q == 0 ? p.status : nullptr);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();

@@ -34,6 +34,9 @@ struct MidParams {
     int host_ids;               // 1: ids points at host memory the device can read (written before the launch, so
                                 // it may be read ahead of the predecessor's completion); read once per CTA
     int early_ids;              // 1: no kernel ahead of this one in the stream writes the ids (device memory)
+    // host_ids only: where the previous step's finalisation may already have left this step's ids in device
+    // memory (valid when *pref_tag == pref_seq); otherwise the ids are fetched across the host link
+    const int* pref_ids; const unsigned* pref_tag; unsigned pref_seq;
     int* ids_copy;              // one-kernel forward: device copy of the batch's (clamped) ids for the later kernels, or null
     int u_swz;                  // STATE_TILES: a token row's 4-column groups are stored at (group ^ (token & u_swz))
     const float* u; long long lstride;
@@ -134,11 +137,13 @@ __device__ __forceinline__ void mid_head_products(const MidParams& p, const MidS
         }
     }
 }
-// After a cluster-wide barrier behind mid_head_products: the sum over the cluster, in rank order.
+// After a cluster-wide barrier behind mid_head_products: the sum over the cluster, in rank order.  The
+// last row also takes the classifier bias, so the head needs no global load of its own later on.
 __device__ __forceinline__ void mid_sum_products(const MidParams& p, const MidShared& h, cg::cluster_group& cluster, int t, int nthr) {
     for (int e = t; e < (p.r + 1) * p.C; e += nthr) {
         float acc = 0.f;
         for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(h.prodq, g)[e];
+        if (e >= p.r * p.C) acc = p.b_head[e - p.r * p.C] + acc;      // b_head + (mean_s h_L) W_head
         h.prod[e] = acc;
     }
 }
@@ -305,18 +310,21 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(colsum, g)[j];
         pooled[j] = acc / (float)p.S;                     // mean_s a_L
     }
+    // That was this CTA's last access to a peer's shared memory: say so now and wait, at the very end, only
+    // for the peers to have said the same (a CTA must not exit while a peer may still read its memory).
+    cluster.barrier_arrive();
     __syncthreads();
 
     // ---- head: logits, loss, dlogits and d loss / d a_L, the same in every CTA of the cluster ----
     if (t < C) {
-        float acc = p.b_head[t] + prod[r * C + t];        // b_head + (mean_s h_L) W_head
+        float acc = prod[r * C + t];                      // b_head + (mean_s h_L) W_head
         for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], prod[j * C + t], acc);
         lg[t] = acc;
         if (q == 0) p.logits_out[(long long)b * C + t] = acc;
     }
     __syncthreads();
     if (!p.train) {
-        cluster.sync();                                   // peers may still be reading this CTA's shared memory
+        cluster.barrier_wait();                           // peers may still be reading this CTA's shared memory
         return;
     }
     {
@@ -413,7 +421,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int wv = 0; wv < nwarps; ++wv) acc += lred[wv * LT + t];
         p.lam_part[(long long)t * (p.B * p.G) + blockIdx.x] = acc;
     }
-    cluster.sync();                                       // keep shared memory alive until every peer has read it
+    cluster.barrier_wait();                               // keep shared memory alive until every peer has read it
 }
 
 // The stand-alone kernel: u comes from the global buffer written by the down-projection kernel.
@@ -449,7 +457,22 @@ struct FinalizeParams {
     float *params, *m, *v;
     pac_adamw hp; float bc1, bc2;
     bf16* wdT;                                               // [L][2][d][r] bf16 hi/lo shadow of W_down (may be null)
+    // Ids of the NEXT step (pac_train_step_async): if the host has already published them in its page-locked
+    // ring (tag == next_seq), block 0 copies them to device memory, off every kernel's critical path.
+    const int* next_host_ids; const unsigned* next_host_tag; unsigned next_seq; int next_n;
+    int* next_dev_ids; unsigned* next_dev_tag;
 };
+
+__device__ __forceinline__ unsigned ld_acquire_sys(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     pdl_trigger();
@@ -458,17 +481,22 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     // previous finalisation writes them, and that one was over before the predecessor's own predecessor
     // finished (every kernel of a step lets its successor start only after its own wait has returned or
     // does not touch these arrays before its wait)
-    const long long i_wd = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-    const bool wd_thread = (int)blockIdx.x < f.wd_blocks && blockIdx.x != gridDim.x - 1 && i_wd < lay.lam;
+    // block 0 takes dlambda and the loss (scheduled first, so it runs at once); blocks 1 .. wd_blocks take
+    // W_down, the remaining ones the head parameters
+    const int blk = (int)blockIdx.x - 1;
+    const long long i_wd = ((long long)blk * blockDim.x + threadIdx.x) * 4;
+    const bool wd_thread = blk >= 0 && blk < f.wd_blocks && i_wd < lay.lam;
     float4 p4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = p4, v4 = p4;
     if (wd_thread && f.adam) {
         p4 = *reinterpret_cast<const float4*>(f.params + i_wd);
         m4 = *reinterpret_cast<const float4*>(f.m + i_wd);
         v4 = *reinterpret_cast<const float4*>(f.v + i_wd);
     }
-    pdl_wait();
-    if (blockIdx.x == gridDim.x - 1) {
-        // the last block: dlambda_l (one warp per layer, lanes over the per-block partials, fixed
+    // Block 0 (dlambda and the mean loss) needs only what the forward half left behind, which is
+    // complete whenever this kernel runs (see above): it does not wait for the second pass at all, so a loss
+    // that goes straight to host memory is on its way long before the step ends.
+    if (blk < 0) {
+        // dlambda_l (one warp per layer, lanes over the per-block partials, fixed
         // shuffle order) and the mean loss
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
         for (int l = warp; l < f.L; l += nw) {
@@ -487,11 +515,22 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
             acc = warp_sum(acc);
             if (lane == 0) *f.loss_out = acc / (float)f.B;
         }
+        if (warp == 0 && f.next_host_tag) {
+            // the host writes a slot's ids first and its tag last; tag read first here, ids after it
+            const unsigned tag = ld_acquire_sys(f.next_host_tag);
+            if (tag == f.next_seq) {
+                for (int b = lane; b < f.next_n; b += 32) f.next_dev_ids[b] = *reinterpret_cast<const volatile int*>(f.next_host_ids + b);
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicExch(f.next_dev_tag, f.next_seq);
+            }
+        }
         return;
     }
-    if ((int)blockIdx.x < f.wd_blocks) {
+    pdl_wait();
+    if (blk < f.wd_blocks) {
         // W_down block, four consecutive elements per thread
-        const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+        const long long i = i_wd;
         if (i >= lay.lam) return;
         float4 g4;
         if (f.splits > 1) {
@@ -507,10 +546,10 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         if (f.adam) adamw_w_down4_loaded(f.params, f.m, f.v, i, p4, m4, v4, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
         return;
     }
-    const long long i = lay.lam + (long long)(blockIdx.x - f.wd_blocks) * blockDim.x + threadIdx.x;
+    const long long i = lay.lam + (long long)(blk - f.wd_blocks) * blockDim.x + threadIdx.x;
     if (i >= lay.total) return;
     float g;
-    if (i < lay.w_up) return;                            // lambda is handled by the last block
+    if (i < lay.w_up) return;                            // lambda is handled by block 0
     if (i < lay.w_head) {
         const long long e = i - lay.w_up;
         const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
