@@ -137,8 +137,10 @@ pac_status pac_train_step(pac_ctx* ctx, const int* sample_ids, int B, float* los
  * arrives there once the step has run: loss_out is HOST memory that must stay valid until the next
  * pac_sync; read it after pac_sync.  Page-locked memory (cudaHostAlloc / cudaHostRegister) is written
  * by the last kernel of the step itself; other memory gets a copy behind the step.  With the one-launch
- * forward the ids are likewise read by the kernel from a page-locked ring inside the library, so a
- * step is three kernels back to back and consecutive steps overlap as in pac_train_epoch_dev.  Errors of the arguments are reported at once,
+ * forward the ids are likewise taken by the kernels from a page-locked ring inside the library (the
+ * step before fetches them into device memory when the host is already a call ahead, otherwise the
+ * forward kernel reads them across the host link), so a step is three kernels back to back and
+ * consecutive steps overlap as in pac_train_epoch_dev.  Errors of the arguments are reported at once,
  * device-side errors by the next pac_sync.  The step a caller loops over when the minibatches
  * are chosen on the host one at a time (Section IV-B: from the second epoch on a step needs
  * nothing but the cached activations of its samples). */
