@@ -599,6 +599,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         f.next_dev_tag = c->zc_dev_tag + (next_seq & 1u);
     }
     const unsigned rest_blocks = cdiv(c->lay.total - c->lay.lam, 256);
+    f.rest_blocks = (int)rest_blocks;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     pdl_launch_config(&cfg, attr, dim3(f.wd_blocks + rest_blocks + 1), dim3(256), 0, c->stream);   // + one block for lambda and the loss

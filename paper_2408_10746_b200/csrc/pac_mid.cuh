@@ -451,7 +451,8 @@ struct FinalizeParams {
     const float* lam_part; int lam_blocks;
     const float *pooled_a, *gvec, *pooled_y, *dlogits, *loss_b;
     float* grads; float* loss_out;
-    int wd_blocks;                                           // leading blocks that handle W_down, 4 elements per thread
+    int wd_blocks;                                           // blocks that handle W_down, 4 elements per thread
+    int rest_blocks;                                         // blocks that handle W_up, W_head, b_head, one element per thread
     // AdamW
     int adam;
     float *params, *m, *v;
@@ -481,11 +482,11 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     // previous finalisation writes them, and that one was over before the predecessor's own predecessor
     // finished (every kernel of a step lets its successor start only after its own wait has returned or
     // does not touch these arrays before its wait)
-    // block 0 takes dlambda and the loss (scheduled first, so it runs at once); blocks 1 .. wd_blocks take
-    // W_down, the remaining ones the head parameters
+    // block 0 takes dlambda and the loss (scheduled first, so it runs at once), the next rest_blocks blocks the
+    // head parameters, the remaining wd_blocks blocks W_down
     const int blk = (int)blockIdx.x - 1;
-    const long long i_wd = ((long long)blk * blockDim.x + threadIdx.x) * 4;
-    const bool wd_thread = blk >= 0 && blk < f.wd_blocks && i_wd < lay.lam;
+    const long long i_wd = ((long long)(blk - f.rest_blocks) * blockDim.x + threadIdx.x) * 4;
+    const bool wd_thread = blk >= f.rest_blocks && i_wd < lay.lam;
     float4 p4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = p4, v4 = p4;
     if (wd_thread && f.adam) {
         p4 = *reinterpret_cast<const float4*>(f.params + i_wd);
@@ -527,8 +528,36 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         }
         return;
     }
+    if (blk < f.rest_blocks) {
+        // head parameters: like block 0 they need only the forward half's per-sample vectors, so these blocks
+        // finish (and make room for the W_down blocks) while the second pass still runs
+        const long long i = lay.lam + (long long)blk * blockDim.x + threadIdx.x;
+        if (i >= lay.total) return;
+        float g;
+        if (i < lay.w_up) return;                            // lambda is handled by block 0
+        if (i < lay.w_head) {
+            const long long e = i - lay.w_up;
+            const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
+            g = 0.f;
+#pragma unroll 16
+            for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], f.gvec[(long long)b * f.d + k], g);
+        } else if (i < lay.b_head) {
+            const long long e = i - lay.w_head;
+            const int k = (int)(e / f.C), c = (int)(e - (long long)k * f.C);
+            g = 0.f;
+#pragma unroll 16
+            for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_y[(long long)b * f.d + k], f.dlogits[(long long)b * f.C + c], g);
+        } else {
+            const int c = (int)(i - lay.b_head);
+            g = 0.f;
+            for (int b = 0; b < f.B; ++b) g += f.dlogits[(long long)b * f.C + c];
+        }
+        f.grads[i] = g;
+        if (f.adam) adamw_element(f.params, f.m, f.v, i, g, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        return;
+    }
     pdl_wait();
-    if (blk < f.wd_blocks) {
+    {
         // W_down block, four consecutive elements per thread
         const long long i = i_wd;
         if (i >= lay.lam) return;
@@ -546,29 +575,6 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         if (f.adam) adamw_w_down4_loaded(f.params, f.m, f.v, i, p4, m4, v4, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
         return;
     }
-    const long long i = lay.lam + (long long)(blk - f.wd_blocks) * blockDim.x + threadIdx.x;
-    if (i >= lay.total) return;
-    float g;
-    if (i < lay.w_up) return;                            // lambda is handled by block 0
-    if (i < lay.w_head) {
-        const long long e = i - lay.w_up;
-        const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
-        g = 0.f;
-#pragma unroll 16
-        for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], f.gvec[(long long)b * f.d + k], g);
-    } else if (i < lay.b_head) {
-        const long long e = i - lay.w_head;
-        const int k = (int)(e / f.C), c = (int)(e - (long long)k * f.C);
-        g = 0.f;
-#pragma unroll 16
-        for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_y[(long long)b * f.d + k], f.dlogits[(long long)b * f.C + c], g);
-    } else {
-        const int c = (int)(i - lay.b_head);
-        g = 0.f;
-        for (int b = 0; b < f.B; ++b) g += f.dlogits[(long long)b * f.C + c];
-    }
-    f.grads[i] = g;
-    if (f.adam) adamw_element(f.params, f.m, f.v, i, g, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
 }
 
 // Shape test and launch geometry of the fused kernel: G CTAs per sample, one 4-column
