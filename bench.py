@@ -70,7 +70,7 @@ class ClockSampler(threading.Thread):
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
 
-    def __init__(self, device_index: int, period_s: float = 0.005):
+    def __init__(self, device_index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
         self.period, self.samples, self.reasons, self.max_mhz = period_s, [], set(), None
         self._stop_evt = threading.Event()
@@ -326,6 +326,59 @@ def run_host_cache(args, spec):
     print(json.dumps(out))
 
 
+def measure_aux_workload(spec, dev, stream, peaks, K=64, W=8, R=5):
+    """A second shape beside the headline one: the same per-step shapes as the named workload on a
+    cache cut to fewer samples (still far larger than L2).  Median of R timed K-step regions plus the
+    event-bracketed kernels and the device-timed stream phases."""
+    import torch
+    import paper_2408_10746_b200 as pac
+    from paper_2408_10746_b200 import binding
+    cache = pi.cache_full(spec, 0, dev)
+    labels = pi.labels(spec, 0, dev)
+    ctx = pac.PacContext(dev.index, stream.cuda_stream)
+    ctx.cache_register(cache, labels)
+    ctx.adapter_init(r=spec.r, n_out=spec.n_out, max_batch=spec.B)
+    hp = pac.AdamW()
+    B = spec.B
+    d_ids = torch.from_numpy(epoch_ids(spec, K)).to(dev)
+    ctx.train_epoch_dev(d_ids[:W * B], B, hp, None)
+    ctx.sync()
+    regions = []
+    for _ in range(R):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            ctx.train_epoch_dev(d_ids, B, hp, None)
+            b.record(stream)
+        torch.cuda.synchronize()
+        regions.append(a.elapsed_time(b))
+    ms = float(np.median(regions))
+    pass_bytes = B * spec.L * spec.S * spec.d * spec.elem_bytes
+    ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 1)
+    ctx.kernel_times()
+    ctx.train_epoch_dev(d_ids[:min(K, 32) * B], B, hp, None)
+    kt = ctx.kernel_times()
+    ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 2)
+    ctx.train_epoch_dev(d_ids[:min(K, 32) * B], B, hp, None)
+    pt = ctx.stream_phase_times()
+    ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 0)
+    stream_gbs = 2 * pass_bytes / (ms * 1e-3 / K) / 1e9
+    out = {"workload": workload_name(spec), "kernel_path": ctx.kernel_path(), "steps": K, "repeats": R,
+           "ms_per_step": ms / K, "samples_per_s": K * B / (ms * 1e-3),
+           "cache_stream": {"gbs_two_reads": stream_gbs, "frac_of_peak": stream_gbs / peaks["hbm_gbs"]},
+           "kernels": {n: {"avg_ms": t / c, **({"gbs": pass_bytes / (t / c * 1e-3) / 1e9,
+                                                 "frac": pass_bytes / (t / c * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                                                if n in ("down_projection", "dw_down") else {})}
+                       for n, (t, c) in kt.items() if c},
+           "stream_phase": {n: {"avg_ms": t / c, "frac": pass_bytes / (t / c * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                            for n, (t, c) in pt.items() if c}}
+    ctx.close()
+    del cache, labels
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -345,6 +398,11 @@ def main():
                     help="measure the block-wise absmax INT8 codec (paper Eq. 1-2) instead of the train step")
     ap.add_argument("--cache", choices=["device", "host"], default="device",
                     help="host: keep the cache in page-locked host memory and reload every minibatch (N defaults to 1024)")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="how many times the K-step region is timed (median reported); default: at least 5, more "
+                         "for short regions")
+    ap.add_argument("--no-aux-workloads", action="store_true",
+                    help="skip the reduced-N BART-Large / T5-Large entries of aux.workloads")
     ap.add_argument("--n-samples", type=int, default=0,
                     help="profiling aid: shrink the cache to this many samples (same per-step shapes); "
                          "the JSON line then names the reduced workload")
@@ -418,24 +476,48 @@ def main():
         return run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world)
 
     # ---------------- device-resident timing (value) ----------------
+    # The K-step region is timed R >= 5 times (each bracketed by a barrier and a device synchronisation
+    # on both sides, CUDA events on the context's stream); the line reports the median region.  R grows
+    # for short regions so that the clock sampler, which runs across all repeats, sees enough samples.
     ctx.train_epoch_dev(d_warm, B, hp, None)
     ctx.sync()
-    sampler = ClockSampler(local)
+    probe0, probe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        probe0.record(stream)
+        ctx.train_epoch_dev(d_ids, B, hp, None)
+        probe1.record(stream)
+    ctx.sync()
+    region_est_ms = max(1e-3, probe0.elapsed_time(probe1))
+    R = args.repeats if args.repeats > 0 else int(min(100, max(5, np.ceil(150.0 / region_est_ms))))
+    if dist is not None:
+        rt = torch.tensor([R], dtype=torch.int64, device=dev)
+        dist.all_reduce(rt, op=dist.ReduceOp.MAX)
+        R = int(rt.item())
+    sampler = ClockSampler(local, period_s=0.002)
     launches0 = ctx.launch_count()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    region_ms, t_enq = [], 0.0
     barrier()
     sampler.start()
-    with torch.cuda.stream(stream):
-        start.record(stream)
-        t_enq = time.perf_counter()
-        ctx.train_epoch_dev(d_ids, B, hp, d_losses)
-        t_enq = time.perf_counter() - t_enq                 # the call returns once everything is enqueued
-        end.record(stream)
-    barrier()
+    for rep in range(R):
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            start.record(stream)
+            t0 = time.perf_counter()
+            ctx.train_epoch_dev(d_ids, B, hp, d_losses)
+            t_enq += time.perf_counter() - t0               # the call returns once everything is enqueued
+            end.record(stream)
+        barrier()
+        region_ms.append(start.elapsed_time(end))
     clocks = sampler.finish()
-    ms = start.elapsed_time(end)
-    launches = ctx.launch_count() - launches0
+    t_enq /= R
+    launches = (ctx.launch_count() - launches0) // R        # launches of ONE K-step region
     ctx.sync()
+    if dist is not None:
+        t = torch.tensor(region_ms, dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)            # per repeat, the slowest rank
+        region_ms = t.tolist()
+    ms = float(np.median(region_ms))
     losses = d_losses.cpu().numpy()
     if not np.isfinite(losses).all():
         raise SystemExit("non-finite loss in the timed region")
@@ -450,21 +532,25 @@ def main():
     for i in range(3):
         ctx.train_step_async(ids_view[i * B:(i + 1) * B], hp, loss_ptr + 4 * i)
     ctx.sync()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    t0 = time.perf_counter()
-    with torch.cuda.stream(stream):
-        e0.record(stream)
-        for i in range(Ke):
-            ctx.train_step_async(ids_view[i * B:(i + 1) * B], hp, loss_ptr + 4 * i)
-        e1.record(stream)
-    enqueue_ms = 1e3 * (time.perf_counter() - t0)           # host time to enqueue the Ke steps
-    ctx.sync()
-    barrier()
-    wall_ms = 1e3 * (time.perf_counter() - t0)
-    e2e_ms = max(e0.elapsed_time(e1), wall_ms)
-    if not np.isfinite(h_losses.numpy()).all():
-        raise SystemExit("non-finite loss in the end-to-end region")
+    e2e_regions, enqueue_ms = [], 0.0
+    for rep in range(R):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0 = time.perf_counter()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for i in range(Ke):
+                ctx.train_step_async(ids_view[i * B:(i + 1) * B], hp, loss_ptr + 4 * i)
+            e1.record(stream)
+        enqueue_ms += 1e3 * (time.perf_counter() - t0)      # host time to enqueue the Ke steps
+        ctx.sync()
+        barrier()
+        wall_ms = 1e3 * (time.perf_counter() - t0)
+        e2e_regions.append(max(e0.elapsed_time(e1), wall_ms))
+        if not np.isfinite(h_losses.numpy()).all():
+            raise SystemExit("non-finite loss in the end-to-end region")
+    enqueue_ms /= R
+    e2e_ms = float(np.median(e2e_regions))
 
     # ---------------- per-kernel times of the two cache-stream kernels ----------------
     ctx.set_option(binding.PAC_OPT_KERNEL_TIMING, 1)
@@ -506,9 +592,9 @@ def main():
         aux["note"] = "host ids per call (H2D of B ids inside the timed region), events on the context's stream"
 
     if dist is not None:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = t.tolist()
+        e2e_ms = float(t.item())
 
     peaks = load_peaks()
     pass_bytes = B * spec.L * spec.S * spec.d * spec.elem_bytes          # one read of the minibatch's slabs
@@ -565,6 +651,8 @@ def main():
         "metric": METRIC, "value": world * K * B / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if spec.dtype == "bf16" else "f32", "data": "synthetic",
+        "repeats": {"n": R, "statistic": "median", "region_ms_min": float(np.min(region_ms)), "region_ms_median": ms,
+                    "region_ms_max": float(np.max(region_ms))},
         "config": {"workload": workload_name(spec), "kernel_path": ctx.kernel_path(),
                    "l2": "each step gathers a different minibatch from a cache far larger than L2 "
                          f"({spec.cache_bytes / 1e9:.2f} GB)", "parallelism": "replicas" if world > 1 else "1 GPU",
@@ -581,6 +669,16 @@ def main():
         "final_loss": float(losses[-1]),
         "aux": aux,
     }
+    if rank == 0 and world == 1 and args.config == "t5_base" and not args.n_samples and not args.no_aux_workloads \
+            and not args.force_simt:
+        # two more shapes beside the headline one, each named as a reduced-N entry
+        ctx.close()
+        del cache, d_ids, d_warm
+        torch.cuda.empty_cache()
+        out["aux"]["workloads"] = []
+        for name in ("bart_large", "t5_large"):
+            big = pi.CONFIGS[name]
+            out["aux"]["workloads"].append(measure_aux_workload(big.scaled(N=512, name=f"{name}[N=512]"), dev, stream, peaks))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = oracle_baseline(spec, args.cpu_budget, 256)
     elif rank == 0:

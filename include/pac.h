@@ -146,6 +146,21 @@ pac_status pac_train_step(pac_ctx* ctx, const int* sample_ids, int B, float* los
  * nothing but the cached activations of its samples). */
 pac_status pac_train_step_async(pac_ctx* ctx, const int* sample_ids, int B, const pac_adamw* hp, float* loss_out);
 
+/* pac_train_step without any wait and with the loss left on the device: the step is enqueued and
+ * the call returns; the mean loss of the minibatch is written to *dev_loss (device, one float; NULL
+ * keeps it in a buffer of the context).  The per-step call of data-parallel training (Section V-B:
+ * every device trains on its share of the minibatch, then the devices combine the adapter
+ * gradients): a collective enqueued behind this call on the context's stream reduces the gradient
+ * buffer of pac_device_buffers in place, pac_adam_step follows, and the host reads losses once per
+ * epoch instead of once per step. */
+pac_status pac_train_step_dev_loss(pac_ctx* ctx, const int* sample_ids, int B, float* dev_loss);
+
+/* Factor in (0, 1] that every optimizer update (pac_adam_step and the updates fused into
+ * pac_train_step_async / pac_train_epoch*) applies to each gradient as it reads it; the gradient
+ * buffer keeps its values.  1 by default.  With W data-parallel ranks whose gradient buffers hold the
+ * SUM over ranks after an all-reduce, 1/W makes the update use the mean (Section V-B). */
+pac_status pac_set_grad_scale(pac_ctx* ctx, float scale);
+
 /* AdamW on the adapter parameters (and the classifier head) from the current gradients:
  * decoupled decay on W_down, W_up, W_head; none on lambda and b_head; bias-corrected
  * moments; step counter advances by one. */
@@ -220,6 +235,22 @@ pac_status pac_launch_count(pac_ctx* ctx, long long* n);
 /* Waits for the context's stream; reports device-side status words (bounded waits that
  * ran out, ids clamped by pac_train_epoch_dev). */
 pac_status pac_sync(pac_ctx* ctx);
+/* What a timeout means for the training state.  Every wait inside the pipeline kernels (on a copy, an
+ * accumulator, a peer CTA) gives up after about a second, records PAC_ERR_TIMEOUT in the device status
+ * words and lets its kernel finish without its results.  From that moment until the next pac_sync every
+ * optimizer update (fused or pac_adam_step) finds the flag and leaves parameters, moments and gradients
+ * untouched; pac_sync reports PAC_ERR_TIMEOUT once, clears the flag and takes the skipped updates off the
+ * step counter.  Only the step in which the wait ran out can be half applied (when it was the second
+ * pass that gave up, the head-side parameters of that step are already updated): restore the last
+ * checkpoint (pac_set_params / pac_set_opt_state) after a PAC_ERR_TIMEOUT unless the timed-out call was
+ * pac_selftest_wait_expiry.
+ *
+ * pac_selftest_wait_expiry exercises that path without breaking anything: one CTA allocates tensor
+ * memory, waits limit_ns nanoseconds (1e3 .. 1e8) on a barrier nobody arrives at, and leaves the way the
+ * pipeline kernels do after an abort.  The call waits for the stream; it returns PAC_OK when the wait
+ * reported expiry, and the status word it set is then reported by the next pac_sync like any other
+ * timeout.  The paper describes no failure handling for this path; this is the library's own contract. */
+pac_status pac_selftest_wait_expiry(pac_ctx* ctx, unsigned long long limit_ns);
 const char* pac_last_error(const pac_ctx* ctx);
 /* Which kernels the next train step will use (valid after adapter_init): "simt", "tensor", or
  * "tensor+fused_forward" when a batch of max_batch samples runs the down-projections
@@ -266,7 +297,9 @@ pac_status pac_dequantize_absmax(int device, void* cuda_stream, const signed cha
  * (pac_act), n_out = C; dev_sample_ids: device, B int32 ids (an id outside [0, N) is clamped
  * into range, not reported); dev_out: device, fp32 [B][C]; err / err_len: optional host buffer
  * that receives a message when the status is not PAC_OK.  The work is enqueued on the stream;
- * dev_out is valid once the stream has reached that point. */
+ * dev_out is valid once the stream has reached that point.  The call makes `device` current while
+ * it runs and puts the caller's current device back before it returns.  Limits beside the scratch
+ * size: L <= 65535, (d + C + 32) floats within 48 KB of shared memory. */
 #define PAC_STATIC_SCRATCH_BYTES (8u << 20)
 pac_status pac_eval_logits_static(int device, void* cuda_stream, const void* dev_cache, int dtype, long long N, int L,
                                   int S, int d, const float* dev_params, int r, int act, int n_out,

@@ -22,10 +22,10 @@ STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_S
                 "PAC_ERR_UNSUPPORTED", "PAC_ERR_NOMEM", "PAC_ERR_CUDA", "PAC_ERR_TIMEOUT"]
 
 # every symbol include/pac.h declares
-EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_cache_register_host", "pac_adapter_init", "pac_train_step", "pac_train_step_async",
+EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_cache_register_host", "pac_adapter_init", "pac_train_step", "pac_train_step_dev_loss", "pac_set_grad_scale", "pac_train_step_async",
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
-           "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_stream_phase_times", "pac_launch_count", "pac_sync", "pac_last_error",
+           "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_stream_phase_times", "pac_launch_count", "pac_sync", "pac_selftest_wait_expiry", "pac_last_error",
            "pac_kernel_path", "pac_eval_logits_static", "pac_quantize_absmax", "pac_dequantize_absmax"]
 
 
@@ -92,6 +92,8 @@ def load_library() -> C.CDLL:
         "pac_kernel_times": [P, C.POINTER(C.c_double), C.POINTER(LL)],
         "pac_stream_phase_times": [P, C.POINTER(C.c_double), C.POINTER(LL)],
         "pac_device_buffers": [P, C.POINTER(P), C.POINTER(P)], "pac_params_changed": [P],
+        "pac_selftest_wait_expiry": [P, C.c_ulonglong],
+        "pac_train_step_dev_loss": [P, P, I, P], "pac_set_grad_scale": [P, F],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -201,6 +203,17 @@ class PacContext:
         self._ck(self._lib.pac_train_step(self._h, ids.ctypes.data, ids.size, C.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
 
+    def train_step_dev_loss(self, sample_ids, dev_loss_ptr: int = 0):
+        """Enqueues forward + backward of one minibatch and returns at once; the mean loss goes to the
+        device float at dev_loss_ptr (0: kept inside the context)."""
+        ids = _ids(sample_ids)
+        st = self._lib.pac_train_step_dev_loss(self._h, ids.ctypes.data, ids.size, dev_loss_ptr or None)
+        if st != 0:
+            self._ck(st)
+
+    def set_grad_scale(self, scale: float):
+        self._ck(self._lib.pac_set_grad_scale(self._h, scale))
+
     def train_step_async(self, sample_ids, hp: AdamW, loss_out_ptr: int = 0):
         """Enqueues one whole step (forward, backward, AdamW) and returns at once.  loss_out_ptr: address
         of one host float (page-locked for a truly asynchronous copy) that receives the loss, or 0."""
@@ -309,6 +322,11 @@ class PacContext:
 
     def sync(self):
         self._ck(self._lib.pac_sync(self._h))
+
+    def selftest_wait_expiry(self, limit_ns: int = 100_000):
+        """Runs the bounded-wait self-test (a wait nobody satisfies gives up after limit_ns); the next
+        sync() then raises PAC_ERR_TIMEOUT once."""
+        self._ck(self._lib.pac_selftest_wait_expiry(self._h, limit_ns))
 
     def kernel_path(self) -> str:
         return self._lib.pac_kernel_path(self._h).decode()

@@ -94,6 +94,7 @@ struct pac_ctx {
     ParamLayout lay{};
     float *params = nullptr, *grads = nullptr, *m = nullptr, *v = nullptr;
     long long step = 0;
+    float grad_scale = 1.f;        // factor the optimizer applies to every gradient (data parallel: 1 / world)
     int max_rows = 0;              // max_batch * S
     int chain_blocks_max = 0;
     Scratch sc;
@@ -586,6 +587,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         f.params = c->params; f.m = c->m; f.v = c->v; f.hp = *hp;
         bias_corrections(hp, c->step, &f.bc1, &f.bc2);
         f.wdT = sc.wdT;
+        f.grad_scale = c->grad_scale;
     }
     f.wd_blocks = (int)cdiv(c->lay.lam / 4, 256);
     if (c->step_host_ids) {
@@ -598,6 +600,7 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         f.next_dev_ids = c->zc_dev_ids + (size_t)(next_seq & 1u) * c->cfg.max_batch;
         f.next_dev_tag = c->zc_dev_tag + (next_seq & 1u);
     }
+    f.status = c->status;
     const unsigned rest_blocks = cdiv(c->lay.total - c->lay.lam, 256);
     f.rest_blocks = (int)rest_blocks;
     cudaLaunchConfig_t cfg = {};
@@ -634,7 +637,7 @@ pac_status adam_enqueue(pac_ctx* c, const pac_adamw* hp) {
     const int wd_blocks = (c->lay.lam % 4 == 0) ? (int)cdiv(c->lay.lam / 4, 256) : 0;
     const unsigned rest = cdiv(c->lay.total - (wd_blocks ? c->lay.lam : 0), 256);
     adamw_kernel<<<wd_blocks + rest, 256, 0, c->stream>>>(c->params, c->grads, c->m, c->v, c->lay.total, c->lay, *hp, bc1, bc2,
-                                                          c->sc.wdT, c->dm.d, c->dm.r, wd_blocks);
+                                                          c->sc.wdT, c->dm.d, c->dm.r, wd_blocks, c->status, c->grad_scale);
     LAUNCH_CHECK(c);
     return PAC_OK;
 }
@@ -885,7 +888,10 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             cudaEventCreateWithFlags(&c->zc_ev[1], cudaEventDisableTiming) != cudaSuccess)
             st = fail(c, PAC_ERR_NOMEM, "pinned id ring allocation failed");
         else
+        {
             std::memset(c->zc_tags, 0, sizeof(unsigned) * ZC_SLOTS);      // sequence numbers start at 1
+            std::memset(c->zc_ids, 0, sizeof(int) * ZC_SLOTS * cfg->max_batch);
+        }
     }
     // tensor-core path: bf16 cache with TMA/UMMA-compatible sizes
     c->tensor_ok = false;
@@ -1017,6 +1023,22 @@ pac_status pac_train_step(pac_ctx* c, const int* sample_ids, int B, float* loss_
         CU_OK(c, cudaStreamSynchronize(c->stream));
         *loss_out = *c->h_loss;
     }
+    return PAC_OK;
+}
+
+pac_status pac_train_step_dev_loss(pac_ctx* c, const int* sample_ids, int B, float* dev_loss) {
+    NEED_INIT(c, "pac_train_step_dev_loss");
+    const int* d_ids = nullptr;
+    pac_status st = prepare_ids(c, sample_ids, B, "pac_train_step_dev_loss", &d_ids);
+    if (st != PAC_OK) return st;
+    if ((st = train_enqueue(c, d_ids, B, dev_loss ? dev_loss : c->sc.loss, nullptr)) != PAC_OK) return st;
+    return finish_ids(c);
+}
+
+pac_status pac_set_grad_scale(pac_ctx* c, float scale) {
+    NEED_CTX(c);
+    if (!(scale > 0.f) || !(scale <= 1.f)) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_grad_scale: scale must lie in (0, 1]");
+    c->grad_scale = scale;
     return PAC_OK;
 }
 
@@ -1318,9 +1340,37 @@ pac_status pac_sync(pac_ctx* c) {
     CU_OK(c, cudaMemcpyAsync(c->h_status, c->status, sizeof(unsigned) * ST_WORDS, cudaMemcpyDeviceToHost, c->stream));
     CU_OK(c, cudaMemsetAsync(c->status, 0, sizeof(unsigned) * ST_WORDS, c->stream));
     CU_OK(c, cudaStreamSynchronize(c->stream));
-    if (c->h_status[ST_TIMEOUT]) return fail(c, PAC_ERR_TIMEOUT, "a bounded device-side wait ran out (%u)", c->h_status[ST_TIMEOUT]);
+    // optimizer updates that found the timeout flag set were left out: they do not count as steps
+    const long long skipped = (long long)c->h_status[ST_SKIPPED_STEPS];
+    c->step = c->step > skipped ? c->step - skipped : 0;
+    if (c->h_status[ST_TIMEOUT])
+        return fail(c, PAC_ERR_TIMEOUT, "a bounded device-side wait ran out (%u); %lld later optimizer updates were skipped",
+                    c->h_status[ST_TIMEOUT], skipped);
     if (c->h_status[ST_CLAMPED_IDS])
         return fail(c, PAC_ERR_SAMPLE_ID_RANGE, "%u device-resident sample ids were outside [0, N) and were clamped", c->h_status[ST_CLAMPED_IDS]);
+    return PAC_OK;
+}
+
+pac_status pac_selftest_wait_expiry(pac_ctx* c, unsigned long long limit_ns) {
+    NEED_CTX(c);
+    if (limit_ns < 1000ull || limit_ns > 100000000ull)
+        return fail(c, PAC_ERR_INVALID_ARG, "pac_selftest_wait_expiry: limit_ns must lie in [1e3, 1e8]");
+    CU_OK(c, cudaSetDevice(c->device));
+    unsigned* d_res = nullptr;
+    CU_OK(c, cudaMalloc((void**)&d_res, 2 * sizeof(unsigned)));
+    unsigned h_res[2] = {0u, 0u};
+    cudaError_t e = cudaMemsetAsync(d_res, 0, 2 * sizeof(unsigned), c->stream);
+    if (e == cudaSuccess) {
+        selftest_wait_expiry_kernel<<<1, 64, 0, c->stream>>>(c->status, limit_ns, d_res);
+        c->launches++;
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_res, d_res, sizeof h_res, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    cudaFree(d_res);
+    if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "pac_selftest_wait_expiry: %s", cudaGetErrorString(e));
+    if (h_res[0] != 1u || h_res[1] != 1u)
+        return fail(c, PAC_ERR_BAD_STATE, "pac_selftest_wait_expiry: the wait did not report expiry (expired=%u abort=%u)", h_res[0], h_res[1]);
     return PAC_OK;
 }
 
@@ -1385,11 +1435,17 @@ cudaError_t static_forward(cudaStream_t st, const T* cache, long long N, int L, 
     MatB_RowMajor Bm{{params + lay.w_down, (long long)d * r, r}};
     StoreRowMajor E{u, n, r};
     dim3 grid(cdiv(r, SG_BN), cdiv(M, SG_BM), (unsigned)L);
+    cudaError_t e;
+    // a launch that is rejected ends the call: later kernels would read scratch the earlier one never wrote
     gemm_simt<<<grid, 256, 0, st>>>(M, r, d, A, Bm, E);                                  // u_l = h_l W_down^l
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (act == PAC_ACT_RELU) chain_fwd_kernel<PAC_ACT_RELU><<<cdiv(n, 256), 256, 0, st>>>(u, a, params + lay.lam, L, n, n);
     else chain_fwd_kernel<PAC_ACT_IDENTITY><<<cdiv(n, 256), 256, 0, st>>>(u, a, params + lay.lam, L, n, n);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     pool_tokens_kernel<<<B, 128, 0, st>>>(a + (long long)(L - 1) * n, pooled_a, S, r);     // mean_s a_L
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     pool_last_layer_batch_kernel<T><<<B, 256, 0, st>>>(cache, ids, N, L, S, d, hbar_b, iota);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     cls_head_kernel<<<B, 256, sizeof(float) * (d + C + 32), st>>>(hbar_b, iota, B, nullptr, pooled_a, params + lay.w_up,
                                                                  params + lay.w_head, params + lay.b_head, B, S, d, r, C, 0,
                                                                  nullptr, out, nullptr, nullptr, nullptr, nullptr, nullptr);
@@ -1408,8 +1464,24 @@ extern "C" pac_status pac_eval_logits_static(int device, void* cuda_stream, cons
     if (N < 1 || L < 1 || S < 1 || d < 1 || r < 1 || n_out < 1 || B < 1)
         return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: sizes must be positive");
     if (device < 0 || device >= MAX_DEVICES) return static_fail(err, err_len, PAC_ERR_INVALID_ARG, "pac_eval_logits_static: bad device %d", device);
-    if ((size_t)(d + n_out + 32) * sizeof(float) > 48 * 1024)
-        return static_fail(err, err_len, PAC_ERR_UNSUPPORTED, "pac_eval_logits_static: d + C = %d is beyond the head kernel's shared memory", d + n_out);
+    if (((size_t)d + (size_t)n_out + 32) * sizeof(float) > 48 * 1024)
+        return static_fail(err, err_len, PAC_ERR_UNSUPPORTED, "pac_eval_logits_static: d + C is beyond the head kernel's shared memory");
+    // every factor is bounded by the scratch size before any product is formed, so none can wrap:
+    // afterwards B*S*r*L*4 <= 8 MiB, B*S fits an int and the grid dimensions (L, B*S/64) are legal
+    {
+        const size_t cap = (size_t)PAC_STATIC_SCRATCH_BYTES / sizeof(float);
+        size_t prod = 1;
+        const long long factors[4] = {B, S, r, L};
+        for (long long f : factors) {
+            if ((size_t)f > cap / prod)
+                return static_fail(err, err_len, PAC_ERR_UNSUPPORTED,
+                                   "pac_eval_logits_static: L=%d B=%d S=%d r=%d needs more scratch than the fixed array holds (%u bytes)",
+                                   L, B, S, r, (unsigned)PAC_STATIC_SCRATCH_BYTES);
+            prod *= (size_t)f;
+        }
+        if (L > 65535 || (size_t)B * (size_t)d > cap)
+            return static_fail(err, err_len, PAC_ERR_UNSUPPORTED, "pac_eval_logits_static: L or B*d too large");
+    }
     // scratch layout: u | a | pooled_a | hbar_b | iota, each block rounded up to 256 bytes
     const size_t Mr = (size_t)B * S * r;
     const size_t o_u = 0, o_a = o_u + up256(sizeof(float) * Mr * L), o_p = o_a + up256(sizeof(float) * Mr * L);
@@ -1419,6 +1491,13 @@ extern "C" pac_status pac_eval_logits_static(int device, void* cuda_stream, cons
         return static_fail(err, err_len, PAC_ERR_UNSUPPORTED,
                            "pac_eval_logits_static: L=%d B=%d S=%d r=%d d=%d needs %zu bytes of scratch, the fixed array holds %u",
                            L, B, S, r, d, need, (unsigned)PAC_STATIC_SCRATCH_BYTES);
+    // the caller's current device is put back before returning
+    struct DeviceGuard {
+        int prev = -1;
+        ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+    } guard;
+    int cur = -1;
+    if (cudaGetDevice(&cur) == cudaSuccess && cur != device) guard.prev = cur;
     cudaError_t e = cudaSetDevice(device);
     if (e != cudaSuccess) return static_fail(err, err_len, PAC_ERR_CUDA, "pac_eval_logits_static: cudaSetDevice: %s", cudaGetErrorString(e));
     unsigned char* base;

@@ -4,7 +4,10 @@
 #include <cuda_bf16.h>
 #include <cstdint>
 #include <cstdio>
+#include <map>
+#include <mutex>
 #include <string>
+#include <utility>
 
 #include "pac.h"
 
@@ -16,7 +19,11 @@ __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(bf16 x) { return __bfloat162float(x); }
 
 // Device-side status words (one small array per context).
-enum { ST_CLAMPED_IDS = 0, ST_TIMEOUT = 1, ST_WORDS = 4 };
+// ST_SKIPPED_STEPS: optimizer updates that were left out because ST_TIMEOUT was already set when they ran.
+enum { ST_CLAMPED_IDS = 0, ST_TIMEOUT = 1, ST_SKIPPED_STEPS = 2, ST_WORDS = 4 };
+__device__ __forceinline__ bool status_timed_out(const unsigned* status) {
+    return status && *reinterpret_cast<const volatile unsigned*>(status + ST_TIMEOUT) != 0u;
+}
 
 // Sample id of batch row b, clamped into [0, N) so that no kernel can read outside
 // the cache even if a device-resident id is bad; clamps are counted.
@@ -27,6 +34,23 @@ __device__ __forceinline__ long long safe_id(const int* __restrict__ ids, int b,
         id = id < 0 ? 0 : N - 1;
     }
     return id;
+}
+
+// Dynamic shared memory above 48 KB needs an opt-in per kernel, and the attribute belongs to the
+// device the call is made on.  Several contexts (other shapes, other devices) share the kernels, so
+// the largest size granted so far is kept per (device, kernel) and never lowered.
+inline cudaError_t smem_opt_in(const void* kernel, size_t bytes) {
+    static std::mutex mu;
+    static std::map<std::pair<int, const void*>, size_t> granted;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    size_t& g = granted[std::make_pair(dev, kernel)];
+    if (bytes <= g) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) g = bytes;
+    return e;
 }
 
 struct Dims {

@@ -244,7 +244,7 @@ inline FusedFwdPlan fused_fwd_plan(const Dims& dm, int max_smem) {
 // How many of the plan's clusters can be resident at once (0 when the query fails).
 template <int ACT>
 inline int fused_fwd_max_clusters_act(const FusedFwdPlan& pl) {
-    if (cudaFuncSetAttribute(fwd_cluster_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem) != cudaSuccess) {
+    if (smem_opt_in((const void*)fwd_cluster_kernel<ACT>, pl.smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -273,11 +273,9 @@ inline int fused_fwd_max_clusters(const FusedFwdPlan& pl, int act) {
 template <int ACT>
 inline cudaError_t fused_fwd_launch_act(const FusedFwdPlan& pl, const CUtensorMap& map_cache, const CUtensorMap& map_w,
                                         const FusedFwdParams& fp, cudaStream_t stream) {
-    static size_t opted_in = 0;                      // dynamic shared memory the kernel has been allowed so far
-    if (pl.smem > opted_in) {
-        cudaError_t e = cudaFuncSetAttribute(fwd_cluster_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+    {
+        cudaError_t e = smem_opt_in((const void*)fwd_cluster_kernel<ACT>, pl.smem);
         if (e != cudaSuccess) return e;
-        opted_in = pl.smem;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(fp.mid.B * pl.mp.G), 1, 1);

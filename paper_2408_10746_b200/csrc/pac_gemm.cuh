@@ -259,12 +259,10 @@ inline bool lm_ce_stream_supported(int V, int max_smem) {
 // rows [M][V] fp32 -> loss_row [M], dlog16 [M][V] (may be null: loss only)
 inline cudaError_t lm_ce_stream_launch(cudaStream_t stream, int sms, const float* logits, const int* ids, long long N,
                                        const int* targets, int S, int V, int M, float* loss_row, bf16* dlog16, unsigned* status) {
-    static size_t opted_in = 0;
     const size_t smem = (size_t)V * 4;
-    if (smem > opted_in) {
-        cudaError_t e = cudaFuncSetAttribute(lm_ce_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    {
+        cudaError_t e = smem_opt_in((const void*)lm_ce_stream_kernel, smem);
         if (e != cudaSuccess) return e;
-        opted_in = smem;
     }
     const int grid = M < sms ? M : sms;
     lm_ce_stream_kernel<<<grid, CE_THREADS, smem, stream>>>(logits, ids, N, targets, S, V, M, loss_row, dlog16, status);
@@ -304,7 +302,7 @@ inline pac_status gemm_plan_create(GemmPlan& gp, int device, const bf16* A, long
         cuuint32_t box[2] = {GT_BK, GT_BN};
         if (!make_map(&gp.map_b, B, 2, dims, str, box)) return PAC_ERR_UNSUPPORTED;
     }
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM) != cudaSuccess) {
+    if (smem_opt_in((const void*)gemm_tc_kernel, GT_SMEM) != cudaSuccess) {
         tensor_err() = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
         cudaGetLastError();
         return PAC_ERR_CUDA;

@@ -457,11 +457,15 @@ struct FinalizeParams {
     int adam;
     float *params, *m, *v;
     pac_adamw hp; float bc1, bc2;
+    float grad_scale;                                        // factor on every gradient entering the fused update
     bf16* wdT;                                               // [L][2][d][r] bf16 hi/lo shadow of W_down (may be null)
     // Ids of the NEXT step (pac_train_step_async): if the host has already published them in its page-locked
     // ring (tag == next_seq), block 0 copies them to device memory, off every kernel's critical path.
     const int* next_host_ids; const unsigned* next_host_tag; unsigned next_seq; int next_n;
     int* next_dev_ids; unsigned* next_dev_tag;
+    // Device status words: when a bounded wait of this or an earlier step has run out, the gradients
+    // are not trustworthy, so nothing is written to the gradients, parameters or moments.
+    unsigned* status;
 };
 
 __device__ __forceinline__ unsigned ld_acquire_sys(const unsigned* p) {
@@ -496,18 +500,23 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     // Block 0 (dlambda and the mean loss) needs only what the forward half left behind, which is
     // complete whenever this kernel runs (see above): it does not wait for the second pass at all, so a loss
     // that goes straight to host memory is on its way long before the step ends.
+    // Set by a wait that ran out in this step's forward half or in any earlier step since the last
+    // pac_sync (the forward half has completed whenever this kernel runs); a wait that runs out in this
+    // step's second pass is seen by the W_down blocks behind their own wait below.
+    const bool dead = status_timed_out(f.status);
     if (blk < 0) {
         // dlambda_l (one warp per layer, lanes over the per-block partials, fixed
         // shuffle order) and the mean loss
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-        for (int l = warp; l < f.L; l += nw) {
+        if (dead && f.adam && threadIdx.x == 0) atomicAdd(&f.status[ST_SKIPPED_STEPS], 1u);
+        for (int l = warp; l < f.L && !dead; l += nw) {
             float acc = 0.f;
             for (int k = lane; k < f.lam_blocks; k += 32) acc += f.lam_part[(long long)l * f.lam_blocks + k];
             acc = warp_sum(acc);
             if (lane == 0) {
                 const long long i = lay.lam + l;
                 f.grads[i] = acc;
-                if (f.adam) adamw_element(f.params, f.m, f.v, i, acc, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+                if (f.adam) adamw_element(f.params, f.m, f.v, i, acc * f.grad_scale, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
             }
         }
         if (warp == nw - 1) {
@@ -521,9 +530,13 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
             const unsigned tag = ld_acquire_sys(f.next_host_tag);
             if (tag == f.next_seq) {
                 for (int b = lane; b < f.next_n; b += 32) f.next_dev_ids[b] = *reinterpret_cast<const volatile int*>(f.next_host_ids + b);
-                __threadfence();
+                // publish: the warp barrier orders every lane's id stores before lane 0, whose fence then
+                // comes between them and the tag
                 __syncwarp();
-                if (lane == 0) atomicExch(f.next_dev_tag, f.next_seq);
+                if (lane == 0) {
+                    __threadfence();
+                    atomicExch(f.next_dev_tag, f.next_seq);
+                }
             }
         }
         return;
@@ -532,7 +545,7 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         // head parameters: like block 0 they need only the forward half's per-sample vectors, so these blocks
         // finish (and make room for the W_down blocks) while the second pass still runs
         const long long i = lay.lam + (long long)blk * blockDim.x + threadIdx.x;
-        if (i >= lay.total) return;
+        if (i >= lay.total || dead) return;
         float g;
         if (i < lay.w_up) return;                            // lambda is handled by block 0
         if (i < lay.w_head) {
@@ -553,14 +566,14 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
             for (int b = 0; b < f.B; ++b) g += f.dlogits[(long long)b * f.C + c];
         }
         f.grads[i] = g;
-        if (f.adam) adamw_element(f.params, f.m, f.v, i, g, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        if (f.adam) adamw_element(f.params, f.m, f.v, i, g * f.grad_scale, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
         return;
     }
     pdl_wait();
     {
         // W_down block, four consecutive elements per thread
         const long long i = i_wd;
-        if (i >= lay.lam) return;
+        if (i >= lay.lam || status_timed_out(f.status)) return;
         float4 g4;
         if (f.splits > 1) {
             g4 = *reinterpret_cast<const float4*>(f.dw_part + i);
@@ -572,7 +585,10 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         } else {
             g4 = *reinterpret_cast<const float4*>(f.grads + i);
         }
-        if (f.adam) adamw_w_down4_loaded(f.params, f.m, f.v, i, p4, m4, v4, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        if (f.adam) {
+            g4.x *= f.grad_scale; g4.y *= f.grad_scale; g4.z *= f.grad_scale; g4.w *= f.grad_scale;
+            adamw_w_down4_loaded(f.params, f.m, f.v, i, p4, m4, v4, g4, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        }
         return;
     }
 }
@@ -642,12 +658,9 @@ inline MidPlan mid_plan(const Dims& dm) {
 
 template <int ACT, typename DU, int GPT, bool SMEM_STATE>
 inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
-    static bool opted_in = false;                    // dynamic shared memory above 48 KB needs an opt-in per kernel
-    if (!opted_in) {
-        cudaError_t e = cudaFuncSetAttribute(mid_cls_kernel<ACT, DU, GPT, SMEM_STATE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)MID_SMEM_BUDGET);
+    {
+        cudaError_t e = smem_opt_in((const void*)mid_cls_kernel<ACT, DU, GPT, SMEM_STATE>, MID_SMEM_BUDGET);
         if (e != cudaSuccess) return e;
-        opted_in = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.B * mp.G), 1, 1);

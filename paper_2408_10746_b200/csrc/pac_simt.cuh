@@ -530,17 +530,29 @@ __device__ __forceinline__ void adamw_w_down4_loaded(float* __restrict__ p, floa
 
 // wd_blocks leading blocks take the W_down block four elements per thread (0 when its size is
 // not a multiple of 4); the remaining blocks take everything else one element per thread.
+// grad_scale multiplies every gradient on its way into the update (1 for a single device; 1/world
+// when the gradient buffer holds the SUM over data-parallel ranks); the buffer itself is not changed.
 __global__ void adamw_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,
                              float* __restrict__ v, long long n, ParamLayout lay, pac_adamw hp, float bc1,
-                             float bc2, bf16* __restrict__ wdT, int d, int r, int wd_blocks) {
+                             float bc2, bf16* __restrict__ wdT, int d, int r, int wd_blocks, unsigned* status,
+                             float grad_scale) {
+    // gradients computed after a bounded wait ran out are not trustworthy: leave the state alone
+    if (status_timed_out(status)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&status[ST_SKIPPED_STEPS], 1u);
+        return;
+    }
     if ((int)blockIdx.x < wd_blocks) {
         const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-        if (i < lay.lam) adamw_w_down4(p, m, v, i, *reinterpret_cast<const float4*>(g + i), hp, bc1, bc2, wdT, d, r);
+        if (i < lay.lam) {
+            float4 g4 = *reinterpret_cast<const float4*>(g + i);
+            g4.x *= grad_scale; g4.y *= grad_scale; g4.z *= grad_scale; g4.w *= grad_scale;
+            adamw_w_down4(p, m, v, i, g4, hp, bc1, bc2, wdT, d, r);
+        }
         return;
     }
     const long long i = (wd_blocks ? lay.lam : 0) + (long long)(blockIdx.x - wd_blocks) * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    adamw_element(p, m, v, i, g[i], lay, hp, bc1, bc2, wdT, d, r);
+    adamw_element(p, m, v, i, g[i] * grad_scale, lay, hp, bc1, bc2, wdT, d, r);
 }
 
 // bf16 hi/lo shadow of W_down from the fp32 master, same [d][r] order:

@@ -59,27 +59,30 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait (about one second of wall time).  Returns false when the limit ran out or
 // another role of this CTA gave up; the caller then stops issuing work.
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                            unsigned long long limit_ns) {
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
     if (status) atomicAdd(&status[ST_TIMEOUT], 1u);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status);
+    return mbar_wait_slow(bar, parity, abort_flag, status, limit_ns);
 }
 // The same for a whole warp: lane 0 waits, every lane gets the same answer.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status) {
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                               unsigned long long limit_ns = WAIT_LIMIT_NS) {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, limit_ns) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
 }
@@ -183,6 +186,36 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Self-test of the bounded-wait discipline: one CTA allocates TMEM like the pipeline kernels, waits
+// on an mbarrier that nobody will ever arrive at, and, once limit_ns have passed, leaves exactly the
+// way the pipeline kernels leave after an abort (status word, abort flag, drain, TMEM release).
+// result[0] = 1 if the wait reported expiry, result[1] = the abort flag.
+__global__ void __launch_bounds__(64, 1) selftest_wait_expiry_kernel(unsigned* status, unsigned long long limit_ns, unsigned* result) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ int abort_sh;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        abort_sh = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), 32u); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    volatile int* abort_flag = &abort_sh;
+    if (warp == 0) {
+        const bool ok = mbar_wait_warp(smem_u32(&bar), 0, abort_flag, status, limit_ns);
+        if (threadIdx.x == 0) result[0] = ok ? 0u : 1u;
+    }
+    tc_fence_before();
+    __syncthreads();
+    drain_after_abort(abort_flag);
+    if (threadIdx.x == 0) result[1] = (unsigned)abort_sh;
+    if (warp == 1) tmem_dealloc(tmem_base_sh, 32u);
+}
 
 // Shared-memory matrix descriptor for tcgen05.mma, 128-byte swizzle.
 //   bits [0,14) start address >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte
@@ -696,8 +729,8 @@ inline pac_status tensor_plan_create(TensorPlan& tp, int device, const bf16* cac
     tp.dw_elems = (long long)dm.L * dm.d * dm.r;
     *part_floats = b.splits > 1 ? tp.dw_elems * b.splits : 0;
 
-    if (cudaFuncSetAttribute(down_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tp.smem_fwd) != cudaSuccess ||
-        cudaFuncSetAttribute(dw_down_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tp.smem_bwd) != cudaSuccess) {
+    if (smem_opt_in((const void*)down_fwd_tc_kernel, tp.smem_fwd) != cudaSuccess ||
+        smem_opt_in((const void*)dw_down_tc_kernel, tp.smem_bwd) != cudaSuccess) {
         tensor_err() = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
         cudaGetLastError();
         return PAC_ERR_CUDA;

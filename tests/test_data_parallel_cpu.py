@@ -30,10 +30,20 @@ class OracleLocal:
         self._p = torch.from_numpy(po.flatten(self.tr.P))
         self._g = torch.zeros_like(self._p)
 
-    def train_step(self, ids):
+    def train_step(self, ids, loss_slot):
         loss = self.tr.train_step(ids)
         self._g.copy_(torch.from_numpy(po.flatten(self.tr.grads)))
-        return loss
+        loss_slot.fill_(loss)
+
+    def set_grad_scale(self, scale):
+        self.scale = scale
+
+    def new_loss_buffer(self, n):
+        return torch.zeros(n, dtype=torch.float64)
+
+    def stream_context(self):
+        import contextlib
+        return contextlib.nullcontext()
 
     def grad_buffer(self):
         return self._g
@@ -45,7 +55,8 @@ class OracleLocal:
         self.tr.P = po.unflatten(self._p.numpy().copy(), SPEC.L, SPEC.d, SPEC.r, SPEC.n_out)
 
     def adam_step(self, hp):
-        self.tr.grads = po.unflatten(self._g.numpy().copy(), SPEC.L, SPEC.d, SPEC.r, SPEC.n_out)
+        # the factor a device-side optimizer applies while reading the (summed) gradient buffer
+        self.tr.grads = po.unflatten(self._g.numpy().copy() * self.scale, SPEC.L, SPEC.d, SPEC.r, SPEC.n_out)
         self.tr.hp = hp
         self.tr.adam_step()
         self._p.copy_(torch.from_numpy(po.flatten(self.tr.P)))
@@ -60,13 +71,103 @@ def _worker(rank, world, port, out):
     flat = pi.random_params(SPEC, 3 if rank == 0 else 9)
     dp = DataParallel(OracleLocal(flat))
     perm = pi.epoch_permutation(SPEC.N, 2)
-    losses = []
     for s in range(STEPS):
         gids = perm[s * SPEC.B:(s + 1) * SPEC.B].tolist()
-        losses.append(dp.train_step(shard_ids(gids, rank, world)))
+        assert dp.train_step(shard_ids(gids, rank, world)) is None
         dp.adam_step(po.AdamW())
+    losses = dp.epoch_losses().tolist()
     out[rank] = (losses, dp.local.param_buffer().numpy().copy())
     dist.destroy_process_group()
+
+
+class RecordingLocal:
+    """A local trainer that computes nothing and records what the orchestrator asks of it."""
+
+    def __init__(self, n, rank):
+        self.log, self.rank = [], rank
+        self._p = torch.full((n,), float(rank + 1))
+        self._g = torch.zeros(n)
+
+    def train_step(self, ids, loss_slot):
+        self.log.append(("train_step", tuple(ids)))
+        self._g.fill_(float(self.rank + 1))           # rank-dependent "gradient"
+        loss_slot.fill_(10.0 * (self.rank + 1) + len(self.log))
+
+    def grad_buffer(self):
+        return self._g
+
+    def param_buffer(self):
+        return self._p
+
+    def params_changed(self):
+        self.log.append(("params_changed",))
+
+    def set_grad_scale(self, scale):
+        self.log.append(("set_grad_scale", scale))
+
+    def adam_step(self, hp):
+        self.log.append(("adam_step", self._g[:1].clone()))   # what the optimizer would read (kept as a tensor)
+
+    def new_loss_buffer(self, n):
+        return torch.zeros(n)
+
+    def stream_context(self):
+        import contextlib
+        return contextlib.nullcontext()
+
+
+def _recording_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2408_10746_b200.data_parallel import DataParallel
+    local = RecordingLocal(5, rank)
+    dp = DataParallel(local)
+    # from here on a step must not read anything back to the host: count every route a tensor has
+    reads = []
+    patched = {}
+    for name in ("item", "tolist", "cpu", "numpy", "__float__", "__int__", "__bool__"):
+        orig = getattr(torch.Tensor, name)
+        patched[name] = orig
+
+        def spy(self, *a, _orig=orig, _name=name, **k):
+            reads.append(_name)
+            return _orig(self, *a, **k)
+        setattr(torch.Tensor, name, spy)
+    try:
+        for s in range(3):
+            assert dp.train_step([s, s + 1]) is None
+            dp.adam_step(None)
+        reads_in_steps = list(reads)
+    finally:
+        for name, orig in patched.items():
+            setattr(torch.Tensor, name, orig)
+    losses = dp.epoch_losses().tolist()
+    log = [(e[0], float(e[1][0])) if e[0] == "adam_step" else e for e in local.log]
+    out[rank] = (log, reads_in_steps, losses, local.param_buffer().tolist())
+    dist.destroy_process_group()
+
+
+def test_orchestration_order_and_no_host_read_per_step():
+    """Two ranks with recording trainers: parameters are broadcast once, the 1/world factor is handed
+    to the optimizer (not applied in Python), every step is train_step -> all-reduce -> adam_step with
+    the SUM of the ranks' gradients in the buffer, and no tensor is read back to the host until the
+    losses of the epoch are asked for."""
+    world, port = 2, 31000 + os.getpid() % 2000
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_recording_worker, args=(world, port, out), nprocs=world, join=True)
+    for rank in range(world):
+        log, reads_in_steps, losses, params = out[rank]
+        assert reads_in_steps == []
+        assert params == [1.0] * 5                              # rank 0's parameters everywhere
+        assert log[0] == ("params_changed",) and log[1] == ("set_grad_scale", 0.5)
+        steps = log[2:]
+        assert [e[0] for e in steps] == ["train_step", "adam_step"] * 3
+        assert all(e == ("adam_step", 3.0) for e in steps[1::2])          # 1 + 2: the sum, unscaled
+        assert [e[1] for e in steps[0::2]] == [(0, 1), (1, 2), (2, 3)]
+        # mean over ranks of the per-rank losses 10*(rank+1) + k
+        assert np.allclose(losses, [15.0 + k for k in (3, 5, 7)])
 
 
 def test_two_ranks_match_single_process_oracle():

@@ -6,6 +6,8 @@ import pytest
 import torch
 
 import pac_inputs as pi
+from oracle import pac_oracle as po
+from tests.common import rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -60,12 +62,30 @@ def test_host_cache_steps_match_device_cache(spec):
     dev.eval_logits(ids, la); host.eval_logits(ids, lb)
     dev.sync(); host.sync()
     assert torch.equal(la, lb)
+    # the staged path against the oracle directly (not only against the resident path): logits, then the
+    # loss and every gradient block of the first step; fp32 caches at 1e-4, bf16 caches at the tensor
+    # path's bounds
+    flat = pi.random_params(spec, 3)
+    C = spec.n_out if spec.head == "cls" else None
+    P = po.unflatten(flat, spec.L, spec.d, spec.r, C)
+    H = pi.cache_samples(spec, 0, ids, "cpu").float().numpy()
+    W_lm = pi.lm_head(spec, 0, "cpu").float().numpy() if spec.head == "lm" else None
+    tight = spec.dtype == "f32"
+    assert rel_l2(lb.cpu().numpy(), po.eval_logits(P, H, 0, W_lm)) < (1e-4 if tight else 3e-3)
+    labels_np = pi.labels(spec, 0, "cpu").numpy().astype(np.int64)
     # steps, partial batch included
     for i in range(5):
         step_ids = perm[i * B:(i + 1) * B] if i != 2 else perm[i * B:i * B + max(1, B // 2)]
         l1, l2 = dev.train_step(step_ids), host.train_step(step_ids)
         assert l1 == l2
         assert np.array_equal(dev.get_grads(), host.get_grads())
+        if i == 0:
+            Hs = pi.cache_samples(spec, 0, step_ids.tolist(), "cpu").float().numpy()
+            lab = labels_np[step_ids]
+            ref_loss, ref_g, _ = (po.loss_and_grads_cls(P, Hs, lab) if spec.head == "cls"
+                                  else po.loss_and_grads_lm(P, Hs, lab, W_lm))
+            assert abs(l2 - ref_loss) <= (1e-4 if tight else 2e-2) * abs(ref_loss)
+            assert rel_l2(host.get_grads(), po.flatten(ref_g)) < (1e-4 if tight else 1e-2)
         dev.adam_step(hp); host.adam_step(hp)
     assert np.array_equal(dev.get_params(), host.get_params())
 

@@ -83,7 +83,7 @@ def test_params_and_permutation():
 
 def test_golden_first_values():
     """A few stored values (written by tests/golden/make_inputs_golden.py from this
-    module alone) so that the generator cannot drift unnoticed between rounds."""
+    module alone) so that a change to the generator cannot go unnoticed."""
     import json, os
     with open(os.path.join(os.path.dirname(__file__), "golden", "inputs_golden.json")) as f:
         gold = json.load(f)

@@ -42,6 +42,14 @@ def test_gather_bit_exact(spec):
         assert po.gather(ref.permute(1, 0, 2, 3).float().numpy(), range(len(ids))).shape[0] == len(ids)
 
 
+def test_generator_is_bit_identical_on_both_devices():
+    """The oracle's slabs may be generated on either device: same bits (outlier channels included)."""
+    for spec, ids in ((pi.CONFIGS["t5_large"], [0, 4095]), (pi.CONFIGS["llama_7b"].scaled(S=64), [255]), (TINY, [3, 200])):
+        a = pi.cache_samples(spec, 0, ids, "cuda").cpu()
+        b = pi.cache_samples(spec, 0, ids, "cpu")
+        assert a.view(torch.uint8).flatten().equal(b.view(torch.uint8).flatten())
+
+
 # ------------------------------------------------------------------ loss + gradients
 def check_loss_grads(case, ids, act, loss_tol, grad_tol, force_simt=False, seed=3):
     spec = case.spec
@@ -120,13 +128,23 @@ def test_zero_up_projection_is_head_only(tiny):
 
 
 # ------------------------------------------------------------------ trajectories
+# Bound on the relative L2 error of the 10-step UPDATE p_10 - p_0 (the initial values removed).  Adam
+# normalises g / sqrt(v), so an entry whose gradient sits at the bf16 noise floor moves by +-lr with a
+# sign that depends on rounding.  Observed on the full-size classifier workloads (hi+lo weights, bf16 du):
+# 2.6e-2 (T5-Base), 2.4e-2 (BART-Large), 1.6e-2 (T5-Large); with the frozen LM head, whose y and dlogits
+# also enter their GEMMs rounded to bf16, 4.9e-2.
+UPDATE_TOL = 5e-2
+UPDATE_TOL_LM = 8e-2
+
+
 def run_trajectory(case, steps, act=0, force_simt=False, hp=None, kernel_path=0):
     import paper_2408_10746_b200 as pac
     spec = case.spec
     hp = hp or po.AdamW()
     ctx = case.context(act=act, force_simt=force_simt, kernel_path=kernel_path)
     flat0 = ctx.get_params()
-    perm = pi.epoch_permutation(spec.N, 2)
+    n_epochs = 1 + steps * spec.B // spec.N
+    perm = np.concatenate([pi.epoch_permutation(spec.N, 2, epoch=e) for e in range(n_epochs)])
     batches = [perm[i * spec.B:(i + 1) * spec.B].tolist() for i in range(steps)]
     tr, remap = case.oracle_trainer(flat0, act, hp, ids_universe=[i for b in batches for i in b])
     losses, ref_losses = [], []
@@ -149,9 +167,10 @@ def test_tiny_fp32_ten_adamw_steps(tiny):
 
 def test_bf16_ten_steps_plain_kernels():
     case = Case(RAGGED_BF16)
-    _, losses, ref_losses, p, ref_p, _ = run_trajectory(case, 4, force_simt=True)
+    _, losses, ref_losses, p, ref_p, p0 = run_trajectory(case, 10, force_simt=True)
     assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses))
     assert rel_l2(p, ref_p) < 1e-2
+    assert rel_l2(p - p0, ref_p - p0) < UPDATE_TOL
 
 
 # ------------------------------------------------------------------ runtime behaviour
@@ -356,7 +375,7 @@ def test_tensor_path_ten_steps_t5_base_shape(kernel_path):
     assert ctx.kernel_path() == ("tensor+fused_forward" if kernel_path == 3 else "tensor")
     assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses))
     assert rel_l2(p, ref_p) < 1e-2
-    assert rel_l2(p - p0, ref_p - p0) < 0.1          # the update itself is reproduced, not only the initial values
+    assert rel_l2(p - p0, ref_p - p0) < UPDATE_TOL   # the update itself is reproduced, not only the initial values
 
 
 # ------------------------------------------------------------------ full-size launch configurations
@@ -376,6 +395,15 @@ class SparseCase(Case):
         self.labels_np = pi.labels(spec, seed, "cpu").numpy().astype(np.int64)
         self.lm_np = pi.lm_head(spec, seed, "cpu").float().numpy() if spec.head == "lm" else None
         self.cache_np = None
+
+    def H(self, ids):
+        """Oracle-side slabs, regenerated on the GPU (bit-identical to the CPU generator, far faster
+        at these sizes) and copied to the host."""
+        ids = list(ids)
+        out = np.empty((len(ids), self.spec.L, self.spec.S, self.spec.d), dtype=np.float32)
+        for i in range(0, len(ids), 4):
+            out[i:i + 4] = pi.cache_samples(self.spec, self.seed, ids[i:i + 4], "cuda").float().cpu().numpy()
+        return out
 
 
 @pytest.mark.parametrize("name,kernel_path", [("t5_base", 0), ("t5_base", 2), ("t5_base", 3), ("bart_large", 0), ("t5_large", 0)])
@@ -397,6 +425,63 @@ def test_full_size_step_matches_oracle(name, kernel_path):
     ctx.sync()
     ref = pi.cache_samples(spec, 0, ids[:4], "cpu").permute(1, 0, 2, 3).contiguous()
     assert out.cpu().view(torch.uint8).flatten().equal(ref.view(torch.uint8).flatten())
+
+
+class LazyCache:
+    """Oracle-side stand-in for a full-size cache: indexing with sample ids regenerates those slabs
+    from the seeded generator (on the GPU, whose values are bit-identical to the CPU's, then copied),
+    so ten minibatches of a 51 GB cache never sit in host memory at once."""
+
+    def __init__(self, spec, seed=0):
+        self.spec, self.seed = spec, seed
+        self.shape = (spec.N, spec.L, spec.S, spec.d)
+
+    def __getitem__(self, ids):
+        ids = [int(i) for i in np.asarray(ids).ravel()]
+        out = np.empty((len(ids),) + self.shape[1:], dtype=np.float32)
+        for i in range(0, len(ids), 4):
+            out[i:i + 4] = pi.cache_samples(self.spec, self.seed, ids[i:i + 4], "cuda").float().cpu().numpy()
+        return out
+
+
+def full_size_trajectory(spec, steps, B):
+    """`steps` fused train steps (pac_train_epoch, the call the benchmark loops over) of B samples on
+    a cache of the full size and strides, from the seeded initial state, against the oracle's
+    trainer on the same minibatches."""
+    import paper_2408_10746_b200 as pac
+    free, _ = torch.cuda.mem_get_info()
+    if spec.cache_bytes + (8 << 30) > free:
+        pytest.skip("cache does not fit this device")
+    perm = pi.epoch_permutation(spec.N, 2)[:steps * B].copy()
+    perm[0], perm[-1] = 0, spec.N - 1                      # both ends of the cache are touched
+    case = SparseCase(spec, perm.tolist())
+    ctx = case.context(max_batch=spec.B)
+    p0 = ctx.get_params()
+    assert np.array_equal(p0, pi.init_params(spec, 1))
+    hp = po.AdamW()
+    losses = ctx.train_epoch(perm, B, pac.AdamW(hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay))
+    p = ctx.get_params()
+    tr = po.Trainer(LazyCache(spec), case.labels_np, case.oracle_params(p0), 0, case.lm_np, hp)
+    ref_losses = []
+    for i in range(steps):
+        ref_losses.append(tr.train_step(perm[i * B:(i + 1) * B]))
+        tr.adam_step()
+    ref_p = po.flatten(tr.P)
+    return np.asarray(losses), np.asarray(ref_losses), p, ref_p, p0
+
+
+@pytest.mark.parametrize("name", ["t5_base", "bart_large", "t5_large"])
+def test_full_size_ten_step_trajectory(name):
+    """Every classifier workload at its full N, L, S, d, r and full B: 10 AdamW steps from the
+    seeded initial state, per-step loss within 2e-2 and the parameter vector within 1e-2 relative L2
+    of the oracle's."""
+    spec = pi.CONFIGS[name]
+    losses, ref_losses, p, ref_p, p0 = full_size_trajectory(spec, 10, spec.B)
+    assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses)), (losses, ref_losses)
+    assert rel_l2(p, ref_p) < 1e-2, rel_l2(p, ref_p)
+    assert rel_l2(p - p0, ref_p - p0) < UPDATE_TOL, rel_l2(p - p0, ref_p - p0)
+    print(f"{name}: params rel L2 {rel_l2(p, ref_p):.2e}, update rel L2 {rel_l2(p - p0, ref_p - p0):.2e}, "
+          f"max loss err {np.max(np.abs(losses - ref_losses) / np.abs(ref_losses)):.2e}")
 
 
 # ------------------------------------------------------------------ frozen LM head on the tensor cores
@@ -427,15 +512,32 @@ def test_lm_head_tensor_path_eval_logits():
 
 
 def test_full_size_llama_step_matches_oracle():
-    """LLaMA-7B-shaped cache (L=32, S=512, d=4096, V=32000) at full strides; two samples of the
-    batch of 16 are run so that the oracle finishes in seconds."""
+    """LLaMA-7B-shaped cache (L=32, S=512, d=4096, V=32000) at full strides and the full batch of 16
+    (M = 8192 rows: the launch geometry the benchmark times), one step against the oracle."""
     spec = pi.CONFIGS["llama_7b"]
     free, _ = torch.cuda.mem_get_info()
-    if spec.cache_bytes + (8 << 30) > free:
+    if spec.cache_bytes + (12 << 30) > free:
         pytest.skip("cache does not fit this device")
-    ids = [spec.N - 1, 0]
+    ids = pi.epoch_permutation(spec.N, 2)[:spec.B].tolist()
+    ids[0], ids[-1] = spec.N - 1, 0
     case = SparseCase(spec, ids)
     tc_check(spec, spec.B, 0, ids=ids, case=case, head_tol=5e-3)
+
+
+LLAMA_TRAJECTORY_B = 4
+
+
+def test_llama_ten_step_trajectory():
+    """10 AdamW steps on the LLaMA-7B-shaped cache (full strides, frozen 32000 x 4096 head) with
+    minibatches of 4 samples (M = 2048 rows): the largest batch whose ten oracle steps (about 1.2
+    TFLOP each in fp32 on the host) finish in a few minutes.  The full-batch geometry is pinned by the
+    single step above."""
+    spec = pi.CONFIGS["llama_7b"]
+    losses, ref_losses, p, ref_p, p0 = full_size_trajectory(spec, 10, LLAMA_TRAJECTORY_B)
+    assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses)), (losses, ref_losses)
+    assert rel_l2(p, ref_p) < 1e-2, rel_l2(p, ref_p)
+    assert rel_l2(p - p0, ref_p - p0) < UPDATE_TOL_LM, rel_l2(p - p0, ref_p - p0)
+    print(f"llama_7b: params rel L2 {rel_l2(p, ref_p):.2e}, update rel L2 {rel_l2(p - p0, ref_p - p0):.2e}")
 
 
 def test_tensor_path_epoch_equals_step_loop():
@@ -552,10 +654,95 @@ def test_device_buffer_views_and_single_rank_data_parallel(tiny):
         created = True
     try:
         dp = DataParallel(PacLocalTrainer(ctx))
-        loss = dp.train_step(ids)
+        assert dp.train_step(ids) is None
         assert np.array_equal(grads.cpu().numpy(), ctx.get_grads())
         dp.adam_step(hp)
+        loss = float(dp.epoch_losses()[0])
     finally:
         if created:
             dist.destroy_process_group()
     assert loss == ref_loss and np.array_equal(ctx.get_params(), ref.get_params())
+    # the gradient factor of data-parallel training: halving every gradient leaves Adam's first step
+    # unchanged up to rounding (the update is g / |g|), and the buffer keeps its values
+    half = tiny.context()
+    half.set_params(pi.random_params(TINY, 3))
+    half.set_grad_scale(0.5)
+    half.train_step(ids)
+    g_before = half.get_grads()
+    half.adam_step(hp)
+    assert np.array_equal(half.get_grads(), g_before)
+    m_half, v_half, _ = half.get_opt_state()
+    m_ref, v_ref, _ = ref.get_opt_state()
+    assert np.allclose(m_half, 0.5 * m_ref, rtol=1e-6, atol=0) and np.allclose(v_half, 0.25 * v_ref, rtol=1e-6, atol=0)
+    with pytest.raises(pac.PacError):
+        half.set_grad_scale(0.0)
+
+
+# ------------------------------------------------------------------ failure handling, several contexts
+@pytest.mark.parametrize("which", ["tensor_fused", "plain_fp32"])
+def test_wait_expiry_is_reported_once_and_leaves_the_state_alone(which, tiny):
+    """A bounded device-side wait that runs out (a self-test CTA waits 100 us on a barrier nobody
+    arrives at; nothing hangs, no product kernel is broken): steps enqueued behind it change neither
+    parameters nor moments nor the step counter, the next sync reports PAC_ERR_TIMEOUT exactly once,
+    and the step after that matches the oracle again (tensor memory was released, the context lives)."""
+    import paper_2408_10746_b200 as pac
+    if which == "tensor_fused":
+        spec = TC_BASE.scaled(N=32, name="tc_timeout")
+        case = Case(spec)
+    else:
+        spec, case = TINY, tiny
+    hp = pac.AdamW()
+    ctx = case.context()
+    flat = pi.random_params(spec, 3)
+    ctx.set_params(flat)
+    ids = list(range(spec.B))
+    ctx.train_step_async(ids, hp)                              # one healthy step first
+    ctx.sync()
+    p1, (m1, v1, step1) = ctx.get_params(), ctx.get_opt_state()
+    assert step1 == 1 and not np.array_equal(p1, flat)
+    ctx.selftest_wait_expiry(100_000)
+    ctx.train_step_async(ids, hp)                              # fused update behind the timeout
+    ctx.train_step(ids, want_loss=False)
+    ctx.adam_step(hp)                                          # separate update behind the timeout
+    with pytest.raises(pac.PacError) as e:
+        ctx.sync()
+    assert e.value.status_name == "PAC_ERR_TIMEOUT"
+    ctx.sync()                                                 # reported once
+    p2, (m2, v2, step2) = ctx.get_params(), ctx.get_opt_state()
+    assert step2 == 1 and np.array_equal(p2, p1) and np.array_equal(m2, m1) and np.array_equal(v2, v1)
+    # the context is healthy: the next step matches the oracle from the same state
+    loss = ctx.train_step(ids)
+    g = ctx.get_grads()
+    ref_loss, ref_g, _ = case.oracle_loss_grads(p1, ids, 0)
+    tight = spec.dtype == "f32"
+    assert abs(loss - ref_loss) <= (1e-4 if tight else 2e-2) * abs(ref_loss)
+    assert rel_l2(g, po.flatten(ref_g)) < (1e-4 if tight else 1e-2)
+    ctx.adam_step(hp)
+    assert ctx.get_opt_state()[2] == 2
+    with pytest.raises(pac.PacError):
+        ctx.selftest_wait_expiry(10)                           # limit outside the documented range
+
+
+def test_two_contexts_of_different_shapes_share_the_kernels():
+    """The shared-memory opt-in of a kernel is kept at the largest size any context asked for: a
+    second, smaller context must not take the first one's launches away."""
+    big_spec = pi.CONFIGS["t5_base"].scaled(N=16, B=4, name="t5_base_two_ctx")
+    small_spec = TC_BASE.scaled(name="tc_small_two_ctx", S=19, d=72, r=16)
+    big_case, small_case = Case(big_spec, materialize_cpu=False), Case(small_spec, materialize_cpu=False)
+    ids_big, ids_small = [0, 5, 15, 3], [0, 1, 2, 3]
+    results = []
+    for path in (0, 2):
+        a = big_case.context(kernel_path=path)
+        a.set_params(pi.random_params(big_spec, 3))
+        first = a.train_step(ids_big)
+        g_first = a.get_grads()
+        b = small_case.context(kernel_path=path)               # smaller pipelines, smaller shared memory
+        b.set_params(pi.random_params(small_spec, 3))
+        b.train_step(ids_small)
+        b.sync()
+        again = a.train_step(ids_big)                          # the first context still launches
+        a.sync()
+        assert again == first and np.array_equal(a.get_grads(), g_first)
+        results.append(first)
+        b.close(); a.close()
+    assert abs(results[0] - results[1]) <= 1e-5 * abs(results[1])

@@ -2,13 +2,14 @@
 not allocate device memory: its scratch is a fixed array inside the library.  Collected last on
 purpose, so that a run that stops at the first failure has already run every other test.
 
-Checked against the context-based pac_eval_logits on the same inputs, on two calls in a row (the
+Checked against the context-based pac_eval_logits and against the CPU oracle on the same inputs, on two calls in a row (the
 second with other ids and a smaller batch, so stale scratch from the first call would show)."""
 import numpy as np
 import pytest
 import torch
 
 import pac_inputs as pi
+from oracle import pac_oracle as po
 from tests.common import Case, rel_l2
 
 pytestmark = pytest.mark.gpu
@@ -32,6 +33,9 @@ def run_pair(spec, force_simt, tol):
         torch.cuda.synchronize()
         assert torch.isfinite(got).all()
         assert rel_l2(got.cpu().numpy(), want.cpu().numpy()) < tol
+        # and against the oracle itself, not only against the other CUDA entry point
+        ref = po.eval_logits(case.oracle_params(flat), case.H(ids), 0)
+        assert rel_l2(got.cpu().numpy(), ref) < tol
     ctx.close()
 
 
