@@ -115,6 +115,34 @@ pac_status pac_cache_register(pac_ctx* ctx, const void* dev_cache, int dtype, lo
 pac_status pac_cache_register_host(pac_ctx* ctx, const void* host_cache, int dtype, long long N, int L, int S, int d,
                                    const int* host_labels, int labels_per_sample);
 
+/* The same for a cache kept in a FILE (Section IV-B: the activations are recorded during the first
+ * epoch; Section V-B, storage cost analysis: they live on storage and are reloaded per micro-batch).
+ * `path` (host string) names a file written by pac_cache_writer_*: a 64-byte header (magic
+ * "PACCACHE", version, dtype, N, L, S, d, labels_per_sample), the cache [N][L][S][d], then, at the next
+ * multiple of 64 bytes, the int32 labels.
+ * The file is mapped read-only until pac_destroy and then treated as a host-resident cache
+ * (pageable memory: the copies of a step overlap the GPU work of the step before, the host waits for
+ * the page cache / storage).  Errors: PAC_ERR_INVALID_ARG for a missing, truncated or foreign file,
+ * PAC_ERR_NOMEM when the mapping fails, PAC_ERR_BAD_STATE after pac_adapter_init. */
+pac_status pac_cache_register_file(pac_ctx* ctx, const char* path);
+
+/* Writer side of a cache file: what the first epoch does with each sample's backbone activations
+ * (Section IV-B).  create makes (or truncates) `path` for N samples of L x S x d elements of `dtype`
+ * with labels_per_sample (1 or S) int32 labels each; store copies one sample - `slabs` is [L][S][d],
+ * device memory when slabs_on_device != 0 (copied on cuda_stream, which the call waits for) or host
+ * memory - and its labels (host) into place, in any order, any number of times; close flushes and
+ * unmaps.  Samples never stored read as zeros.  The writer needs no pac_ctx; a backbone forward hands
+ * it each layer stack as it is produced.  info reads a file's header (any pointer may be NULL).
+ * Errors: PAC_ERR_INVALID_ARG (bad sizes, unopenable path, foreign file), PAC_ERR_SAMPLE_ID_RANGE,
+ * PAC_ERR_NOMEM, PAC_ERR_CUDA (device copy failed, or a device source without a usable device). */
+typedef struct pac_cache_writer pac_cache_writer;
+pac_status pac_cache_writer_create(pac_cache_writer** out, const char* path, int dtype, long long N, int L, int S, int d,
+                                   int labels_per_sample);
+pac_status pac_cache_writer_store(pac_cache_writer* w, long long sample_id, const void* slabs, int slabs_on_device,
+                                  const int* host_labels, void* cuda_stream);
+pac_status pac_cache_writer_close(pac_cache_writer* w);
+pac_status pac_cache_file_info(const char* path, int* dtype, long long* N, int* L, int* S, int* d, int* labels_per_sample);
+
 /* Allocates parameters, gradients, AdamW moments and scratch for batches up to
  * cfg->max_batch and fills the parameters from `seed`:
  * W_down ~ N(0, 1/d), lambda = lambda_init, W_up = 0, W_head ~ N(0, 1/d), b_head = 0

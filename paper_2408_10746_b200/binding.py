@@ -22,7 +22,8 @@ STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_S
                 "PAC_ERR_UNSUPPORTED", "PAC_ERR_NOMEM", "PAC_ERR_CUDA", "PAC_ERR_TIMEOUT"]
 
 # every symbol include/pac.h declares
-EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_cache_register_host", "pac_adapter_init", "pac_train_step", "pac_train_step_dev_loss", "pac_set_grad_scale", "pac_train_step_async",
+EXPORTS = ["pac_create", "pac_destroy", "pac_cache_register", "pac_cache_register_host", "pac_cache_register_file",
+           "pac_cache_writer_create", "pac_cache_writer_store", "pac_cache_writer_close", "pac_cache_file_info", "pac_adapter_init", "pac_train_step", "pac_train_step_dev_loss", "pac_set_grad_scale", "pac_train_step_async",
            "pac_adam_step", "pac_eval_logits", "pac_gather", "pac_train_epoch", "pac_train_epoch_dev",
            "pac_param_count", "pac_get_params", "pac_set_params", "pac_get_grads", "pac_get_opt_state",
            "pac_set_opt_state", "pac_set_option", "pac_device_buffers", "pac_params_changed", "pac_kernel_times", "pac_stream_phase_times", "pac_launch_count", "pac_sync", "pac_selftest_wait_expiry", "pac_last_error",
@@ -94,6 +95,10 @@ def load_library() -> C.CDLL:
         "pac_device_buffers": [P, C.POINTER(P), C.POINTER(P)], "pac_params_changed": [P],
         "pac_selftest_wait_expiry": [P, C.c_ulonglong],
         "pac_train_step_dev_loss": [P, P, I, P], "pac_set_grad_scale": [P, F],
+        "pac_cache_register_file": [P, C.c_char_p],
+        "pac_cache_writer_create": [C.POINTER(P), C.c_char_p, I, LL, I, I, I, I],
+        "pac_cache_writer_store": [P, LL, P, I, P, P], "pac_cache_writer_close": [P],
+        "pac_cache_file_info": [C.c_char_p, C.POINTER(I), C.POINTER(LL), C.POINTER(I), C.POINTER(I), C.POINTER(I), C.POINTER(I)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -185,6 +190,14 @@ class PacContext:
         self._keep += [cache, labels]
         self.shape = (N, L, S, d)
         self.cache_dtype = cache.dtype
+
+    def cache_register_file(self, path: str):
+        """A cache file written by CacheWriter: mapped read-only and reloaded per minibatch."""
+        import torch
+        dt, N, L, S, d, per = cache_file_info(path)
+        self._ck(self._lib.pac_cache_register_file(self._h, path.encode()))
+        self.shape = (N, L, S, d)
+        self.cache_dtype = {PAC_F32: torch.float32, PAC_BF16: torch.bfloat16}[dt]
 
     def adapter_init(self, r: int, n_out: int, max_batch: int, act: int = PAC_ACT_RELU,
                      head: int = PAC_HEAD_MEANPOOL_CLS, lambda_init: float = 0.5, lm_head=None, seed: int = 1):
@@ -333,6 +346,54 @@ class PacContext:
 
 
 STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def cache_file_info(path: str):
+    """(dtype, N, L, S, d, labels_per_sample) from a cache file's header."""
+    lib = load_library()
+    dt, L, S, d, per = C.c_int(), C.c_int(), C.c_int(), C.c_int(), C.c_int()
+    N = C.c_longlong()
+    st = lib.pac_cache_file_info(path.encode(), C.byref(dt), C.byref(N), C.byref(L), C.byref(S), C.byref(d), C.byref(per))
+    if st != 0:
+        raise PacError(st, f"{path} is not a complete cache file")
+    return dt.value, N.value, L.value, S.value, d.value, per.value
+
+
+class CacheWriter:
+    """Writer side of a cache file: store(sample_id, slabs, labels) records one sample's [L][S][d]
+    activations (a CUDA or CPU tensor) and its labels, in any order, as a backbone's first epoch would."""
+
+    def __init__(self, path: str, dtype, N: int, L: int, S: int, d: int, labels_per_sample: int = 1):
+        import torch
+        self._lib = load_library()
+        dt = {torch.float32: PAC_F32, torch.bfloat16: PAC_BF16}[dtype]
+        h = C.c_void_p()
+        st = self._lib.pac_cache_writer_create(C.byref(h), path.encode(), dt, N, L, S, d, labels_per_sample)
+        if st != 0:
+            raise PacError(st, f"pac_cache_writer_create({path}) failed")
+        self._h, self.shape, self.per = h, (L, S, d), labels_per_sample
+
+    def store(self, sample_id: int, slabs, labels, stream: Optional[int] = None):
+        assert tuple(slabs.shape) == self.shape and slabs.is_contiguous()
+        lab = np.ascontiguousarray(np.asarray(labels, dtype=np.int32).reshape(-1))
+        assert lab.size == self.per
+        st = self._lib.pac_cache_writer_store(self._h, sample_id, slabs.data_ptr(), 1 if slabs.is_cuda else 0,
+                                              lab.ctypes.data, C.c_void_p(stream) if stream else None)
+        if st != 0:
+            raise PacError(st, f"pac_cache_writer_store(sample {sample_id}) failed")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            st = self._lib.pac_cache_writer_close(self._h)
+            self._h = None
+            if st != 0:
+                raise PacError(st, "pac_cache_writer_close failed")
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
 
 
 def eval_logits_static(cache, dev_params, r: int, n_out: int, dev_sample_ids, out, act: int = PAC_ACT_RELU,

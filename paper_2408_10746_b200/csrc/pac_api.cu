@@ -6,6 +6,11 @@
 #include <new>
 #include <vector>
 
+#include <fcntl.h>
+#include <sys/mman.h>
+#include <sys/stat.h>
+#include <unistd.h>
+
 #include "pac_common.cuh"
 #include "pac_simt.cuh"
 #include "pac_tensor.cuh"
@@ -73,7 +78,42 @@ struct HostCache {
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ready[2] = {nullptr, nullptr};      // slot filled (copy stream)
     cudaEvent_t freed[2] = {nullptr, nullptr};      // slot's step enqueued and done (compute stream)
+    // a cache file mapped by pac_cache_register_file (owned: unmapped in pac_destroy)
+    void* map_base = nullptr;
+    size_t map_bytes = 0;
 };
+
+// ---------------------------------------------------------------------------
+// Cache files (Section IV-B: the activations are recorded during the first epoch and kept on
+// storage; Section V-B, storage cost analysis: reloaded per micro-batch).  Layout: a 64-byte
+// header, the cache [N][L][S][d] in its dtype, then the labels [N][labels_per_sample] as int32.
+// ---------------------------------------------------------------------------
+struct CacheFileHeader {
+    char magic[8];                 // "PACCACHE"
+    unsigned version;              // 1
+    int dtype;                     // pac_dtype
+    long long N;
+    int L, S, d, labels_per_sample;
+    char pad[24];
+};
+static_assert(sizeof(CacheFileHeader) == 64, "cache file header is 64 bytes");
+const char CACHE_MAGIC[8] = {'P', 'A', 'C', 'C', 'A', 'C', 'H', 'E'};
+
+inline size_t cache_file_data_bytes(const CacheFileHeader& h) {
+    return (size_t)h.N * h.L * h.S * h.d * (h.dtype == PAC_F32 ? 4 : 2);
+}
+// the labels start at the next multiple of 64 bytes behind the data
+inline size_t cache_file_labels_offset(const CacheFileHeader& h) {
+    return sizeof(CacheFileHeader) + ((cache_file_data_bytes(h) + 63) & ~(size_t)63);
+}
+inline size_t cache_file_bytes(const CacheFileHeader& h) {
+    return cache_file_labels_offset(h) + (size_t)h.N * h.labels_per_sample * sizeof(int);
+}
+inline bool cache_file_header_ok(const CacheFileHeader& h) {
+    return std::memcmp(h.magic, CACHE_MAGIC, 8) == 0 && h.version == 1u && (h.dtype == PAC_F32 || h.dtype == PAC_BF16) &&
+           h.N >= 1 && h.N <= 0x7fffffffLL && h.L >= 1 && h.S >= 1 && h.d >= 1 &&
+           (h.labels_per_sample == 1 || h.labels_per_sample == h.S);
+}
 
 }  // namespace
 
@@ -676,6 +716,7 @@ void free_all(pac_ctx* c) {
     }
     if (c->hc.iota) cudaFree(c->hc.iota);
     if (c->hc.copy_stream) cudaStreamDestroy(c->hc.copy_stream);
+    if (c->hc.map_base) munmap(c->hc.map_base, c->hc.map_bytes);
     if (c->zc_ids) cudaFreeHost(c->zc_ids);
     if (c->zc_tags) cudaFreeHost(c->zc_tags);
     if (c->zc_dev_ids) cudaFree(c->zc_dev_ids);
@@ -774,6 +815,33 @@ pac_status pac_cache_register_host(pac_ctx* c, const void* host_cache, int dtype
     c->hc.sample_bytes = (long long)L * S * d * (dtype == PAC_F32 ? 4 : 2);
     c->cache = nullptr;                  // bound to a staging slot before every use
     c->labels = nullptr;
+    return PAC_OK;
+}
+
+pac_status pac_cache_register_file(pac_ctx* c, const char* path) {
+    NEED_CTX(c);
+    if (!path) return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register_file: path is NULL");
+    if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_cache_register_file: adapters already initialised");
+    if (c->hc.map_base) return fail(c, PAC_ERR_BAD_STATE, "pac_cache_register_file: a cache file is already registered");
+    const int fd = open(path, O_RDONLY);
+    if (fd < 0) return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register_file: cannot open %s", path);
+    CacheFileHeader h;
+    struct stat sb;
+    if (read(fd, &h, sizeof h) != (ssize_t)sizeof h || !cache_file_header_ok(h) || fstat(fd, &sb) != 0 ||
+        (size_t)sb.st_size < cache_file_bytes(h)) {
+        close(fd);
+        return fail(c, PAC_ERR_INVALID_ARG, "pac_cache_register_file: %s is not a complete cache file", path);
+    }
+    const size_t bytes = cache_file_bytes(h);
+    void* base = mmap(nullptr, bytes, PROT_READ, MAP_SHARED, fd, 0);
+    close(fd);
+    if (base == MAP_FAILED) return fail(c, PAC_ERR_NOMEM, "pac_cache_register_file: mmap of %zu bytes failed", bytes);
+    const unsigned char* data = (const unsigned char*)base + sizeof(CacheFileHeader);
+    const int* labels = (const int*)((const unsigned char*)base + cache_file_labels_offset(h));
+    pac_status st = pac_cache_register_host(c, data, h.dtype, h.N, h.L, h.S, h.d, labels, h.labels_per_sample);
+    if (st != PAC_OK) { munmap(base, bytes); return st; }
+    c->hc.map_base = base;
+    c->hc.map_bytes = bytes;
     return PAC_OK;
 }
 
@@ -1570,4 +1638,103 @@ extern "C" pac_status pac_dequantize_absmax(int device, void* cuda_stream, const
         dequantize_absmax_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(dev_q, dev_c, n, block, dev_out);
     }
     return cudaGetLastError() == cudaSuccess ? PAC_OK : PAC_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
+// Writer side of a cache file: what the first epoch does (Section IV-B) - every sample's per-layer
+// backbone activations are recorded once, as they come out of the caller's backbone forward.
+// ---------------------------------------------------------------------------
+struct pac_cache_writer {
+    int fd = -1;
+    void* base = nullptr;
+    size_t bytes = 0;
+    CacheFileHeader h{};
+    unsigned char* bounce = nullptr;       // page-locked, one sample
+    size_t sample_bytes = 0;
+    long long written = 0;
+};
+
+extern "C" pac_status pac_cache_writer_create(pac_cache_writer** out, const char* path, int dtype, long long N, int L, int S, int d,
+                                              int labels_per_sample) {
+    if (!out || !path) return PAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    CacheFileHeader h{};
+    std::memcpy(h.magic, CACHE_MAGIC, 8);
+    h.version = 1u; h.dtype = dtype; h.N = N; h.L = L; h.S = S; h.d = d; h.labels_per_sample = labels_per_sample;
+    if (!cache_file_header_ok(h)) return PAC_ERR_INVALID_ARG;
+    pac_cache_writer* w = new (std::nothrow) pac_cache_writer();
+    if (!w) return PAC_ERR_NOMEM;
+    w->h = h;
+    w->bytes = cache_file_bytes(h);
+    w->sample_bytes = cache_file_data_bytes(h) / (size_t)N;
+    w->fd = open(path, O_RDWR | O_CREAT | O_TRUNC, 0644);
+    if (w->fd < 0 || ftruncate(w->fd, (off_t)w->bytes) != 0) {
+        if (w->fd >= 0) close(w->fd);
+        delete w;
+        return PAC_ERR_INVALID_ARG;
+    }
+    w->base = mmap(nullptr, w->bytes, PROT_READ | PROT_WRITE, MAP_SHARED, w->fd, 0);
+    if (w->base == MAP_FAILED) { close(w->fd); delete w; return PAC_ERR_NOMEM; }
+    std::memcpy(w->base, &h, sizeof h);
+    if (cudaMallocHost((void**)&w->bounce, w->sample_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        w->bounce = nullptr;               // without a device (or page-locked memory) only host sources can be stored
+    }
+    *out = w;
+    return PAC_OK;
+}
+
+extern "C" pac_status pac_cache_writer_store(pac_cache_writer* w, long long sample_id, const void* slabs, int slabs_on_device,
+                                             const int* host_labels, void* cuda_stream) {
+    if (!w || !slabs || !host_labels) return PAC_ERR_INVALID_ARG;
+    if (sample_id < 0 || sample_id >= w->h.N) return PAC_ERR_SAMPLE_ID_RANGE;
+    unsigned char* data = (unsigned char*)w->base + sizeof(CacheFileHeader);
+    unsigned char* dst = data + (size_t)sample_id * w->sample_bytes;
+    if (slabs_on_device) {
+        if (!w->bounce) return PAC_ERR_CUDA;
+        cudaStream_t st = (cudaStream_t)cuda_stream;
+        // device -> page-locked bounce buffer -> file mapping (the mapping itself is pageable)
+        if (cudaMemcpyAsync(w->bounce, slabs, w->sample_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess) {
+            cudaGetLastError();
+            return PAC_ERR_CUDA;
+        }
+        std::memcpy(dst, w->bounce, w->sample_bytes);
+    } else {
+        std::memcpy(dst, slabs, w->sample_bytes);
+    }
+    int* lab = (int*)((unsigned char*)w->base + cache_file_labels_offset(w->h)) + (size_t)sample_id * w->h.labels_per_sample;
+    std::memcpy(lab, host_labels, sizeof(int) * (size_t)w->h.labels_per_sample);
+    w->written++;
+    return PAC_OK;
+}
+
+extern "C" pac_status pac_cache_writer_close(pac_cache_writer* w) {
+    if (!w) return PAC_ERR_INVALID_ARG;
+    pac_status st = PAC_OK;
+    if (w->base && msync(w->base, w->bytes, MS_SYNC) != 0) st = PAC_ERR_CUDA;
+    if (w->base) munmap(w->base, w->bytes);
+    if (w->fd >= 0) close(w->fd);
+    if (w->bounce) cudaFreeHost(w->bounce);
+    delete w;
+    return st;
+}
+
+extern "C" pac_status pac_cache_file_info(const char* path, int* dtype, long long* N, int* L, int* S, int* d, int* labels_per_sample) {
+    if (!path) return PAC_ERR_INVALID_ARG;
+    const int fd = open(path, O_RDONLY);
+    if (fd < 0) return PAC_ERR_INVALID_ARG;
+    CacheFileHeader h;
+    struct stat sb;
+    const bool ok = read(fd, &h, sizeof h) == (ssize_t)sizeof h && cache_file_header_ok(h) && fstat(fd, &sb) == 0 &&
+                    (size_t)sb.st_size >= cache_file_bytes(h);
+    close(fd);
+    if (!ok) return PAC_ERR_INVALID_ARG;
+    if (dtype) *dtype = h.dtype;
+    if (N) *N = h.N;
+    if (L) *L = h.L;
+    if (S) *S = h.S;
+    if (d) *d = h.d;
+    if (labels_per_sample) *labels_per_sample = h.labels_per_sample;
+    return PAC_OK;
 }

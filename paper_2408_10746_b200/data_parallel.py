@@ -34,7 +34,9 @@ import torch.distributed as dist
 
 class PacLocalTrainer:
     """Adapter around a PacContext: exposes its device buffers for in-place collectives.  `stream` is
-    the torch stream whose handle the context was created on (None: torch's current stream)."""
+    the torch stream whose handle the context was created on; collectives are issued under it, so that
+    they are ordered behind the step's kernels and ahead of the optimizer's.  With None the context must
+    have been created on the stream that is torch's current one whenever the orchestrator runs."""
 
     def __init__(self, ctx, stream: Optional["torch.cuda.Stream"] = None):
         self.ctx, self.stream = ctx, stream

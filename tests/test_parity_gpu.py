@@ -655,6 +655,7 @@ def test_device_buffer_views_and_single_rank_data_parallel(tiny):
     try:
         dp = DataParallel(PacLocalTrainer(ctx))
         assert dp.train_step(ids) is None
+        ctx.sync()                                     # the step was only enqueued (on the context's own stream)
         assert np.array_equal(grads.cpu().numpy(), ctx.get_grads())
         dp.adam_step(hp)
         loss = float(dp.epoch_losses()[0])
