@@ -570,7 +570,6 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     const FusedFwdPlan& pl = c->fplan;
     FusedFwdParams fp{};
     fp.mid = mid_params(c, pl.mp, d_ids, B, train, d_logits_out);
-    fp.mid.u = nullptr;
     fp.mid.layers_per_cta = pl.layers_per_cta;
     if (c->step_host_ids) {
         fp.mid.host_ids = 1; fp.mid.ids_copy = c->sc.ids;
@@ -580,8 +579,7 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
         fp.mid.pref_seq = seq;
     }
     fp.mid.early_ids = c->step_early_ids ? 1 : 0;
-    fp.mid.u_swz = pl.u_swz;
-    fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset;
+    fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset; fp.wide_n = pl.wide_n;
     fp.stamp = next_stamp(c, 0);
     cudaError_t e = fused_fwd_launch(pl, c->tplan.map_cache_fwd, c->tplan.map_w, fp, c->cfg.act, c->stream);
     c->launches++;
