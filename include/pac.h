@@ -71,15 +71,17 @@ typedef struct { float lr, beta1, beta2, eps, weight_decay; } pac_adamw;
 
 /* Options for pac_set_option. */
 typedef enum {
-    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic: tensor-core path when the shape allows; its forward half
-                                     (down-projections + classifier-head phase) runs as ONE launch per
-                                     step when the shape allows it (bf16 cache, classifier head, S <= 128,
-                                     r <= 64) and the batch's clusters all fit on the device at once,
-                                     otherwise as two launches,
+    PAC_OPT_KERNEL_PATH = 0,  /* 0 = automatic: tensor-core path when the shape allows.  Its forward half
+                                     (down-projections + classifier-head phase) runs as ONE launch per step for
+                                     short sequences (bf16 cache, classifier head, S <= 128, r <= 64) when the
+                                     batch's clusters all fit on the device at once; with enough 128-token
+                                     tiles to fill the device (2 * B * ceil(S/128) >= SMs, r a multiple of 32 up
+                                     to 128) the merge / activation chain runs in the epilogue of the
+                                     down-projection kernel instead; otherwise two plain launches,
                                  1 = force the plain fp32-FMA kernels,
-                                 2 = tensor-core path, forward half always as two launches,
-                                 3 = tensor-core path, forward half as one launch whenever the shape
-                                     allows it, whatever the batch size;
+                                 2 = tensor-core path, forward half always as two plain launches,
+                                 3 = tensor-core path, one-launch forward whenever the shape allows it,
+                                 4 = tensor-core path, chain-in-epilogue forward whenever the shape allows it;
                                  set before adapter_init */
     PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events
                                  (pac_kernel_times), 2 = device-side timestamps of the two passes' stream
@@ -280,9 +282,10 @@ pac_status pac_sync(pac_ctx* ctx);
  * timeout.  The paper describes no failure handling for this path; this is the library's own contract. */
 pac_status pac_selftest_wait_expiry(pac_ctx* ctx, unsigned long long limit_ns);
 const char* pac_last_error(const pac_ctx* ctx);
-/* Which kernels the next train step will use (valid after adapter_init): "simt", "tensor", or
+/* Which kernels the next train step will use (valid after adapter_init): "simt", "tensor",
  * "tensor+fused_forward" when a batch of max_batch samples runs the down-projections
- * (Section IV-A) and the whole classifier-head phase as one launch per step. */
+ * (Section IV-A) and the whole classifier-head phase as one launch per step, or
+ * "tensor+chain_forward" when the merge / activation chain runs in the down-projection kernel's epilogue. */
 const char* pac_kernel_path(const pac_ctx* ctx);
 
 /* Block-wise absmax INT8 quantisation, Section IV-D, Eq. 1 (the paper applies it to the frozen

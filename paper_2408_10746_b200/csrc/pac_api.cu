@@ -16,6 +16,7 @@
 #include "pac_tensor.cuh"
 #include "pac_mid.cuh"
 #include "pac_fused_fwd.cuh"
+#include "pac_chain_fwd.cuh"
 #include "pac_gemm.cuh"
 #include "pac_quant.cuh"
 
@@ -55,6 +56,8 @@ struct Scratch {
     bf16* wdT = nullptr;           // [L][2][d][r] bf16 hi/lo shadow of W_down
     float* lm_part = nullptr;      // [slices][...] partial sums of the LM path's two skinny products (dW_up, da_L)
     float* dw_part = nullptr;      // split partials of dW_down
+    unsigned* gates = nullptr;     // [M][r] ReLU gates of all layers, one word per element (chain-in-epilogue forward)
+    float* pool_part = nullptr;    // [B][s_chunks * 4][r] token sums of a_L per 32-token group (chain-in-epilogue forward)
 };
 
 // A cache that lives in host memory (Section V-B, storage cost analysis: the cache is kept on
@@ -161,7 +164,10 @@ struct pac_ctx {
     TensorPlan tplan{};
     MidPlan mplan{};               // fused classifier-head kernel (when the shape allows)
     FusedFwdPlan fplan{};          // down-projections + classifier-head kernel in one launch (short sequences)
-    int forward_mode = 0;          // 0: one-launch forward when a batch's clusters fit the device at once, 2: never, 3: whenever the shape allows
+    MidPlan pplan{};               // head / reverse-chain kernel behind the chain-in-epilogue forward
+    bool chain_ok = false;         // the chain-in-epilogue forward can take this shape
+    int forward_mode = 0;          // 0: automatic, 2: down-projections and head phase as two plain launches, 3: one-launch
+                                   // forward whenever the shape allows, 4: chain-in-epilogue forward whenever the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
     bool lm_tensor = false;
     int sms = 0;                   // multiprocessors of the device
@@ -506,9 +512,20 @@ bool use_fused_cls(const pac_ctx* c) { return c->cfg.head == PAC_HEAD_MEANPOOL_C
 // and chain phases do not overlap across waves); larger batches keep the two separate kernels.
 bool use_fused_fwd(const pac_ctx* c, int B) {
     if (!use_fused_cls(c) || !use_tensor(c) || !c->fplan.ok) return false;
+    if (c->forward_mode == 4 && c->chain_ok) return false;
     return c->forward_mode == 3 || B <= c->fplan.max_clusters;
 }
-int cls_cluster_size(const pac_ctx* c, int B) { return use_fused_fwd(c, B) ? c->fplan.mp.G : c->mplan.G; }
+// Chain-in-epilogue forward: one CTA per 128-token tile walks all layers, so it needs enough tiles to fill
+// the device (long sequences or large batches); the one-launch cluster forward keeps the short shapes.
+bool use_chain_fwd(const pac_ctx* c, int B) {
+    if (!use_fused_cls(c) || !use_tensor(c) || !c->chain_ok || c->forward_mode == 2 || c->forward_mode == 3) return false;
+    if (c->forward_mode == 4) return true;
+    if (use_fused_fwd(c, B)) return false;
+    return 2 * B * c->tplan.fp.s_chunks >= c->sms;
+}
+int cls_cluster_size(const pac_ctx* c, int B) {
+    return use_chain_fwd(c, B) ? c->pplan.G : use_fused_fwd(c, B) ? c->fplan.mp.G : c->mplan.G;
+}
 
 pac_status down_projection(pac_ctx* c, const int* d_ids, int B) {
     pac_status st;
@@ -546,12 +563,12 @@ MidParams mid_params(pac_ctx* c, const MidPlan& mp, const int* d_ids, int B, boo
     p.ids = d_ids; p.N = dm.N; p.labels = c->labels;
     p.L = dm.L; p.S = dm.S; p.d = dm.d; p.r = dm.r; p.C = dm.C; p.B = B;
     p.G = mp.G; p.Sg = mp.Sg; p.dg = mp.dg; p.train = train ? 1 : 0;
-    p.scratch = mp.scratch; p.wup_smem = mp.wup_smem;
+    p.scratch = mp.scratch;
     p.u = sc.u; p.lstride = (long long)c->max_rows * dm.r;
     p.lam = c->params + c->lay.lam; p.W_up = c->params + c->lay.w_up;
     p.W_head = c->params + c->lay.w_head; p.b_head = c->params + c->lay.b_head; p.hbar = sc.hbar;
     p.du = use_tensor(c) ? (void*)sc.du16 : (void*)sc.du;
-    p.pooled_a = sc.pooled_a; p.pooled_y = sc.pooled_y; p.gvec = sc.gvec; p.dlogits = sc.dlogits;
+    p.pooled_a = sc.pooled_a; p.dlogits = sc.dlogits;
     p.loss_b = sc.loss_b; p.lam_part = sc.lam_part; p.logits_out = train ? sc.logits : d_logits_out;
     p.status = c->status;
     return p;
@@ -587,9 +604,36 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     return PAC_OK;
 }
 
+// Down-projections with the chain in their epilogue, then head / loss / reverse chain from the parked state.
+pac_status chain_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    const Dims& dm = c->dm;
+    ChainFwdParams cp{};
+    cp.ids = d_ids; cp.N = dm.N; cp.L = dm.L; cp.S = dm.S; cp.d = dm.d; cp.r = dm.r; cp.B = B;
+    cp.s_chunks = c->tplan.fp.s_chunks; cp.k_chunks = c->tplan.fp.k_chunks; cp.stages = c->tplan.fp.stages;
+    cp.train = train ? 1 : 0;
+    cp.lam = c->params + c->lay.lam;
+    cp.parked = c->sc.du16; cp.layer_stride = (long long)c->max_rows * dm.r;
+    cp.gates = c->sc.gates; cp.pool_part = c->sc.pool_part;
+    cp.status = c->status; cp.stamp = next_stamp(c, 0);
+    time_mark(c, 0, false);
+    cudaError_t e = chain_fwd_launch(c->tplan.map_cache_fwd, c->tplan.map_w, cp, c->tplan.smem_fwd, c->cfg.act, c->stream);
+    c->launches++;
+    time_mark(c, 0, true);
+    if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "chain-in-epilogue forward launch failed: %s", cudaGetErrorString(e));
+    MidParams p = mid_params(c, c->pplan, d_ids, B, train, d_logits_out);
+    p.gates = c->sc.gates; p.pool_part = c->sc.pool_part; p.n_pool_parts = cp.s_chunks * CF_POOL_PARTS;
+    time_mark(c, 1, false);
+    e = mid_launch_parked(c->pplan, p, c->cfg.act, c->stream);
+    c->launches++;
+    time_mark(c, 1, true);
+    if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "head kernel launch failed: %s", cudaGetErrorString(e));
+    return PAC_OK;
+}
+
 // Forward half of a classifier-head step (everything up to du and the per-sample head vectors).
 pac_status cls_forward_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
     pac_status st;
+    if (use_chain_fwd(c, B)) return chain_fwd_enqueue(c, d_ids, B, train, d_logits_out);
     if (use_fused_fwd(c, B)) {
         time_mark(c, 0, false);
         st = fused_fwd_enqueue(c, d_ids, B, train, d_logits_out);
@@ -608,7 +652,7 @@ void bias_corrections(const pac_adamw* hp, long long step, float* bc1, float* bc
     *bc2 = (float)(1.0 - std::pow((double)hp->beta2, (double)step));
 }
 
-pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* hp) {
+pac_status finalize_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, const pac_adamw* hp) {
     const Dims& dm = c->dm;
     Scratch& sc = c->sc;
     FinalizeParams f{};
@@ -617,7 +661,8 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
     f.splits = use_tensor(c) ? tensor_splits(c->tplan, B) : 1;
     f.dw_elems = (long long)dm.L * dm.d * dm.r;
     f.lam_part = sc.lam_part; f.lam_blocks = B * cls_cluster_size(c, B);
-    f.pooled_a = sc.pooled_a; f.gvec = sc.gvec; f.pooled_y = sc.pooled_y; f.dlogits = sc.dlogits; f.loss_b = sc.loss_b;
+    f.pooled_a = sc.pooled_a; f.dlogits = sc.dlogits; f.loss_b = sc.loss_b;
+    f.hbar = sc.hbar; f.ids = d_ids; f.N = dm.N; f.params_in = c->params;
     f.grads = c->grads; f.loss_out = d_loss;
     f.adam = hp ? 1 : 0;
     if (hp) {
@@ -639,11 +684,13 @@ pac_status finalize_enqueue(pac_ctx* c, int B, float* d_loss, const pac_adamw* h
         f.next_dev_tag = c->zc_dev_tag + (next_seq & 1u);
     }
     f.status = c->status;
-    const unsigned rest_blocks = cdiv(c->lay.total - c->lay.lam, 256);
+    const unsigned rest_blocks = cdiv(dm.d, FIN_KB);
     f.rest_blocks = (int)rest_blocks;
+    const size_t fin_smem = sizeof(float) * ((size_t)2 * B * FIN_KB + (size_t)dm.r * FIN_KB + (size_t)FIN_KB * dm.C);
+    if (fin_smem > 48 * 1024) return fail(c, PAC_ERR_UNSUPPORTED, "finalisation: batch or adapter width beyond its shared memory");
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    pdl_launch_config(&cfg, attr, dim3(f.wd_blocks + rest_blocks + 1), dim3(256), 0, c->stream);   // + one block for lambda and the loss
+    pdl_launch_config(&cfg, attr, dim3(f.wd_blocks + rest_blocks + 1), dim3(256), fin_smem, c->stream);   // + one block for lambda and the loss
     cudaError_t le = cudaLaunchKernelEx(&cfg, finalize_cls_kernel, f);
     c->launches++;
     if (le != cudaSuccess) return fail(c, PAC_ERR_CUDA, "finalize kernel launch failed: %s", cudaGetErrorString(le));
@@ -658,7 +705,7 @@ pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, con
         if (c->step_host_ids) d_ids = c->sc.ids;          // the forward kernel left a device copy for the later kernels
         if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
         time_mark(c, 3, false);
-        st = finalize_enqueue(c, B, d_loss, hp);
+        st = finalize_enqueue(c, d_ids, B, d_loss, hp);
         time_mark(c, 3, true);
         return st;
     }
@@ -700,7 +747,7 @@ void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
-                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.lm_part, s.dw_part, c->params, c->grads,
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, c->params, c->grads,
                     c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -887,7 +934,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     const long long Mr = (long long)c->max_rows * dm.r;
     c->chain_blocks_max = (int)cdiv(Mr, 256);
     c->mplan = cls ? mid_plan(dm) : MidPlan{};
-    if (c->mplan.ok && cfg->max_batch * c->mplan.G > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * c->mplan.G;
+    if (c->mplan.ok && cfg->max_batch * 8 > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * 8;     // clusters of up to 8
     FusedFwdPlan fwd_plan{};
     if (c->mplan.ok && c->dtype == PAC_BF16 && tensor_shape_supported(dm) && !c->force_simt && c->forward_mode != 2) {
         int max_smem = 0;
@@ -976,6 +1023,15 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             }
             if (ts == PAC_OK) {
                 A(dmalloc(c, &s.dw_part, part_floats));
+                c->chain_ok = false;
+                if (st == PAC_OK && cls && c->mplan.ok && chain_fwd_supported(dm) && c->tplan.fp.wide_n) {
+                    c->pplan = mid_plan_parked(dm);
+                    if (c->pplan.ok) {
+                        A(dmalloc(c, &s.gates, Mr));
+                        A(dmalloc(c, &s.pool_part, (long long)cfg->max_batch * c->tplan.fp.s_chunks * CF_POOL_PARTS * dm.r));
+                        c->chain_ok = (st == PAC_OK);
+                    }
+                }
                 c->tensor_ok = (st == PAC_OK);
                 if (c->tensor_ok && fwd_plan.ok) {
                     fwd_plan.max_clusters = fused_fwd_max_clusters(fwd_plan, cfg->act);
@@ -1337,7 +1393,7 @@ pac_status pac_params_changed(pac_ctx* c) {
 pac_status pac_set_option(pac_ctx* c, int option, int value) {
     NEED_CTX(c);
     if (option == PAC_OPT_KERNEL_PATH) {
-        if (value < 0 || value > 3) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0, 1, 2 or 3");
+        if (value < 0 || value > 4) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0, 1, 2, 3 or 4");
         if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_set_option: set the kernel path before pac_adapter_init");
         c->force_simt = value == 1;
         c->forward_mode = value >= 2 ? value : 0;
@@ -1444,6 +1500,7 @@ const char* pac_last_error(const pac_ctx* c) { return c ? c->err.c_str() : "null
 
 const char* pac_kernel_path(const pac_ctx* c) {
     if (!c || !c->inited || !use_tensor(c)) return "simt";
+    if (use_chain_fwd(c, c->cfg.max_batch)) return "tensor+chain_forward";
     return use_fused_fwd(c, c->cfg.max_batch) ? "tensor+fused_forward" : "tensor";
 }
 

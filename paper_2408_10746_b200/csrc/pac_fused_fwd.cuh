@@ -234,12 +234,11 @@ inline FusedFwdPlan fused_fwd_plan(const Dims& dm, int max_smem) {
         if (th < 256) th = 256;                                  // producer, MMA, prefetch and drain warps
         int scratch;
         size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
-        const size_t wup = (size_t)dm.r * dg;
         const size_t state = (size_t)dm.L * th * sizeof(float4);   // chain state of mid_body: [L][threads] float4
         const size_t budget = (size_t)max_smem - 2048;
-        // stage ring / chain state share one region, head vectors (with the W_up slice when it fits) behind it
-        for (int with_wup = 1; with_wup >= 0; --with_wup) {
-            const size_t mid_bytes = (floats + (with_wup ? wup : 0)) * sizeof(float);
+        // stage ring / chain state share one region, head vectors behind it
+        {
+            const size_t mid_bytes = floats * sizeof(float);
             if (mid_bytes + state > budget) continue;
             int st = (int)((budget - mid_bytes) / stage);
             if (st > 16) st = 16;
@@ -247,7 +246,7 @@ inline FusedFwdPlan fused_fwd_plan(const Dims& dm, int max_smem) {
             size_t region = (size_t)st * stage;
             if (region < state) region = (state + 1023) & ~(size_t)1023;
             fp.mp.ok = true; fp.mp.G = G; fp.mp.Sg = Sg; fp.mp.dg = dg; fp.mp.threads = th; fp.mp.scratch = scratch;
-            fp.mp.gpt = 1; fp.mp.smem_state = 1; fp.mp.wup_smem = with_wup;
+            fp.mp.gpt = 1; fp.mp.smem_state = 1;
             fp.layers_per_cta = lpc; fp.stages = st; fp.k_chunks = (dm.d + KC - 1) / KC;
             fp.wide_n = lpc <= 4 ? 1 : 0;
             fp.mid_offset = region;

@@ -29,7 +29,6 @@ struct MidParams {
     int dg;                     // head columns per CTA = ceil(d / G)
     int train;
     int scratch;                // floats of block-local reduction scratch
-    int wup_smem;               // 1: this CTA's [r][dg] slice of W_up is staged in shared memory
     int layers_per_cta;         // one-kernel forward: layers whose down-projections each CTA of the cluster computes
     int host_ids;               // 1: ids points at host memory the device can read (written before the launch, so
                                 // it may be read ahead of the predecessor's completion); read once per CTA
@@ -38,13 +37,14 @@ struct MidParams {
     // memory (valid when *pref_tag == pref_seq); otherwise the ids are fetched across the host link
     const int* pref_ids; const unsigned* pref_tag; unsigned pref_seq;
     int* ids_copy;              // one-kernel forward: device copy of the batch's (clamped) ids for the later kernels, or null
-    int u_swz;                  // STATE_TILES: a token row's 4-column groups are stored at (group ^ (token & u_swz))
+    // STATE_PARKED: what the down-projection kernel's epilogue left behind
+    const unsigned* gates;      // [max_rows][r] bit l = gate of layer l
+    const float* pool_part;     // [B][n_pool_parts][r] token sums of a_L per token group
+    int n_pool_parts;
     const float* u; long long lstride;
     const float* lam; const float* W_up; const float* W_head; const float* b_head; const float* hbar;
     void* du;                   // [L][max_rows][r] bf16 or fp32
-    float* pooled_a;            // [B][r]
-    float* pooled_y;            // [B][d]
-    float* gvec;                // [B][d]
+    float* pooled_a;            // [B][r]   mean_s a_L, for the gradient finalisation
     float* dlogits;             // [B][C]
     float* loss_b;              // [B]
     float* lam_part;            // [L][B*G]
@@ -71,13 +71,14 @@ enum {
     STATE_SMEM = 0,      // this CTA's shared memory, prefetched from the global u buffer with cp.async
     STATE_DU = 1,        // u read from global memory; u_l - a_{l-1} parked, in du's type, in the du slot
                          // that the reverse pass overwrites with du_l once it has consumed it
-    STATE_TILES = 2      // this CTA's shared memory, filled by the cluster's own GEMMs before the call:
-                         // [L][Sg tokens][r] fp32, a token row's 4-column groups permuted by u_swz
+    STATE_PARKED = 2     // the forward chain already ran in the down-projection kernel's epilogue: u_l - a_{l-1} is
+                         // parked in the du slots, the gates of all layers are one word per element in global
+                         // memory, and the token sums of a_L come as per-group partial sums
 };
 
 // The small per-CTA vectors of the head computation, carved from one shared-memory region.
 struct MidShared {
-    float *aL, *colsum, *prodq, *prod, *pooled, *daL, *py, *lg, *lam_s, *wh_s, *lred, *wup_s;
+    float *aL, *colsum, *prodq, *prod, *plq, *daL, *py, *lg, *lam_s, *cprod, *wh_s, *lred;
 };
 __device__ __forceinline__ MidShared mid_carve(float* sm, const MidParams& p) {
     MidShared h;
@@ -86,29 +87,32 @@ __device__ __forceinline__ MidShared mid_carve(float* sm, const MidParams& p) {
     h.colsum = h.aL + (size_t)p.Sg * p.r;             // [r]       exchanged through DSMEM
     h.prodq = h.colsum + p.r;                         // [r+1][C]  this CTA's partial head products, exchanged
     h.prod = h.prodq + rc;                            // [r+1][C]  their sum over the cluster
-    h.pooled = h.prod + rc;                           // [r]
-    h.daL = h.pooled + p.r;                           // [r]
+    h.plq = h.prod + rc;                              // [MID_MAX_C] this CTA's tokens' share of S * (mean_s a_L)(W_up W_head), exchanged
+    h.daL = h.plq + MID_MAX_C;                        // [r]
     h.py = h.daL + p.r;                               // [dg]  slice of mean_s h_L
     h.lg = h.py + p.dg;                               // [MID_MAX_C] logits, then dlogits
     h.lam_s = h.lg + MID_MAX_C;                       // [MID_MAX_L]
-    h.wh_s = h.lam_s + MID_MAX_L;                     // [dg][C] slice of W_head
+    h.cprod = h.lam_s + MID_MAX_L;                    // [MID_MAX_L] prod_{l' > l} (1 - lambda_l')
+    h.wh_s = h.cprod + MID_MAX_L;                     // [dg][C] slice of W_head
     h.lred = h.wh_s + (size_t)p.dg * p.C;             // [nwarps][MID_MAX_L]; also [parts][r] scratch
-    h.wup_s = h.lred + (size_t)p.scratch;             // [r][dg] slice of W_up (when p.wup_smem)
     return h;
 }
 
-// cp.async requests for the head operands of CTA rank q (hbar slice of sample `id`, W_head and W_up
-// slices) and plain loads of lambda, issued by threads t0 .. t0 + nthr - 1 of the block.
+// cp.async requests for the head operands of CTA rank q (hbar slice of sample `id`, W_head slice)
+// and plain loads of lambda, issued by threads t0 .. t0 + nthr - 1 of the block.
 __device__ __forceinline__ void mid_prefetch_head(const MidParams& p, const MidShared& h, int q, long long id, int t, int nthr) {
     const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));
     for (int kk = t; kk < kn; kk += nthr) cp_async_4(h.py + kk, p.hbar + id * p.d + k0 + kk);
     for (int e = t; e < kn * p.C; e += nthr) cp_async_4(h.wh_s + e, p.W_head + (long long)k0 * p.C + e);
-    if (p.wup_smem) {
-        const int w = t >> 5, ln = t & 31, nw = nthr >> 5;
-        for (int j = w; j < p.r; j += nw)
-            for (int kk = ln; kk < kn; kk += 32) cp_async_4(h.wup_s + (size_t)j * p.dg + kk, p.W_up + (long long)j * p.d + k0 + kk);
-    }
     for (int l = t; l < MID_MAX_L; l += nthr) h.lam_s[l] = l < p.L ? p.lam[l] : 0.f;
+    if (t == nthr - 1) {
+        // prod_{l' > l} (1 - lambda_l'), multiplied in the order the reverse recursion meets the layers
+        float c = 1.f;
+        for (int l = p.L - 1; l >= 0; --l) {
+            h.cprod[l] = c;
+            c *= 1.f - p.lam[l];
+        }
+    }
 }
 
 // The head is linear in mean_s a_L, so both directions through it reduce to one small matrix:
@@ -123,8 +127,7 @@ __device__ __forceinline__ void mid_head_products(const MidParams& p, const MidS
         for (int c0 = 0; c0 < p.C; c0 += 4) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
             for (int kk = lane; kk < kn; kk += 32) {
-                const float a = j == p.r ? h.py[kk]
-                              : p.wup_smem ? h.wup_s[(size_t)j * p.dg + kk] : p.W_up[(long long)j * p.d + k0 + kk];
+                const float a = j == p.r ? h.py[kk] : p.W_up[(long long)j * p.d + k0 + kk];     // each W_up element is read once
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     if (c0 + c < p.C) acc[c] = fmaf(a, h.wh_s[kk * p.C + c0 + c], acc[c]);
@@ -150,7 +153,7 @@ __device__ __forceinline__ void mid_sum_products(const MidParams& p, const MidSh
 
 // Everything after the down-projections for one sample, executed by one CTA (rank q) of the
 // sample's cluster.  GPT: 4-column groups per thread.  u_s: STATE_SMEM: [L][GPT][nt] float4 state;
-// STATE_TILES: [L][Sg][r] fp32 u tiles.  products_ready: the caller has already prefetched the head
+// products_ready: the caller has already prefetched the head
 // operands, run mid_head_products and passed a cluster barrier.
 template <int ACT, typename DU, int GPT, int STATE>
 __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& cluster, float4* u_s, const MidShared& h,
@@ -161,8 +164,8 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     const int t = threadIdx.x, nt = blockDim.x;
     const int r = p.r, L = p.L, C = p.C;
     const int warp = t >> 5, lane = t & 31, nwarps = nt >> 5;
-    float *aL = h.aL, *colsum = h.colsum, *prod = h.prod, *pooled = h.pooled, *daL = h.daL, *py = h.py,
-          *lg = h.lg, *lam_s = h.lam_s, *wh_s = h.wh_s, *lred = h.lred, *wup_s = h.wup_s;
+    float *aL = h.aL, *colsum = h.colsum, *prod = h.prod, *plq = h.plq,
+          *lg = h.lg, *lam_s = h.lam_s, *lred = h.lred, *cprod = h.cprod, *daL = h.daL;
 
     const int groups_per_tok = r >> 2;
     int s_local[GPT], j4[GPT];
@@ -179,20 +182,13 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     }
     DU* du = reinterpret_cast<DU*>(p.du);
     // layer l of group g: read u, park / fetch the reverse-pass state
-    auto tile_slot = [&](int l, int g) -> float4* {          // STATE_TILES
-        float* row = reinterpret_cast<float*>(u_s) + ((size_t)l * p.Sg + s_local[g]) * r;
-        return reinterpret_cast<float4*>(row + (((j4[g] >> 2) ^ (s_local[g] & p.u_swz)) << 2));
-    };
     auto load_u = [&](int l, int g) -> float4 {
         if constexpr (STATE == STATE_SMEM) return u_s[((size_t)l * GPT + g) * nt + t];
-        else if constexpr (STATE == STATE_TILES) return *tile_slot(l, g);
         else return *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base[g]);
     };
     auto store_w = [&](int l, int g, const float* wv) {
         if constexpr (STATE == STATE_SMEM) {
             u_s[((size_t)l * GPT + g) * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
-        } else if constexpr (STATE == STATE_TILES) {
-            *tile_slot(l, g) = make_float4(wv[0], wv[1], wv[2], wv[3]);
         } else if constexpr (sizeof(DU) == 2) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]), hi = __floats2bfloat162_rn(wv[2], wv[3]);
             uint2 pk;
@@ -206,8 +202,6 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     auto load_w = [&](int l, int g) -> float4 {
         if constexpr (STATE == STATE_SMEM) {
             return u_s[((size_t)l * GPT + g) * nt + t];
-        } else if constexpr (STATE == STATE_TILES) {
-            return *tile_slot(l, g);
         } else if constexpr (sizeof(DU) == 2) {
             const uint2 pk = *reinterpret_cast<const uint2*>(du + (long long)l * p.lstride + base[g]);
             const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
@@ -218,7 +212,6 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         }
     };
     const long long id = known_id >= 0 ? known_id : safe_id(p.ids, b, p.N, (t == 0 && q == 0) ? p.status : nullptr);
-    const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));                  // this CTA's slice of the hidden width
     if (!products_ready) mid_prefetch_head(p, h, q, id, t, nt);
     cp_async_commit();                                                          // group: head operands
     if constexpr (STATE == STATE_SMEM) {
@@ -228,7 +221,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 for (int l = 0; l < L; ++l) cp_async_16(u_s + ((size_t)l * GPT + g) * nt + t, p.u + (long long)l * p.lstride + base[g]);
     }
     cp_async_commit();                                                          // group: u
-    const int label = p.train ? p.labels[id] : 0;
+    const int label = p.train ? p.labels[id] : 0;                               // fetched long before the head needs it
     if (!products_ready) {
         cp_async_wait_group<1>();                                               // head operands have landed ...
         __syncthreads();                                                        // ... those of every thread
@@ -249,6 +242,14 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     for (int g = 0; g < GPT; ++g) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) { mask[g][e] = 0u; ap[g][e] = 0.f; }      // a_0 = 0
+        if constexpr (STATE == STATE_PARKED) {
+            // the chain ran in the down-projection kernel's epilogue: only the gate words are fetched
+            if (live[g] && ACT == PAC_ACT_RELU && p.train) {
+                const uint4 gw = *reinterpret_cast<const uint4*>(p.gates + base[g]);
+                mask[g][0] = gw.x; mask[g][1] = gw.y; mask[g][2] = gw.z; mask[g][3] = gw.w;
+            }
+            continue;
+        }
         if (live[g]) {
 #pragma unroll 1
             for (int l0 = 0; l0 < L; l0 += 4) {
@@ -289,13 +290,23 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     // column sums over this CTA's tokens: `parts` partial sums per column over contiguous token
     // ranges, then added in range order
     {
-        const int parts = max(1, min(nt / r, p.Sg));
-        const int per = (p.Sg + parts - 1) / parts;
-        if (t < parts * r) {
-            const int j = t % r, part = t / r;
-            float acc = 0.f;
-            for (int sl = part * per; sl < min(p.Sg, (part + 1) * per); ++sl) acc += aL[(size_t)sl * r + j];
-            lred[part * r + j] = acc;
+        int parts = 1;
+        if constexpr (STATE == STATE_PARKED) {
+            // token-group sums from the down-projection kernel; CTA q of the cluster takes groups q, q + G, ...
+            if (t < r) {
+                float acc = 0.f;
+                for (int pp = q; pp < p.n_pool_parts; pp += p.G) acc += p.pool_part[((long long)b * p.n_pool_parts + pp) * r + t];
+                lred[t] = acc;
+            }
+        } else {
+            parts = max(1, min(nt / r, p.Sg));
+            const int per = (p.Sg + parts - 1) / parts;
+            if (t < parts * r) {
+                const int j = t % r, part = t / r;
+                float acc = 0.f;
+                for (int sl = part * per; sl < min(p.Sg, (part + 1) * per); ++sl) acc += aL[(size_t)sl * r + j];
+                lred[part * r + j] = acc;
+            }
         }
         __syncthreads();
         if (t < r) {
@@ -303,57 +314,83 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             for (int part = 0; part < parts; ++part) acc += lred[part * r + t];
             colsum[t] = acc;
         }
+        // What the head needs of a_L is its token sum times the head's product matrix; this CTA's tokens'
+        // share of that, plq[c] = sum_j colsum[j] prod[j][c], is formed here (warp c), so that only C numbers
+        // per CTA cross the cluster on the way to the logits.
+        for (int c = warp; c < C; c += nwarps) {
+            float pl = 0.f;
+            for (int j = lane; j < r; j += 32) {
+                float cs = 0.f;
+                for (int part = 0; part < parts; ++part) cs += lred[part * r + j];
+                pl = fmaf(cs, prod[j * C + c], pl);
+            }
+            pl = warp_sum(pl);
+            if (lane == 0) plq[c] = pl;
+        }
     }
     cluster.sync();
-    for (int j = t; j < r; j += nt) {
-        float acc = 0.f;
-        for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(colsum, g)[j];
-        pooled[j] = acc / (float)p.S;                     // mean_s a_L
+    // ---- head, by ONE warp: logits from the cluster's C-vectors, loss, dlogits, d loss / d a_L; everybody
+    // else waits at one block barrier.  The same in every CTA of the cluster.  A second warp of the first
+    // CTA forms mean_s a_L for the gradient finalisation meanwhile.
+    if (warp == 0) {
+        float mylogit = -INFINITY;                        // lane c holds logit c (C <= 32)
+        if (lane < C) {
+            float acc = 0.f;
+            for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(plq, g)[lane];
+            mylogit = prod[r * C + lane] + acc / (float)p.S;      // b_head + (mean_s h_L) W_head + (mean_s a_L)(W_up W_head)
+            if (q == 0) p.logits_out[(long long)b * C + lane] = mylogit;
+        }
+        if (p.train) {
+            const float mx = warp_max(mylogit);
+            const float ex = lane < C ? expf(mylogit - mx) : 0.f;
+            const float se = warp_sum(ex);
+            const float lab_logit = __shfl_sync(0xffffffffu, mylogit, label);
+            if (lane == 0 && q == 0) p.loss_b[b] = mx + logf(se) - lab_logit;
+            const float my = lane < C ? (ex / se - (lane == label ? 1.f : 0.f)) / (float)p.B : 0.f;     // dlogits
+            if (lane < C) {
+                lg[lane] = my;
+                if (q == 0) p.dlogits[(long long)b * C + lane] = my;
+            }
+            __syncwarp();
+            for (int j = lane; j < r; j += 32) {
+                float acc = 0.f;
+                for (int c = 0; c < C; ++c) acc = fmaf(prod[j * C + c], lg[c], acc);
+                daL[j] = acc / (float)p.S;                // da_L, the same for every token of the sample
+            }
+        }
+    } else if (warp == 1 && q == 0 && p.train) {
+        for (int j = lane; j < r; j += 32) {
+            float acc = 0.f;
+            for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(colsum, g)[j];
+            p.pooled_a[(long long)b * r + j] = acc / (float)p.S;      // mean_s a_L
+        }
     }
     // That was this CTA's last access to a peer's shared memory: say so now and wait, at the very end, only
     // for the peers to have said the same (a CTA must not exit while a peer may still read its memory).
     cluster.barrier_arrive();
     __syncthreads();
-
-    // ---- head: logits, loss, dlogits and d loss / d a_L, the same in every CTA of the cluster ----
-    if (t < C) {
-        float acc = prod[r * C + t];                      // b_head + (mean_s h_L) W_head
-        for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], prod[j * C + t], acc);
-        lg[t] = acc;
-        if (q == 0) p.logits_out[(long long)b * C + t] = acc;
-    }
-    __syncthreads();
     if (!p.train) {
         cluster.barrier_wait();                           // peers may still be reading this CTA's shared memory
         return;
     }
-    {
-        float mx = -INFINITY;
-        for (int c = 0; c < C; ++c) mx = fmaxf(mx, lg[c]);
-        float se = 0.f;
-        for (int c = 0; c < C; ++c) se += expf(lg[c] - mx);
-        const float my = (t < C) ? (expf(lg[t] - mx) / se - (t == label ? 1.f : 0.f)) / (float)p.B : 0.f;
-        if (t == 0 && q == 0) p.loss_b[b] = mx + logf(se) - lg[label];
-        __syncthreads();
-        if (t < C) {
-            lg[t] = my;                                   // dlogits
-            if (q == 0) p.dlogits[(long long)b * C + t] = my;
-        }
-        __syncthreads();
-    }
-    for (int j = t; j < r; j += nt) {
-        float acc = 0.f;
-        for (int c = 0; c < C; ++c) acc = fmaf(prod[j * C + c], lg[c], acc);
-        daL[j] = acc / (float)p.S;                         // da_L, the same for every token of the sample
-    }
-    __syncthreads();
 
-    // ---- reverse chain ----
-    float da[GPT][4];
+    // ---- reverse chain, in closed form.  da_L is the same vector for every token of the sample and a ReLU
+    // gate only ever multiplies by exactly 1 or 0, so for an element whose gates l..L are all open
+    //     dz_l = da_L[j] * prod_{l' > l} (1 - lambda_l'),   du_l = lambda_l dz_l,
+    // and 0 as soon as one gate at or above l is closed (cprod[l] holds the product, formed once per CTA in
+    // layer order).  No value depends on another layer's, so four layers are in flight at a time, the warp
+    // sums of this thread's shares of dlambda_l = sum gate * dz_l * (u_l - a_{l-1}) included. ----
+    float daLr[GPT][4];
 #pragma unroll
     for (int g = 0; g < GPT; ++g)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) da[g][e] = live[g] ? daL[j4[g] + e] : 0.f;
+        for (int e = 0; e < 4; ++e) daLr[g][e] = live[g] ? daL[j4[g] + e] : 0.f;
+    unsigned closed[GPT][4];                              // bit l set: the gate of layer l is closed
+#pragma unroll
+    for (int g = 0; g < GPT; ++g)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            closed[g][e] = (ACT == PAC_ACT_RELU) ? (~mask[g][e] & (L >= 32 ? 0xffffffffu : ((1u << L) - 1u))) : 0u;
 #pragma unroll 1
     for (int l0 = L - 1; l0 >= 0; l0 -= 4) {
         float4 wq[4][GPT];
@@ -362,23 +399,23 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
 #pragma unroll
             for (int g = 0; g < GPT; ++g)
                 if (l0 - i >= 0 && live[g]) wq[i][g] = load_w(l0 - i, g);
+        float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int l = l0 - i;
             if (l >= 0) {
-                const float lm = lam_s[l];
-                float part = 0.f;
 #pragma unroll
                 for (int g = 0; g < GPT; ++g) {
                     if (live[g]) {
+                        const float cp = cprod[l], lm = lam_s[l];
                         const float wv[4] = {wq[i][g].x, wq[i][g].y, wq[i][g].z, wq[i][g].w};
                         float dv[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float dz = (ACT == PAC_ACT_RELU) ? (((mask[g][e] >> l) & 1u) ? da[g][e] : 0.f) : da[g][e];
-                            part = fmaf(dz, wv[e], part);
-                            dv[e] = lm * dz;                           // du_l
-                            da[g][e] = (1.f - lm) * dz;                // da_{l-1}
+                            const bool open = (closed[g][e] >> l) == 0u;       // gates l .. L all open
+                            const float dz = open ? daLr[g][e] * cp : 0.f;
+                            part[i] = fmaf(dz, wv[e], part[i]);
+                            dv[e] = lm * dz;                                   // du_l
                         }
                         DU* dst = du + (long long)l * p.lstride + base[g];
                         if constexpr (sizeof(DU) == 2) {
@@ -392,29 +429,18 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                         }
                     }
                 }
-                part = warp_sum(part);                             // this warp's share of dlambda_l
-                if (lane == 0) lred[warp * LT + l] = part;
             }
         }
+        // this warp's shares of dlambda of the four layers: four independent shuffle trees
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) part[i] += __shfl_xor_sync(0xffffffffu, part[i], o);
+        if (lane == 0)
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (l0 - i >= 0) lred[warp * LT + (l0 - i)] = part[i];
     }
-    // ---- per-sample vectors the gradient finalisation needs, for this CTA's slice of the hidden
-    // width: mean_s y = mean_s h_L + (mean_s a_L) W_up  and  g = d loss / d mean_s y = W_head dlogits ----
-    for (int kk = t; kk < kn; kk += nt) {
-        const int k = k0 + kk;
-        float acc = 0.f;
-        if (p.wup_smem) {
-#pragma unroll 8
-            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], wup_s[(size_t)j * p.dg + kk], acc);
-        } else {
-            for (int j = 0; j < r; ++j) acc = fmaf(pooled[j], p.W_up[(long long)j * p.d + k], acc);
-        }
-        float gv = 0.f;
-        for (int c = 0; c < C; ++c) gv = fmaf(wh_s[kk * C + c], lg[c], gv);
-        p.pooled_y[(long long)b * p.d + k] = py[kk] + acc;
-        p.gvec[(long long)b * p.d + k] = gv;
-    }
-    if (q == 0)
-        for (int j = t; j < r; j += nt) p.pooled_a[(long long)b * r + j] = pooled[j];
     __syncthreads();
     if (t < L) {
         float acc = 0.f;
@@ -425,16 +451,16 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
 }
 
 // The stand-alone kernel: u comes from the global buffer written by the down-projection kernel.
-template <int ACT, typename DU, int GPT, bool SMEM_STATE>
-__global__ void __launch_bounds__(512, SMEM_STATE ? 1 : 2) mid_cls_kernel(MidParams p) {
+template <int ACT, typename DU, int GPT, int STATE>
+__global__ void __launch_bounds__(512, STATE == STATE_SMEM ? 1 : 2) mid_cls_kernel(MidParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ float4 sm4[];
     float4* u_s = sm4;                           // [L][GPT][nt] each thread's own u values, later u_l - a_{l-1}
-    float* sm = reinterpret_cast<float*>(sm4 + (SMEM_STATE ? (size_t)p.L * GPT * blockDim.x : 0));
+    float* sm = reinterpret_cast<float*>(sm4 + (STATE == STATE_SMEM ? (size_t)p.L * GPT * blockDim.x : 0));
     const MidShared h = mid_carve(sm, p);
     pdl_trigger();
-    pdl_wait();             // u comes from the kernel before this one
-    mid_body<ACT, DU, GPT, SMEM_STATE ? STATE_SMEM : STATE_DU>(p, cluster, u_s, h, false);
+    pdl_wait();             // u (or the parked chain state) comes from the kernel before this one
+    mid_body<ACT, DU, GPT, STATE>(p, cluster, u_s, h, false);
 }
 
 // ---------------------------------------------------------------------------
@@ -449,10 +475,12 @@ struct FinalizeParams {
     int B, d, r, C, L;
     const float* dw_part; int splits; long long dw_elems;     // splits <= 1: W_down gradient already in grads
     const float* lam_part; int lam_blocks;
-    const float *pooled_a, *gvec, *pooled_y, *dlogits, *loss_b;
+    const float *pooled_a, *dlogits, *loss_b;                // per-sample vectors the forward half left: mean_s a_L, dlogits, loss
+    const float* hbar; const int* ids; long long N;          // token mean of the last cached layer, per cache sample; the batch's ids
+    const float* params_in;                                  // the parameters the forward half used (W_up, W_head are read)
     float* grads; float* loss_out;
     int wd_blocks;                                           // blocks that handle W_down, 4 elements per thread
-    int rest_blocks;                                         // blocks that handle W_up, W_head, b_head, one element per thread
+    int rest_blocks;                                         // blocks that handle the head side: FIN_KB columns of the hidden width each
     // AdamW
     int adam;
     float *params, *m, *v;
@@ -467,6 +495,8 @@ struct FinalizeParams {
     // are not trustworthy, so nothing is written to the gradients, parameters or moments.
     unsigned* status;
 };
+
+constexpr int FIN_KB = 4;       // hidden-width columns per head-side block of the finalisation kernel
 
 __device__ __forceinline__ unsigned ld_acquire_sys(const unsigned* p) {
     unsigned v;
@@ -542,31 +572,67 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         return;
     }
     if (blk < f.rest_blocks) {
-        // head parameters: like block 0 they need only the forward half's per-sample vectors, so these blocks
-        // finish (and make room for the W_down blocks) while the second pass still runs
-        const long long i = lay.lam + (long long)blk * blockDim.x + threadIdx.x;
-        if (i >= lay.total || dead) return;
-        float g;
-        if (i < lay.w_up) return;                            // lambda is handled by block 0
-        if (i < lay.w_head) {
-            const long long e = i - lay.w_up;
-            const int j = (int)(e / f.d), k = (int)(e - (long long)j * f.d);
-            g = 0.f;
-#pragma unroll 16
-            for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], f.gvec[(long long)b * f.d + k], g);
-        } else if (i < lay.b_head) {
-            const long long e = i - lay.w_head;
-            const int k = (int)(e / f.C), c = (int)(e - (long long)k * f.C);
-            g = 0.f;
-#pragma unroll 16
-            for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_y[(long long)b * f.d + k], f.dlogits[(long long)b * f.C + c], g);
-        } else {
-            const int c = (int)(i - lay.b_head);
-            g = 0.f;
-            for (int b = 0; b < f.B; ++b) g += f.dlogits[(long long)b * f.C + c];
+        // Head-side parameters: like block 0 these blocks need only what the forward half left behind, so
+        // they finish (and make room for the W_down blocks) while the second pass still runs.  A block owns
+        // FIN_KB columns k of the hidden width: W_up[:, k] and W_head[k, :] (the last block also b_head).
+        // It first rebuilds, for its columns, the two per-sample vectors of the head's backward,
+        //     g[b][k]  = d loss / d mean_s y = sum_c W_head[k][c] dlogits[b][c]
+        //     py[b][k] = mean_s y = hbar[id_b][k] + sum_j pooled_a[b][j] W_up[j][k]
+        // from the OLD values of exactly the parameters it owns (read before any of them is updated), then
+        //     dW_up[j][k] = sum_b pooled_a[b][j] g[b][k],   dW_head[k][c] = sum_b py[b][k] dlogits[b][c].
+        extern __shared__ float fsm[];
+        float* g_s = fsm;                                    // [B][FIN_KB]
+        float* py_s = g_s + (size_t)f.B * FIN_KB;            // [B][FIN_KB]
+        float* wup_s = py_s + (size_t)f.B * FIN_KB;          // [r][FIN_KB]   old W_up[:, k0..]
+        float* wh_s = wup_s + (size_t)f.r * FIN_KB;          // [FIN_KB][C]   old W_head[k0.., :]
+        const int k0 = blk * FIN_KB, kn = min(FIN_KB, f.d - k0), t = threadIdx.x, nt = blockDim.x;
+        const float* W_up = f.params_in + lay.w_up;
+        const float* W_head = f.params_in + lay.w_head;
+        if (dead) return;
+        for (int e = t; e < f.r * FIN_KB; e += nt) {
+            const int j = e / FIN_KB, kk = e - j * FIN_KB;
+            wup_s[e] = kk < kn ? W_up[(long long)j * f.d + k0 + kk] : 0.f;
         }
-        f.grads[i] = g;
-        if (f.adam) adamw_element(f.params, f.m, f.v, i, g * f.grad_scale, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        for (int e = t; e < FIN_KB * f.C; e += nt) {
+            const int kk = e / f.C;
+            wh_s[e] = kk < kn ? W_head[(long long)k0 * f.C + e] : 0.f;
+        }
+        __syncthreads();
+        for (int e = t; e < f.B * FIN_KB; e += nt) {
+            const int b = e / FIN_KB, kk = e - b * FIN_KB;
+            float gv = 0.f, acc = 0.f;
+            for (int c = 0; c < f.C; ++c) gv = fmaf(wh_s[kk * f.C + c], f.dlogits[(long long)b * f.C + c], gv);
+            for (int j = 0; j < f.r; ++j) acc = fmaf(f.pooled_a[(long long)b * f.r + j], wup_s[j * FIN_KB + kk], acc);
+            const long long id = safe_id(f.ids, b, f.N, nullptr);
+            g_s[e] = gv;
+            py_s[e] = kk < kn ? f.hbar[id * f.d + k0 + kk] + acc : 0.f;
+        }
+        __syncthreads();
+        const int n_up = f.r * FIN_KB, n_head = FIN_KB * f.C;
+        const bool last = blk == f.rest_blocks - 1;
+        for (int e = t; e < n_up + n_head + (last ? f.C : 0); e += nt) {
+            long long i;
+            float g = 0.f;
+            if (e < n_up) {
+                const int j = e / FIN_KB, kk = e - j * FIN_KB;
+                if (kk >= kn) continue;
+                i = lay.w_up + (long long)j * f.d + k0 + kk;
+#pragma unroll 8
+                for (int b = 0; b < f.B; ++b) g = fmaf(f.pooled_a[(long long)b * f.r + j], g_s[b * FIN_KB + kk], g);
+            } else if (e < n_up + n_head) {
+                const int kk = (e - n_up) / f.C, c = (e - n_up) - kk * f.C;
+                if (kk >= kn) continue;
+                i = lay.w_head + (long long)(k0 + kk) * f.C + c;
+#pragma unroll 8
+                for (int b = 0; b < f.B; ++b) g = fmaf(py_s[b * FIN_KB + kk], f.dlogits[(long long)b * f.C + c], g);
+            } else {
+                const int c = e - n_up - n_head;
+                i = lay.b_head + c;
+                for (int b = 0; b < f.B; ++b) g += f.dlogits[(long long)b * f.C + c];
+            }
+            f.grads[i] = g;
+            if (f.adam) adamw_element(f.params, f.m, f.v, i, g * f.grad_scale, f.lay, f.hp, f.bc1, f.bc2, f.wdT, f.d, f.r);
+        }
         return;
     }
     pdl_wait();
@@ -597,7 +663,7 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
 // group per thread, chain state in shared memory.
 struct MidPlan {
     bool ok = false;
-    int G = 1, Sg = 0, dg = 0, threads = 0, scratch = 0, wup_smem = 0;
+    int G = 1, Sg = 0, dg = 0, threads = 0, scratch = 0;
     int gpt = 1, smem_state = 1;      // 4-column groups per thread; chain state in shared memory or parked in the du buffer
     size_t smem = 0;
 };
@@ -609,8 +675,8 @@ inline size_t mid_base_floats(const Dims& dm, int Sg, int dg, int th, int* scrat
     const int parts = th / dm.r > 0 ? th / dm.r : 1;
     if (parts * dm.r > scratch) scratch = parts * dm.r;
     *scratch_out = scratch;
-    return (size_t)Sg * dm.r + 3 * (size_t)dm.r + 2 * (size_t)(dm.r + 1) * dm.C + (size_t)dg + MID_MAX_C + MID_MAX_L + scratch +
-           (size_t)dg * dm.C + 4;
+    return (size_t)Sg * dm.r + 2 * (size_t)dm.r + MID_MAX_C + 2 * (size_t)(dm.r + 1) * dm.C + (size_t)dg + MID_MAX_C + MID_MAX_L + scratch +
+           (size_t)dg * dm.C + MID_MAX_L + 4;
 }
 
 inline MidPlan mid_plan(const Dims& dm) {
@@ -627,10 +693,7 @@ inline MidPlan mid_plan(const Dims& dm) {
         int scratch;
         size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch) + 4 * (size_t)dm.L * th;
         if (floats > budget) continue;
-        const size_t wup = (size_t)dm.r * dg;
         mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch; mp.gpt = 1; mp.smem_state = 1;
-        mp.wup_smem = floats + wup <= budget ? 1 : 0;
-        if (mp.wup_smem) floats += wup;
         mp.smem = sizeof(float) * floats;
         mp.ok = true;
         return mp;
@@ -646,20 +709,40 @@ inline MidPlan mid_plan(const Dims& dm) {
         int scratch;
         size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
         if (floats > budget) return mp;
-        const size_t wup = (size_t)dm.r * dg;
         mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch; mp.gpt = gpt; mp.smem_state = 0;
-        mp.wup_smem = floats + wup <= 96 * 1024 / sizeof(float) ? 1 : 0;     // keep several CTAs per SM
-        if (mp.wup_smem) floats += wup;
         mp.smem = sizeof(float) * floats;
         mp.ok = true;
     }
     return mp;
 }
 
-template <int ACT, typename DU, int GPT, bool SMEM_STATE>
+// Geometry for the parked mode: the chain state never needs shared memory, so the smallest cluster with at
+// most four 4-column groups per thread serves (fewer, fuller CTAs than the plan above).
+inline MidPlan mid_plan_parked(const Dims& dm) {
+    MidPlan mp;
+    if (dm.r % 4 != 0 || dm.C > MID_MAX_C || dm.L > MID_MAX_L) return mp;
+    for (int G = 1; G <= 8; G *= 2) {
+        const int Sg = (dm.S + G - 1) / G, dg = (dm.d + G - 1) / G;
+        const long long need = (long long)Sg * (dm.r / 4);
+        if (need > 4 * 512) continue;
+        const int gpt = need <= 512 ? 1 : need <= 1024 ? 2 : 4;
+        int th = (int)(((need + gpt - 1) / gpt + 31) / 32 * 32);
+        if (th < 128) th = 128;
+        int scratch;
+        const size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
+        if (floats > 96 * 1024 / sizeof(float)) continue;
+        mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch; mp.gpt = gpt; mp.smem_state = 0;
+        mp.smem = sizeof(float) * floats;
+        mp.ok = true;
+        return mp;
+    }
+    return mp;
+}
+
+template <int ACT, typename DU, int GPT, int STATE>
 inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
     {
-        cudaError_t e = smem_opt_in((const void*)mid_cls_kernel<ACT, DU, GPT, SMEM_STATE>, MID_SMEM_BUDGET);
+        cudaError_t e = smem_opt_in((const void*)mid_cls_kernel<ACT, DU, GPT, STATE>, MID_SMEM_BUDGET);
         if (e != cudaSuccess) return e;
     }
     cudaLaunchConfig_t cfg = {};
@@ -676,17 +759,30 @@ inline cudaError_t mid_launch_one(const MidPlan& mp, const MidParams& p, cudaStr
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, DU, GPT, SMEM_STATE>, p);
+    return cudaLaunchKernelEx(&cfg, mid_cls_kernel<ACT, DU, GPT, STATE>, p);
 }
 
 template <int ACT, typename DU>
 inline cudaError_t mid_launch_shape(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
-    if (mp.smem_state) return mid_launch_one<ACT, DU, 1, true>(mp, p, stream);
+    if (mp.smem_state) return mid_launch_one<ACT, DU, 1, STATE_SMEM>(mp, p, stream);
     switch (mp.gpt) {
-        case 1: return mid_launch_one<ACT, DU, 1, false>(mp, p, stream);
-        case 2: return mid_launch_one<ACT, DU, 2, false>(mp, p, stream);
-        default: return mid_launch_one<ACT, DU, 4, false>(mp, p, stream);
+        case 1: return mid_launch_one<ACT, DU, 1, STATE_DU>(mp, p, stream);
+        case 2: return mid_launch_one<ACT, DU, 2, STATE_DU>(mp, p, stream);
+        default: return mid_launch_one<ACT, DU, 4, STATE_DU>(mp, p, stream);
     }
+}
+
+// The same kernel behind a down-projection kernel that already ran the forward chain (bf16 state parked in du).
+template <int ACT>
+inline cudaError_t mid_launch_parked_act(const MidPlan& mp, const MidParams& p, cudaStream_t stream) {
+    switch (mp.gpt) {
+        case 1: return mid_launch_one<ACT, bf16, 1, STATE_PARKED>(mp, p, stream);
+        case 2: return mid_launch_one<ACT, bf16, 2, STATE_PARKED>(mp, p, stream);
+        default: return mid_launch_one<ACT, bf16, 4, STATE_PARKED>(mp, p, stream);
+    }
+}
+inline cudaError_t mid_launch_parked(const MidPlan& mp, const MidParams& p, int act, cudaStream_t stream) {
+    return act == PAC_ACT_RELU ? mid_launch_parked_act<PAC_ACT_RELU>(mp, p, stream) : mid_launch_parked_act<PAC_ACT_IDENTITY>(mp, p, stream);
 }
 
 inline cudaError_t mid_launch(const MidPlan& mp, const MidParams& p, int act, bool du_bf16, cudaStream_t stream) {

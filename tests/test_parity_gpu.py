@@ -293,9 +293,14 @@ def tc_check(spec, max_batch, act, ids=None, loss_tol=2e-2, chain_tol=1e-2, head
     ids = ids or [spec.N - 1, 0, 5, 5][:spec.B]
     ctx = case.context(max_batch=max_batch, act=act, kernel_path=kernel_path)
     can_fuse = spec.head == "cls" and spec.S <= 128 and spec.r <= 64
-    if kernel_path == 0:          # automatic: one forward launch when the batch's clusters fit the device at once
-        assert ctx.kernel_path() in (("tensor+fused_forward", "tensor") if can_fuse else ("tensor",))
+    can_chain = spec.head == "cls" and spec.r % 32 == 0 and spec.r <= 128 and spec.L <= 32
+    if kernel_path == 0:          # automatic: one forward launch when the batch's clusters fit the device at once,
+        #                           the chain in the down-projection epilogue when there are enough 128-token tiles
+        assert ctx.kernel_path() in ("tensor+fused_forward", "tensor", "tensor+chain_forward")
         assert ctx.kernel_path() == "tensor+fused_forward" or not can_fuse or max_batch > 8
+        assert ctx.kernel_path() != "tensor+chain_forward" or (can_chain and 2 * max_batch * ((spec.S + 127) // 128) >= 100)
+    elif kernel_path == 4:
+        assert ctx.kernel_path() == ("tensor+chain_forward" if can_chain else "tensor")
     else:
         assert ctx.kernel_path() == ("tensor+fused_forward" if can_fuse and kernel_path == 3 else "tensor")
     flat = pi.random_params(spec, 3)
@@ -325,6 +330,37 @@ def test_tensor_path_loss_and_gradients(spec, max_batch, act):
 def test_tensor_path_separate_forward_kernels(spec, max_batch, act):
     """The same shapes with the down-projections and the head phase as two launches."""
     tc_check(spec, max_batch, act, kernel_path=2)
+
+
+TC_CHAIN_FORWARD = [s for s in TC_SPECS if s[0].r % 32 == 0 and s[0].r <= 128] + [
+    (TC_BASE.scaled(name="tc_chain_r96", S=200, d=264, r=96, L=5, B=3), 3, 0),        # three 16-column chunks per warp, ragged S
+    (TC_BASE.scaled(name="tc_chain_L32", S=130, d=128, r=32, L=32, B=2, N=6), 2, 0),  # every gate bit in use
+]
+
+
+@pytest.mark.parametrize("spec,max_batch,act", TC_CHAIN_FORWARD, ids=[s[0].name for s in TC_CHAIN_FORWARD])
+def test_tensor_path_chain_in_epilogue_forward(spec, max_batch, act):
+    """The merge / activation chain in the epilogue of the down-projection kernel (the path long
+    sequences take): same bounds as the other tensor-core variants, and evaluation against the oracle."""
+    ctx, case = tc_check(spec, max_batch, act, kernel_path=4)
+    ids = [spec.N - 1, 0, 5, 5][:spec.B]
+    flat = pi.random_params(spec, 3)
+    out = torch.zeros((len(ids), spec.n_out), dtype=torch.float32, device="cuda")
+    ctx.eval_logits(ids, out)
+    ctx.sync()
+    ref = po.eval_logits(case.oracle_params(flat), case.H(ids), act)
+    assert rel_l2(out.cpu().numpy(), ref) < 1e-3
+
+
+def test_chain_in_epilogue_forward_ten_steps():
+    """T5-Large layer shape (L=24, S=256, d=1024, r=128, outlier channels) on a short cache: 10 AdamW steps."""
+    spec = pi.CONFIGS["t5_large"].scaled(N=48, B=4, name="t5_large_short")
+    case = Case(spec, materialize_cpu=False)
+    ctx, losses, ref_losses, p, ref_p, p0 = run_trajectory(case, 10, kernel_path=4)
+    assert ctx.kernel_path() == "tensor+chain_forward"
+    assert np.all(np.abs(losses - ref_losses) <= 2e-2 * np.abs(ref_losses))
+    assert rel_l2(p, ref_p) < 1e-2
+    assert rel_l2(p - p0, ref_p - p0) < UPDATE_TOL
 
 
 @pytest.mark.parametrize("spec,max_batch,act", TC_ONE_KERNEL_FORWARD, ids=[s[0].name for s in TC_ONE_KERNEL_FORWARD])
