@@ -563,7 +563,7 @@ MidParams mid_params(pac_ctx* c, const MidPlan& mp, const int* d_ids, int B, boo
     p.ids = d_ids; p.N = dm.N; p.labels = c->labels;
     p.L = dm.L; p.S = dm.S; p.d = dm.d; p.r = dm.r; p.C = dm.C; p.B = B;
     p.G = mp.G; p.Sg = mp.Sg; p.dg = mp.dg; p.train = train ? 1 : 0;
-    p.scratch = mp.scratch;
+    p.scratch = mp.scratch; p.aL_floats = (&mp == &c->pplan) ? 0 : mp.Sg * dm.r;
     p.u = sc.u; p.lstride = (long long)c->max_rows * dm.r;
     p.lam = c->params + c->lay.lam; p.W_up = c->params + c->lay.w_up;
     p.W_head = c->params + c->lay.w_head; p.b_head = c->params + c->lay.b_head; p.hbar = sc.hbar;

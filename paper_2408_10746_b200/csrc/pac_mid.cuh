@@ -12,6 +12,7 @@
 // All cross-thread sums use a fixed order, so results are bit-reproducible.
 #pragma once
 #include <cooperative_groups.h>
+#include <type_traits>
 
 #include "pac_common.cuh"
 #include "pac_simt.cuh"
@@ -29,6 +30,7 @@ struct MidParams {
     int dg;                     // head columns per CTA = ceil(d / G)
     int train;
     int scratch;                // floats of block-local reduction scratch
+    int aL_floats;              // floats of the a_L tile in shared memory (Sg * r; 0 when the chain ran elsewhere)
     int layers_per_cta;         // one-kernel forward: layers whose down-projections each CTA of the cluster computes
     int host_ids;               // 1: ids points at host memory the device can read (written before the launch, so
                                 // it may be read ahead of the predecessor's completion); read once per CTA
@@ -54,10 +56,14 @@ struct MidParams {
 
 constexpr int MID_MAX_C = 32;
 constexpr size_t MID_SMEM_BUDGET = 220 * 1024;    // dynamic shared memory the fused kernel may use
+constexpr int MID_RING = 4;       // layers of parked state in flight per thread in the reverse pass of long sequences
 constexpr int MID_MAX_L = 32;     // ReLU masks of all layers live in one 32-bit word per element
 
 __device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
 }
 __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
@@ -84,7 +90,7 @@ __device__ __forceinline__ MidShared mid_carve(float* sm, const MidParams& p) {
     MidShared h;
     const size_t rc = (size_t)(p.r + 1) * p.C;
     h.aL = sm;                                        // [Sg][r]   a_L of this CTA's tokens
-    h.colsum = h.aL + (size_t)p.Sg * p.r;             // [r]       exchanged through DSMEM
+    h.colsum = h.aL + (size_t)p.aL_floats;            // [r]       exchanged through DSMEM
     h.prodq = h.colsum + p.r;                         // [r+1][C]  this CTA's partial head products, exchanged
     h.prod = h.prodq + rc;                            // [r+1][C]  their sum over the cluster
     h.plq = h.prod + rc;                              // [MID_MAX_C] this CTA's tokens' share of S * (mean_s a_L)(W_up W_head), exchanged
@@ -391,55 +397,91 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
 #pragma unroll
         for (int e = 0; e < 4; ++e)
             closed[g][e] = (ACT == PAC_ACT_RELU) ? (~mask[g][e] & (L >= 32 ? 0xffffffffu : ((1u << L) - 1u))) : 0u;
-#pragma unroll 1
-    for (int l0 = L - 1; l0 >= 0; l0 -= 4) {
-        float4 wq[4][GPT];
+    // one layer of one group: du_l out, this thread's share of dlambda_l added to `part`
+    auto reverse_step = [&](int l, int g, const float4& w4, float& part) {
+        const float cp = cprod[l], lm = lam_s[l];
+        const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
+        float dv[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int g = 0; g < GPT; ++g)
-                if (l0 - i >= 0 && live[g]) wq[i][g] = load_w(l0 - i, g);
-        float part[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int l = l0 - i;
+        for (int e = 0; e < 4; ++e) {
+            const bool open = (closed[g][e] >> l) == 0u;       // gates l .. L all open
+            const float dz = open ? daLr[g][e] * cp : 0.f;
+            part = fmaf(dz, wv[e], part);
+            dv[e] = lm * dz;                                   // du_l
+        }
+        DU* dst = du + (long long)l * p.lstride + base[g];
+        if constexpr (sizeof(DU) == 2) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
+            uint2 pk;
+            pk.x = *reinterpret_cast<unsigned*>(&lo);
+            pk.y = *reinterpret_cast<unsigned*>(&hi);
+            *reinterpret_cast<uint2*>(dst) = pk;
+        } else {
+            *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
+        }
+    };
+    if constexpr (STATE == STATE_PARKED) {
+        // Long sequences: the reverse pass is a pure stream over the parked state.  It is fetched through a
+        // ring of MID_RING layers in shared memory (cp.async, each thread reads back only what it requested),
+        // so that GPT * MID_RING loads per thread are in flight without holding registers.
+        uint2* ring = reinterpret_cast<uint2*>(u_s);
+        auto request = [&](int l) {
             if (l >= 0) {
 #pragma unroll
-                for (int g = 0; g < GPT; ++g) {
-                    if (live[g]) {
-                        const float cp = cprod[l], lm = lam_s[l];
-                        const float wv[4] = {wq[i][g].x, wq[i][g].y, wq[i][g].z, wq[i][g].w};
-                        float dv[4];
+                for (int g = 0; g < GPT; ++g)
+                    if (live[g]) cp_async_8(ring + ((size_t)(l % MID_RING) * GPT + g) * nt + t, du + (long long)l * p.lstride + base[g]);
+            }
+            cp_async_commit();
+        };
+        for (int i = 0; i < MID_RING; ++i) request(L - 1 - i);
+#pragma unroll 1
+        for (int l = L - 1; l >= 0; --l) {
+            cp_async_wait_group<MID_RING - 1>();
+            float part = 0.f;
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const bool open = (closed[g][e] >> l) == 0u;       // gates l .. L all open
-                            const float dz = open ? daLr[g][e] * cp : 0.f;
-                            part[i] = fmaf(dz, wv[e], part[i]);
-                            dv[e] = lm * dz;                                   // du_l
-                        }
-                        DU* dst = du + (long long)l * p.lstride + base[g];
-                        if constexpr (sizeof(DU) == 2) {
-                            __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
-                            uint2 pk;
-                            pk.x = *reinterpret_cast<unsigned*>(&lo);
-                            pk.y = *reinterpret_cast<unsigned*>(&hi);
-                            *reinterpret_cast<uint2*>(dst) = pk;
-                        } else {
-                            *reinterpret_cast<float4*>(dst) = make_float4(dv[0], dv[1], dv[2], dv[3]);
-                        }
-                    }
+            for (int g = 0; g < GPT; ++g) {
+                if (live[g]) {
+                    const uint2 x = ring[((size_t)(l % MID_RING) * GPT + g) * nt + t];
+                    const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.x));
+                    const float2 c2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.y));
+                    reverse_step(l, g, make_float4(a2.x, a2.y, c2.x, c2.y), part);
                 }
             }
+            request(l - MID_RING);
+            part = warp_sum(part);
+            if (lane == 0) lred[warp * LT + l] = part;
         }
-        // this warp's shares of dlambda of the four layers: four independent shuffle trees
+    } else {
+        // layers per batch: about four state loads in flight per thread whatever the number of groups it owns
+        constexpr int LB = GPT >= 4 ? 1 : 4 / GPT;
+#pragma unroll 1
+        for (int l0 = L - 1; l0 >= 0; l0 -= LB) {
+            float4 wq[LB][GPT];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
+            for (int i = 0; i < LB; ++i)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) part[i] += __shfl_xor_sync(0xffffffffu, part[i], o);
-        if (lane == 0)
+                for (int g = 0; g < GPT; ++g)
+                    if (l0 - i >= 0 && live[g]) wq[i][g] = load_w(l0 - i, g);
+            float part[LB];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (l0 - i >= 0) lred[warp * LT + (l0 - i)] = part[i];
+            for (int i = 0; i < LB; ++i) {
+                part[i] = 0.f;
+                if (l0 - i >= 0) {
+#pragma unroll
+                    for (int g = 0; g < GPT; ++g)
+                        if (live[g]) reverse_step(l0 - i, g, wq[i][g], part[i]);
+                }
+            }
+            // this warp's shares of dlambda of the batch's layers: independent shuffle trees
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int i = 0; i < LB; ++i) part[i] += __shfl_xor_sync(0xffffffffu, part[i], o);
+            if (lane == 0)
+#pragma unroll
+                for (int i = 0; i < LB; ++i)
+                    if (l0 - i >= 0) lred[warp * LT + (l0 - i)] = part[i];
+        }
     }
     __syncthreads();
     if (t < L) {
@@ -456,7 +498,8 @@ __global__ void __launch_bounds__(512, STATE == STATE_SMEM ? 1 : 2) mid_cls_kern
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ float4 sm4[];
     float4* u_s = sm4;                           // [L][GPT][nt] each thread's own u values, later u_l - a_{l-1}
-    float* sm = reinterpret_cast<float*>(sm4 + (STATE == STATE_SMEM ? (size_t)p.L * GPT * blockDim.x : 0));
+    float* sm = reinterpret_cast<float*>(sm4 + (STATE == STATE_SMEM ? (size_t)p.L * GPT * blockDim.x
+                                               : STATE == STATE_PARKED ? (size_t)MID_RING * GPT * blockDim.x / 2 : 0));
     const MidShared h = mid_carve(sm, p);
     pdl_trigger();
     pdl_wait();             // u (or the parked chain state) comes from the kernel before this one
@@ -665,17 +708,18 @@ struct MidPlan {
     bool ok = false;
     int G = 1, Sg = 0, dg = 0, threads = 0, scratch = 0;
     int gpt = 1, smem_state = 1;      // 4-column groups per thread; chain state in shared memory or parked in the du buffer
+    int aL_floats = 0;                // a_L tile in shared memory (0: the chain ran in the down-projection kernel)
     size_t smem = 0;
 };
 
 // Shared-memory floats the kernel needs besides the chain state and the W_up slice.
-inline size_t mid_base_floats(const Dims& dm, int Sg, int dg, int th, int* scratch_out) {
+inline size_t mid_base_floats(const Dims& dm, int Sg, int dg, int th, int* scratch_out, bool with_aL = true) {
     const int nw = th / 32;
     int scratch = nw * MID_MAX_L;
     const int parts = th / dm.r > 0 ? th / dm.r : 1;
     if (parts * dm.r > scratch) scratch = parts * dm.r;
     *scratch_out = scratch;
-    return (size_t)Sg * dm.r + 2 * (size_t)dm.r + MID_MAX_C + 2 * (size_t)(dm.r + 1) * dm.C + (size_t)dg + MID_MAX_C + MID_MAX_L + scratch +
+    return (with_aL ? (size_t)Sg * dm.r : 0) + 2 * (size_t)dm.r + MID_MAX_C + 2 * (size_t)(dm.r + 1) * dm.C + (size_t)dg + MID_MAX_C + MID_MAX_L + scratch +
            (size_t)dg * dm.C + MID_MAX_L + 4;
 }
 
@@ -729,8 +773,8 @@ inline MidPlan mid_plan_parked(const Dims& dm) {
         int th = (int)(((need + gpt - 1) / gpt + 31) / 32 * 32);
         if (th < 128) th = 128;
         int scratch;
-        const size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch);
-        if (floats > 96 * 1024 / sizeof(float)) continue;
+        const size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch, false) + (size_t)MID_RING * gpt * th * 2;    // + the state ring (8 bytes per slot)
+        if (floats > 110 * 1024 / sizeof(float)) continue;                // two CTAs per SM
         mp.G = G; mp.Sg = Sg; mp.dg = dg; mp.threads = th; mp.scratch = scratch; mp.gpt = gpt; mp.smem_state = 0;
         mp.smem = sizeof(float) * floats;
         mp.ok = true;
