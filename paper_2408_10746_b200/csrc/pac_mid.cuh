@@ -398,8 +398,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int e = 0; e < 4; ++e)
             closed[g][e] = (ACT == PAC_ACT_RELU) ? (~mask[g][e] & (L >= 32 ? 0xffffffffu : ((1u << L) - 1u))) : 0u;
     // one layer of one group: du_l out, this thread's share of dlambda_l added to `part`
-    auto reverse_step = [&](int l, int g, const float4& w4, float& part) {
-        const float cp = cprod[l], lm = lam_s[l];
+    auto reverse_step = [&](int l, int g, const float4& w4, float& part, float cp, float lm) {
         const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
         float dv[4];
 #pragma unroll
@@ -438,13 +437,17 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int l = L - 1; l >= 0; --l) {
             cp_async_wait_group<MID_RING - 1>();
             float part = 0.f;
+            const float cp = cprod[l], lm = lam_s[l];          // read once per layer (the stores below could alias them)
+            uint2 x[GPT];
+#pragma unroll
+            for (int g = 0; g < GPT; ++g)
+                if (live[g]) x[g] = ring[((size_t)(l % MID_RING) * GPT + g) * nt + t];
 #pragma unroll
             for (int g = 0; g < GPT; ++g) {
                 if (live[g]) {
-                    const uint2 x = ring[((size_t)(l % MID_RING) * GPT + g) * nt + t];
-                    const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.x));
-                    const float2 c2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x.y));
-                    reverse_step(l, g, make_float4(a2.x, a2.y, c2.x, c2.y), part);
+                    const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x[g].x));
+                    const float2 c2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x[g].y));
+                    reverse_step(l, g, make_float4(a2.x, a2.y, c2.x, c2.y), part, cp, lm);
                 }
             }
             request(l - MID_RING);
@@ -467,9 +470,10 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             for (int i = 0; i < LB; ++i) {
                 part[i] = 0.f;
                 if (l0 - i >= 0) {
+                    const float cp = cprod[l0 - i], lm = lam_s[l0 - i];
 #pragma unroll
                     for (int g = 0; g < GPT; ++g)
-                        if (live[g]) reverse_step(l0 - i, g, wq[i][g], part[i]);
+                        if (live[g]) reverse_step(l0 - i, g, wq[i][g], part[i], cp, lm);
                 }
             }
             // this warp's shares of dlambda of the batch's layers: independent shuffle trees
