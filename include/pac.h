@@ -26,7 +26,9 @@
  *    context (allocated in pac_adapter_init, freed in pac_destroy).
  *  - Flat parameter layout (fp32), used by every get/set call:
  *        W_down[L][d][r] | lambda[L] | W_up[r][d] | W_head[d][C] | b_head[C]
- *    (the last two only with PAC_HEAD_MEANPOOL_CLS).
+ *    (the last two only with PAC_HEAD_MEANPOOL_CLS); with PAC_BODY_TRANSFORMER followed, for every
+ *    layer l = 0..L-1, by  g1[r] | b1[r] | Wq[r][r] | Wk[r][r] | Wv[r][r] | Wo[r][r] | g2[r] | b2[r] |
+ *    W1[r][f] | c1[f] | W2[f][r] | c2[r].
  *  - Every call returns a pac_status and never throws or aborts.  Arguments are
  *    checked on the host before any launch; on error no device state changes.
  *    pac_last_error() gives a message for the most recent failure on a context.
@@ -56,6 +58,15 @@ typedef enum {
 typedef enum { PAC_F32 = 0, PAC_BF16 = 1 } pac_dtype;
 typedef enum { PAC_ACT_RELU = 0, PAC_ACT_IDENTITY = 1 } pac_act;
 typedef enum { PAC_HEAD_MEANPOOL_CLS = 0, PAC_HEAD_FROZEN_LM = 1 } pac_head;
+/* Adapter body (Section IV-A): the point-wise activation `act`, or one reduced-width transformer
+ * encoder layer per adapter ("a lightweight version of the backbone"; Section VI-A: every weight and
+ * hidden dimension 1/rho of the backbone's):
+ *     x  = lambda_l u_l + (1 - lambda_l) a_{l-1};  n1 = LayerNorm(x);  q,k,v = n1 Wq, n1 Wk, n1 Wv
+ *     x' = x + concat_h(softmax(q_h k_h^T / sqrt(r/H)) v_h) Wo;  n2 = LayerNorm(x')
+ *     a_l = x' + relu(n2 W1 + c1) W2 + c2
+ * (pre-norm, bidirectional attention over the S tokens of a sample, LayerNorm eps 1e-5 with gain and
+ * bias, no dropout).  Classifier head only; it runs on the plain fp32 kernels. */
+typedef enum { PAC_BODY_POINTWISE = 0, PAC_BODY_TRANSFORMER = 1 } pac_body;
 
 typedef struct {
     int r;               /* adapter width (the paper's d / reduction factor) */
@@ -65,6 +76,9 @@ typedef struct {
     float lambda_init;   /* 0.5 in the paper */
     int max_batch;       /* largest B any later call will pass */
     const void* lm_head; /* device, [V][d] bf16, borrowed, frozen; NULL for the classifier head */
+    int body;            /* pac_body; 0 = point-wise */
+    int n_heads;         /* transformer body: attention heads H (r a multiple of H) */
+    int ffn_width;       /* transformer body: width f of the feed-forward layer (e.g. 4 r) */
 } pac_adapter_cfg;
 
 typedef struct { float lr, beta1, beta2, eps, weight_decay; } pac_adamw;
@@ -148,6 +162,8 @@ pac_status pac_cache_file_info(const char* path, int* dtype, long long* N, int* 
 /* Allocates parameters, gradients, AdamW moments and scratch for batches up to
  * cfg->max_batch and fills the parameters from `seed`:
  * W_down ~ N(0, 1/d), lambda = lambda_init, W_up = 0, W_head ~ N(0, 1/d), b_head = 0
+ * (transformer bodies: LayerNorm gains 1, all biases 0, Wq, Wk, Wv, Wo, W1 ~ N(0, 1/r), W2 ~ N(0, 1/f):
+ * the paper initialises them by pruning the backbone, whose weights are not part of this path)
  * (zero up-projection so the initial model equals backbone + head, the rationale of
  * Section IV-C).  Element i of the flat vector is a function of (seed, i) only.
  * For the classifier head this call also reads the last cached layer of every sample

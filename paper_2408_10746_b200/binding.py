@@ -39,7 +39,8 @@ class PacError(RuntimeError):
 
 class _AdapterCfg(C.Structure):
     _fields_ = [("r", C.c_int), ("act", C.c_int), ("head", C.c_int), ("n_out", C.c_int),
-                ("lambda_init", C.c_float), ("max_batch", C.c_int), ("lm_head", C.c_void_p)]
+                ("lambda_init", C.c_float), ("max_batch", C.c_int), ("lm_head", C.c_void_p),
+                ("body", C.c_int), ("n_heads", C.c_int), ("ffn_width", C.c_int)]
 
 
 class _AdamW(C.Structure):
@@ -200,8 +201,12 @@ class PacContext:
         self.cache_dtype = {PAC_F32: torch.float32, PAC_BF16: torch.bfloat16}[dt]
 
     def adapter_init(self, r: int, n_out: int, max_batch: int, act: int = PAC_ACT_RELU,
-                     head: int = PAC_HEAD_MEANPOOL_CLS, lambda_init: float = 0.5, lm_head=None, seed: int = 1):
-        cfg = _AdapterCfg(r, act, head, n_out, lambda_init, max_batch, lm_head.data_ptr() if lm_head is not None else None)
+                     head: int = PAC_HEAD_MEANPOOL_CLS, lambda_init: float = 0.5, lm_head=None, seed: int = 1,
+                     body: int = 0, n_heads: int = 0, ffn_width: int = 0):
+        """body = 1 (PAC_BODY_TRANSFORMER): every adapter is a width-r transformer layer with n_heads
+        attention heads and a feed-forward layer of ffn_width."""
+        cfg = _AdapterCfg(r, act, head, n_out, lambda_init, max_batch, lm_head.data_ptr() if lm_head is not None else None,
+                          body, n_heads, ffn_width)
         self._ck(self._lib.pac_adapter_init(self._h, C.byref(cfg), seed))
         if lm_head is not None:
             self._keep.append(lm_head)

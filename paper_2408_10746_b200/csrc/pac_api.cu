@@ -19,6 +19,7 @@
 #include "pac_chain_fwd.cuh"
 #include "pac_gemm.cuh"
 #include "pac_quant.cuh"
+#include "pac_tbody.cuh"
 
 using namespace pac;
 
@@ -58,6 +59,20 @@ struct Scratch {
     float* dw_part = nullptr;      // split partials of dW_down
     unsigned* gates = nullptr;     // [M][r] ReLU gates of all layers, one word per element (chain-in-epilogue forward)
     float* pool_part = nullptr;    // [B][s_chunks * 4][r] token sums of a_L per 32-token group (chain-in-epilogue forward)
+};
+
+// Saved activations and work buffers of the transformer-body adapters (fp32, sized for max_batch).
+struct TBody {
+    bool on = false;
+    int H = 0, f = 0;
+    BodyLayout bl{};
+    float* buf = nullptr;          // one allocation, carved below
+    // per layer stacks [L][...]
+    float *x = nullptr, *xhat1 = nullptr, *n1 = nullptr, *qkv = nullptr, *o = nullptr, *x1 = nullptr, *xhat2 = nullptr,
+          *n2 = nullptr, *pre = nullptr, *P = nullptr, *rstd1 = nullptr, *rstd2 = nullptr;
+    // work buffers of the backward pass
+    float *da = nullptr, *dx1 = nullptr, *dn = nullptr, *dqkv = nullptr, *dpre = nullptr, *dtmp = nullptr;
+    long long sMr = 0, sMf = 0, sP = 0, sM = 0;      // per-layer strides of the stacks
 };
 
 // A cache that lives in host memory (Section V-B, storage cost analysis: the cache is kept on
@@ -173,6 +188,7 @@ struct pac_ctx {
     int sms = 0;                   // multiprocessors of the device
     bool lm_ce_stream = false;     // LM cross-entropy as a register-resident stream over the logits (V <= 32768, V % 4 == 0)
     HostCache hc;                  // out-of-core mode (pac_cache_register_host)
+    TBody tb;                      // transformer-body adapters (plain fp32 kernels)
     // pac_train_step_async without copy nodes in the stream: a ring of id slots in page-locked host memory that
     // the forward kernel reads directly (two halves, an event per half orders the reuse)
     int* zc_ids = nullptr;         // [ZC_SLOTS][max_batch]
@@ -257,6 +273,18 @@ void fill_initial_params(const pac_ctx* c, unsigned long long seed, std::vector<
     for (long long i = 0; i < lay.lam; ++i) out[i] = unit_normal(key, (unsigned long long)i) * inv;
     for (long long i = lay.lam; i < lay.w_up; ++i) out[i] = c->cfg.lambda_init;
     for (long long i = lay.w_head; i < lay.b_head; ++i) out[i] = unit_normal(key, (unsigned long long)i) * inv;
+    if (c->tb.on) {
+        // transformer bodies: LayerNorm gains 1, biases 0, Gaussian matrices scaled by 1/sqrt(fan-in)
+        const BodyLayout& bl = c->tb.bl;
+        const float ir = (float)(1.0 / std::sqrt((double)bl.r)), jf = (float)(1.0 / std::sqrt((double)bl.f));
+        for (int l = 0; l < c->dm.L; ++l) {
+            const long long o = lay.body + (long long)l * bl.per_layer;
+            for (int j = 0; j < bl.r; ++j) { out[o + bl.g1 + j] = 1.f; out[o + bl.g2 + j] = 1.f; }
+            for (long long i = o + bl.wq; i < o + bl.g2; ++i) out[i] = unit_normal(key, (unsigned long long)i) * ir;
+            for (long long i = o + bl.w1; i < o + bl.c1; ++i) out[i] = unit_normal(key, (unsigned long long)i) * ir;
+            for (long long i = o + bl.w2; i < o + bl.c2; ++i) out[i] = unit_normal(key, (unsigned long long)i) * jf;
+        }
+    }
 }
 
 // ---- optional event brackets around the two cache-stream kernels ----
@@ -507,6 +535,132 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
     return dw_down(c, d_ids, B, true);
 }
 
+// ---------------------------------------------------------------------------
+// Transformer-body adapters (plain fp32 kernels; see pac_tbody.cuh).  ids are on the device.
+// ---------------------------------------------------------------------------
+template <class AF, class BF, class EF>
+pac_status tb_gemm(pac_ctx* c, int M, int N, int K, int Z, const AF& A, const BF& Bm, const EF& E) {
+    dim3 grid(cdiv(N, SG_BN), cdiv(M, SG_BM), (unsigned)Z);
+    gemm_simt<<<grid, 256, 0, c->stream>>>(M, N, K, A, Bm, E);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+#define TB_OK(call) do { pac_status s_ = (call); if (s_ != PAC_OK) return s_; } while (0)
+
+pac_status tb_forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
+    const Dims& dm = c->dm;
+    TBody& t = c->tb;
+    const BodyLayout& bl = t.bl;
+    Scratch& sc = c->sc;
+    const int M = B * dm.S, r = dm.r, f = t.f;
+    const long long n = (long long)M * r, stride = (long long)c->max_rows * r;
+    cudaStream_t st = c->stream;
+    TB_OK(down_projection(c, d_ids, B));
+    const float* lam = c->params + c->lay.lam;
+    const unsigned rows_grid = cdiv(M, 8), heads_grid = cdiv((long long)B * t.H * dm.S, 128);
+    for (int l = 0; l < dm.L; ++l) {
+        const float* w = c->params + c->lay.body + (long long)l * bl.per_layer;
+        float *x = t.x + l * t.sMr, *xhat1 = t.xhat1 + l * t.sMr, *n1 = t.n1 + l * t.sMr, *qkv = t.qkv + 3 * l * t.sMr,
+              *o = t.o + l * t.sMr, *x1 = t.x1 + l * t.sMr, *xhat2 = t.xhat2 + l * t.sMr, *n2 = t.n2 + l * t.sMr,
+              *pre = t.pre + l * t.sMf, *P = t.P + l * t.sP, *a = sc.a + l * stride;
+        tb_merge_kernel<<<cdiv(n, 256), 256, 0, st>>>(sc.u + l * stride, l ? sc.a + (l - 1) * stride : nullptr, lam, l, n, x);
+        LAUNCH_CHECK(c);
+        tb_layernorm_fwd_kernel<<<rows_grid, 256, 0, st>>>(x, w + bl.g1, w + bl.b1, M, r, n1, xhat1, t.rstd1 + l * t.sM);
+        LAUNCH_CHECK(c);
+        // q | k | v = n1 [Wq | Wk | Wv]  (three products in one launch: the weights are consecutive in the layout)
+        TB_OK(tb_gemm(c, M, r, r, 3, MatA_RowMajor{{n1, 0, r}}, MatB_RowMajor{{w + bl.wq, (long long)r * r, r}},
+                      StoreRowMajor{qkv, t.sMr, r}));
+        tb_attn_fwd_kernel<<<heads_grid, 128, 0, st>>>(qkv, qkv + t.sMr, qkv + 2 * t.sMr, B, dm.S, r, t.H, P, o);
+        LAUNCH_CHECK(c);
+        TB_OK(tb_gemm(c, M, r, r, 1, MatA_RowMajor{{o, 0, r}}, MatB_RowMajor{{w + bl.wo, 0, r}}, StoreAddBias{x1, x, nullptr, r}));
+        tb_layernorm_fwd_kernel<<<rows_grid, 256, 0, st>>>(x1, w + bl.g2, w + bl.b2, M, r, n2, xhat2, t.rstd2 + l * t.sM);
+        LAUNCH_CHECK(c);
+        TB_OK(tb_gemm(c, M, f, r, 1, MatA_RowMajor{{n2, 0, r}}, MatB_RowMajor{{w + bl.w1, 0, f}}, StoreAddBias{pre, nullptr, w + bl.c1, f}));
+        TB_OK(tb_gemm(c, M, r, f, 1, MatA_ReluRowMajor{pre, f}, MatB_RowMajor{{w + bl.w2, 0, r}}, StoreAddBias{a, x1, w + bl.c2, r}));
+    }
+    // head: the same kernels as the point-wise plain path
+    const float* aL = sc.a + (long long)(dm.L - 1) * stride;
+    pool_tokens_kernel<<<B, 128, 0, st>>>(aL, sc.pooled_a, dm.S, r);
+    LAUNCH_CHECK(c);
+    const size_t smem = sizeof(float) * (dm.d + dm.C + 32);
+    cls_head_kernel<<<B, 256, smem, st>>>(sc.hbar, d_ids, dm.N, c->labels, sc.pooled_a, c->params + c->lay.w_up,
+                                          c->params + c->lay.w_head, c->params + c->lay.b_head, B, dm.S, dm.d, r, dm.C,
+                                          train ? 1 : 0, sc.pooled_y, train ? sc.logits : d_logits_out, sc.loss_b, sc.dlogits,
+                                          sc.gvec, sc.daL, c->status);
+    LAUNCH_CHECK(c);
+    return PAC_OK;
+}
+
+pac_status tb_backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
+    const Dims& dm = c->dm;
+    TBody& t = c->tb;
+    const BodyLayout& bl = t.bl;
+    Scratch& sc = c->sc;
+    const int M = B * dm.S, r = dm.r, f = t.f;
+    const long long n = (long long)M * r, stride = (long long)c->max_rows * r;
+    cudaStream_t st = c->stream;
+    {
+        const long long ne = (long long)r * dm.d + (long long)dm.d * dm.C + dm.C + 1;
+        cls_grads_kernel<<<cdiv(ne, 256), 256, 0, st>>>(sc.pooled_a, sc.gvec, sc.pooled_y, sc.dlogits, sc.loss_b, B, dm.d, r, dm.C,
+                                                        c->grads + c->lay.w_up, c->grads + c->lay.w_head, c->grads + c->lay.b_head, d_loss);
+        LAUNCH_CHECK(c);
+    }
+    tb_expand_kernel<<<cdiv(n, 256), 256, 0, st>>>(sc.daL, dm.S, r, n, t.da);
+    LAUNCH_CHECK(c);
+    const float* lam = c->params + c->lay.lam;
+    const unsigned rows_grid = cdiv(M, 8), heads_grid = cdiv((long long)B * t.H * dm.S, 128);
+    for (int l = dm.L - 1; l >= 0; --l) {
+        const float* w = c->params + c->lay.body + (long long)l * bl.per_layer;
+        float* g = c->grads + c->lay.body + (long long)l * bl.per_layer;
+        float *xhat1 = t.xhat1 + l * t.sMr, *n1 = t.n1 + l * t.sMr, *qkv = t.qkv + 3 * l * t.sMr, *o = t.o + l * t.sMr,
+              *xhat2 = t.xhat2 + l * t.sMr, *n2 = t.n2 + l * t.sMr, *pre = t.pre + l * t.sMf, *P = t.P + l * t.sP;
+        float *da = t.da, *dx1 = t.dx1, *dn = t.dn, *dqkv = t.dqkv, *dpre = t.dpre, *dtmp = t.dtmp;
+        // a = x1 + relu(pre) W2 + c2
+        tb_colsum_kernel<<<cdiv(r, 128), 128, 0, st>>>(da, nullptr, M, r, g + bl.c2);
+        LAUNCH_CHECK(c);
+        TB_OK(tb_gemm(c, f, r, M, 1, MatA_ReluColMajor{pre, f}, MatB_RowMajor{{da, 0, r}}, StoreRowMajor{g + bl.w2, 0, r}));
+        TB_OK(tb_gemm(c, M, f, r, 1, MatA_RowMajor{{da, 0, r}}, MatB_ColMajor{{w + bl.w2, 0, r}}, StoreMaskedByPositive{dpre, pre, f}));
+        tb_colsum_kernel<<<cdiv(f, 128), 128, 0, st>>>(dpre, nullptr, M, f, g + bl.c1);
+        LAUNCH_CHECK(c);
+        TB_OK(tb_gemm(c, r, f, M, 1, MatA_ColMajor{{n2, 0, r}}, MatB_RowMajor{{dpre, 0, f}}, StoreRowMajor{g + bl.w1, 0, f}));
+        TB_OK(tb_gemm(c, M, r, f, 1, MatA_RowMajor{{dpre, 0, f}}, MatB_ColMajor{{w + bl.w1, 0, f}}, StoreRowMajor{dn, 0, r}));     // dn2
+        tb_colsum_kernel<<<cdiv(r, 128), 128, 0, st>>>(dn, xhat2, M, r, g + bl.g2);
+        LAUNCH_CHECK(c);
+        tb_colsum_kernel<<<cdiv(r, 128), 128, 0, st>>>(dn, nullptr, M, r, g + bl.b2);
+        LAUNCH_CHECK(c);
+        tb_layernorm_bwd_kernel<<<rows_grid, 256, 0, st>>>(dn, xhat2, t.rstd2 + l * t.sM, w + bl.g2, da, M, r, dx1);             // dx1 = da + LN2 backward
+        LAUNCH_CHECK(c);
+        // x1 = x + o Wo
+        TB_OK(tb_gemm(c, r, r, M, 1, MatA_ColMajor{{o, 0, r}}, MatB_RowMajor{{dx1, 0, r}}, StoreRowMajor{g + bl.wo, 0, r}));
+        TB_OK(tb_gemm(c, M, r, r, 1, MatA_RowMajor{{dx1, 0, r}}, MatB_ColMajor{{w + bl.wo, 0, r}}, StoreRowMajor{dtmp, 0, r}));   // do
+        float *dq = dqkv, *dk = dqkv + t.sMr, *dv = dqkv + 2 * t.sMr;
+        tb_attn_bwd_dv_kernel<<<heads_grid, 128, 0, st>>>(P, dtmp, B, dm.S, r, t.H, dv);
+        LAUNCH_CHECK(c);
+        tb_attn_bwd_dq_kernel<<<heads_grid, 128, 0, st>>>(P, dtmp, qkv + t.sMr, qkv + 2 * t.sMr, B, dm.S, r, t.H, dq);
+        LAUNCH_CHECK(c);
+        tb_attn_bwd_dk_kernel<<<heads_grid, 128, 0, st>>>(P, qkv, B, dm.S, r, t.H, dk);
+        LAUNCH_CHECK(c);
+        // dWq | dWk | dWv = n1^T [dq | dk | dv]
+        TB_OK(tb_gemm(c, r, r, M, 3, MatA_ColMajor{{n1, 0, r}}, MatB_RowMajor{{dqkv, t.sMr, r}}, StoreRowMajor{g + bl.wq, (long long)r * r, r}));
+        // dn1 = dq Wq^T + dk Wk^T + dv Wv^T
+        TB_OK(tb_gemm(c, M, r, r, 1, MatA_RowMajor{{dq, 0, r}}, MatB_ColMajor{{w + bl.wq, 0, r}}, StoreRowMajor{dn, 0, r}));
+        TB_OK(tb_gemm(c, M, r, r, 1, MatA_RowMajor{{dk, 0, r}}, MatB_ColMajor{{w + bl.wk, 0, r}}, StoreAccumulate{dn, r}));
+        TB_OK(tb_gemm(c, M, r, r, 1, MatA_RowMajor{{dv, 0, r}}, MatB_ColMajor{{w + bl.wv, 0, r}}, StoreAccumulate{dn, r}));
+        tb_colsum_kernel<<<cdiv(r, 128), 128, 0, st>>>(dn, xhat1, M, r, g + bl.g1);
+        LAUNCH_CHECK(c);
+        tb_colsum_kernel<<<cdiv(r, 128), 128, 0, st>>>(dn, nullptr, M, r, g + bl.b1);
+        LAUNCH_CHECK(c);
+        tb_layernorm_bwd_kernel<<<rows_grid, 256, 0, st>>>(dn, xhat1, t.rstd1 + l * t.sM, w + bl.g1, dx1, M, r, dtmp);           // dx = dx1 + LN1 backward
+        LAUNCH_CHECK(c);
+        // x = lambda u + (1 - lambda) a_prev
+        tb_unmerge_kernel<<<1, 1024, 0, st>>>(dtmp, sc.u + l * stride, l ? sc.a + (l - 1) * stride : nullptr, lam, l, n,
+                                              sc.du + l * stride, da, c->grads + c->lay.lam);
+        LAUNCH_CHECK(c);
+    }
+    return dw_down(c, d_ids, B, true);
+}
+#undef TB_OK
+
 bool use_fused_cls(const pac_ctx* c) { return c->cfg.head == PAC_HEAD_MEANPOOL_CLS && c->mplan.ok; }
 // The one-launch forward pays off when all of the batch's clusters run at the same time (its GEMM
 // and chain phases do not overlap across waves); larger batches keep the two separate kernels.
@@ -700,6 +854,11 @@ pac_status finalize_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, 
 // One whole train step; with hp != NULL the AdamW update is fused into the last kernel.
 pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, const pac_adamw* hp) {
     pac_status st;
+    if (c->tb.on) {
+        if ((st = tb_forward(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
+        if ((st = tb_backward(c, d_ids, B, d_loss)) != PAC_OK) return st;
+        return hp ? adam_enqueue(c, hp) : PAC_OK;
+    }
     if (use_fused_cls(c)) {
         if ((st = cls_forward_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
         if (c->step_host_ids) d_ids = c->sc.ids;          // the forward kernel left a device copy for the later kernels
@@ -747,7 +906,7 @@ void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
-                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, c->params, c->grads,
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, c->tb.buf, c->params, c->grads,
                     c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -904,9 +1063,17 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     if (!cls && !cfg->lm_head) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: LM head pointer is NULL");
     if (cls && cfg->n_out > 4096) return fail(c, PAC_ERR_UNSUPPORTED, "pac_adapter_init: classifier head supports up to 4096 classes");
     if ((long long)cfg->max_batch * c->dm.S > 0x7fffffffLL / 8) return fail(c, PAC_ERR_UNSUPPORTED, "pac_adapter_init: max_batch*S too large");
+    if (cfg->body != PAC_BODY_POINTWISE && cfg->body != PAC_BODY_TRANSFORMER) return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: bad body");
+    if (cfg->body == PAC_BODY_TRANSFORMER) {
+        if (!cls) return fail(c, PAC_ERR_UNSUPPORTED, "pac_adapter_init: transformer-body adapters need the classifier head");
+        if (cfg->n_heads < 1 || cfg->r % cfg->n_heads != 0 || cfg->ffn_width < 1)
+            return fail(c, PAC_ERR_INVALID_ARG, "pac_adapter_init: transformer body needs n_heads dividing r and a positive ffn_width");
+        if (c->hc.on) return fail(c, PAC_ERR_UNSUPPORTED, "pac_adapter_init: transformer-body adapters need a device-resident cache");
+    }
     CU_OK(c, cudaSetDevice(c->device));
     c->cfg = *cfg;
     c->dm.r = cfg->r; c->dm.C = cfg->n_out;
+    c->tb.on = cfg->body == PAC_BODY_TRANSFORMER;
     if (c->hc.on) {
         // the kernels see a staging slot: a cache of max_batch samples
         HostCache& h = c->hc;
@@ -930,10 +1097,16 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     }
     const Dims& dm = c->dm;
     c->lay = ParamLayout::make(dm.L, dm.d, dm.r, dm.C, cls);
+    if (c->tb.on) {
+        c->tb.H = cfg->n_heads; c->tb.f = cfg->ffn_width;
+        c->tb.bl = BodyLayout::make(dm.r, cfg->ffn_width);
+        c->lay.body_per = c->tb.bl.per_layer; c->lay.br = dm.r; c->lay.bf = cfg->ffn_width;
+        c->lay.total = c->lay.body + (long long)dm.L * c->tb.bl.per_layer;
+    }
     c->max_rows = cfg->max_batch * dm.S;
     const long long Mr = (long long)c->max_rows * dm.r;
     c->chain_blocks_max = (int)cdiv(Mr, 256);
-    c->mplan = cls ? mid_plan(dm) : MidPlan{};
+    c->mplan = (cls && !c->tb.on) ? mid_plan(dm) : MidPlan{};
     if (c->mplan.ok && cfg->max_batch * 8 > c->chain_blocks_max) c->chain_blocks_max = cfg->max_batch * 8;     // clusters of up to 8
     FusedFwdPlan fwd_plan{};
     if (c->mplan.ok && c->dtype == PAC_BF16 && tensor_shape_supported(dm) && !c->force_simt && c->forward_mode != 2) {
@@ -1008,7 +1181,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
     }
     // tensor-core path: bf16 cache with TMA/UMMA-compatible sizes
     c->tensor_ok = false;
-    if (st == PAC_OK && c->dtype == PAC_BF16 && tensor_shape_supported(dm)) {
+    if (st == PAC_OK && c->dtype == PAC_BF16 && tensor_shape_supported(dm) && !c->tb.on) {
         A(dmalloc(c, &s.wdT, (long long)dm.L * 2 * dm.r * dm.d));
         A(dmalloc(c, &s.du16, Mr * dm.L));
         long long part_floats = 0;
@@ -1043,6 +1216,23 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
         }
     }
     if (st == PAC_OK && !use_tensor(c)) A(dmalloc(c, &s.du, Mr * dm.L));    // the plain path keeps du in fp32
+    if (st == PAC_OK && c->tb.on) {
+        TBody& t = c->tb;
+        const long long Mx = c->max_rows;
+        t.sMr = Mx * dm.r; t.sMf = Mx * t.f; t.sP = (long long)cfg->max_batch * t.H * dm.S * dm.S; t.sM = Mx;
+        const long long per_layer = 10 * t.sMr + t.sMf + t.sP + 2 * t.sM;     // x xhat1 n1 qkv(3) o x1 xhat2 n2 | pre | P | rstd1 rstd2
+        const long long work = 7 * t.sMr + t.sMf;                             // da dx1 dn dqkv(3) dtmp | dpre
+        A(dmalloc(c, &t.buf, per_layer * dm.L + work));
+        if (st == PAC_OK) {
+            float* q = t.buf;
+            auto take = [&](long long k) { float* r_ = q; q += k; return r_; };
+            t.x = take(t.sMr * dm.L); t.xhat1 = take(t.sMr * dm.L); t.n1 = take(t.sMr * dm.L); t.qkv = take(3 * t.sMr * dm.L);
+            t.o = take(t.sMr * dm.L); t.x1 = take(t.sMr * dm.L); t.xhat2 = take(t.sMr * dm.L); t.n2 = take(t.sMr * dm.L);
+            t.pre = take(t.sMf * dm.L); t.P = take(t.sP * dm.L); t.rstd1 = take(t.sM * dm.L); t.rstd2 = take(t.sM * dm.L);
+            t.da = take(t.sMr); t.dx1 = take(t.sMr); t.dn = take(t.sMr); t.dqkv = take(3 * t.sMr); t.dtmp = take(t.sMr);
+            t.dpre = take(t.sMf);
+        }
+    }
     if (st != PAC_OK) return st;
     CU_OK(c, cudaMemsetAsync(s.u, 0, sizeof(float) * Mr * dm.L, c->stream));
     CU_OK(c, cudaMemsetAsync(s.a, 0, sizeof(float) * Mr * dm.L, c->stream));
@@ -1224,7 +1414,8 @@ pac_status pac_eval_logits(pac_ctx* c, const int* sample_ids, int B, float* dev_
     const int* d_ids = nullptr;
     pac_status st = prepare_ids(c, sample_ids, B, "pac_eval_logits", &d_ids);
     if (st != PAC_OK) return st;
-    st = use_fused_cls(c) ? cls_forward_enqueue(c, d_ids, B, false, dev_out) : forward(c, d_ids, B, false, dev_out);
+    st = c->tb.on ? tb_forward(c, d_ids, B, false, dev_out)
+       : use_fused_cls(c) ? cls_forward_enqueue(c, d_ids, B, false, dev_out) : forward(c, d_ids, B, false, dev_out);
     if (st != PAC_OK) return st;
     return finish_ids(c);
 }

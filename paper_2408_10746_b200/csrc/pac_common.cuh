@@ -62,8 +62,12 @@ struct Dims {
 
 // Offsets of the flat fp32 parameter vector:
 // W_down[L][d][r] | lambda[L] | W_up[r][d] | W_head[d][C] | b_head[C]
+// With transformer-body adapters the per-layer body blocks follow, layer after layer:
+// ... | body[0] | body[1] | ... | body[L-1],  body[l] = g1 | b1 | Wq | Wk | Wv | Wo | g2 | b2 | W1 | c1 | W2 | c2
 struct ParamLayout {
     long long w_down, lam, w_up, w_head, b_head, total;
+    long long body, body_per;        // first body block and floats per block (body_per == 0: point-wise adapters)
+    int br, bf;                      // adapter width and FFN width of the body blocks
     __host__ __device__ static ParamLayout make(int L, int d, int r, int C, bool cls) {
         ParamLayout p;
         p.w_down = 0;
@@ -72,7 +76,16 @@ struct ParamLayout {
         p.w_head = p.w_up + (long long)r * d;
         p.b_head = p.w_head + (cls ? (long long)d * C : 0);
         p.total = p.b_head + (cls ? C : 0);
+        p.body = p.total; p.body_per = 0; p.br = r; p.bf = 0;
         return p;
+    }
+    // decoupled weight decay: the weight matrices, not lambda, biases or LayerNorm parameters
+    __host__ __device__ bool decays(long long i) const {
+        if (i < lam) return true;
+        if (i < body) return i >= w_up && i < b_head;
+        const long long off = (i - body) % body_per, rr = (long long)br * br, rf = (long long)br * bf;
+        const long long wq = 2LL * br, g2 = wq + 4 * rr, w1 = g2 + 2LL * br, c1 = w1 + rf, w2 = c1 + bf, c2 = w2 + rf;
+        return (off >= wq && off < g2) || (off >= w1 && off < c1) || (off >= w2 && off < c2);
     }
 };
 

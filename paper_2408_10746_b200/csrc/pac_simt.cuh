@@ -478,7 +478,7 @@ __device__ __forceinline__ float adamw_math(float th, float& mi, float& vi, floa
 __device__ __forceinline__ void adamw_element(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
                                               long long i, float gi, const ParamLayout& lay, const pac_adamw& hp,
                                               float bc1, float bc2, bf16* __restrict__ wdT, int d, int r) {
-    const bool decays = (i < lay.lam) || (i >= lay.w_up && i < lay.b_head);
+    const bool decays = lay.decays(i);
     float mi = m[i], vi = v[i];
     const float th = adamw_math(p[i], mi, vi, gi, decays, hp, bc1, bc2);
     m[i] = mi;
