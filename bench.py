@@ -190,28 +190,34 @@ def run_reference(args, spec):
 
 def run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world):
     """N > 1 with a real exchange step: every rank trains on its own cache shard and local
-    minibatch of B samples, gradients are averaged with one NCCL all-reduce per step (global
-    minibatch world*B), then every rank applies the same AdamW step."""
+    minibatch of B samples; the gradient buffers are summed with one NCCL all-reduce per step
+    (enqueued behind the step, no host wait), the optimizer kernel applies 1/world, and the losses
+    of the timed region are reduced and read once at its end (global minibatch world*B)."""
     import torch
     import paper_2408_10746_b200 as pac
     from paper_2408_10746_b200.data_parallel import DataParallel, PacLocalTrainer
     K, W, B = args.steps, args.warmup, spec.B
     hp = pac.AdamW()
+    dp = DataParallel(PacLocalTrainer(ctx, stream), loss_slots=max(K, W) + 8)
+    for i in range(W):
+        dp.train_step(ids_host[(i % K) * B:(i % K + 1) * B]); dp.adam_step(hp)
+    dp.epoch_losses()
+    sampler = ClockSampler(torch.cuda.current_device())
+    l0 = ctx.launch_count()
+    dist.barrier(); torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
-        dp = DataParallel(PacLocalTrainer(ctx))
-        for i in range(W):
-            dp.train_step(ids_host[(i % K) * B:(i % K + 1) * B]); dp.adam_step(hp)
-        sampler = ClockSampler(torch.cuda.current_device())
-        l0 = ctx.launch_count()
-        dist.barrier(); torch.cuda.synchronize()
-        sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for i in range(K):
-            dp.train_step(ids_host[i * B:(i + 1) * B]); dp.adam_step(hp)
+    for i in range(K):
+        dp.train_step(ids_host[i * B:(i + 1) * B]); dp.adam_step(hp)
+    with torch.cuda.stream(stream):
         e1.record(stream)
-        dist.barrier(); torch.cuda.synchronize()
+    dist.barrier(); torch.cuda.synchronize()
     clocks = sampler.finish()
+    losses = dp.epoch_losses()
+    if not np.isfinite(losses).all():
+        raise SystemExit("non-finite loss in the timed region")
     t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms = float(t.item())
@@ -220,9 +226,10 @@ def run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world)
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if spec.dtype == "bf16" else "f32",
            "data": "synthetic",
            "config": {"workload": workload_name(spec), "kernel_path": ctx.kernel_path(), "parallelism": f"dp{world}",
-                      "global_batch": world * B, "collective": "NCCL all-reduce of the flat fp32 adapter gradient per step"},
-           "clocks": clocks, "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 4 * B, "d2h_bytes_per_step": 4, "steps": K},
-           "gpu_launches": int(ctx.launch_count() - l0), "roofline": None, "cpu_baseline": None}
+                      "global_batch": world * B, "comm": dp.comm + "; no host wait per step, losses reduced once per region"},
+           "clocks": clocks, "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 4 * B, "d2h_bytes_per_step": 0, "steps": K,
+                                     "note": "host ids in every step; losses read once at the end of the region"},
+           "gpu_launches": int(ctx.launch_count() - l0), "roofline": None, "cpu_baseline": None, "final_loss": float(losses[-1])}
     ctx.close()
     dist.barrier()
     dist.destroy_process_group()
@@ -434,9 +441,14 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
     torch.cuda.set_device(local)
     dist = None
-    if world > 1:
+    if world > 1 or args.parallelism == "dp":
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if world == 1:                       # a one-rank group: the data-parallel path itself, without an exchange partner
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29531")
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # the cache must fit: keep 8 GB of headroom, halve N otherwise (and say so)
     note = []
@@ -472,7 +484,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    if world > 1 and args.parallelism == "dp":
+    if args.parallelism == "dp":
         return run_data_parallel(args, spec, ctx, dist, stream, ids_host, dev, rank, world)
 
     # ---------------- device-resident timing (value) ----------------

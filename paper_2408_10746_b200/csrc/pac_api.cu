@@ -53,6 +53,9 @@ struct Scratch {
     float* dy = nullptr;           // [M][d]
     bf16* y16 = nullptr;           // [M][d] bf16 y (tensor-core LM head)
     bf16* dlog16 = nullptr;        // [M][V] bf16 dlogits (tensor-core LM head)
+    bf16* aL16 = nullptr;          // [M][r] bf16 a_L, bf16 W_up [r][d], bf16 dy [M][d]: operands of the LM path's skinny products
+    bf16* wup16 = nullptr;
+    bf16* dy16 = nullptr;
     // tensor path
     bf16* wdT = nullptr;           // [L][2][d][r] bf16 hi/lo shadow of W_down
     float* lm_part = nullptr;      // [slices][...] partial sums of the LM path's two skinny products (dW_up, da_L)
@@ -184,7 +187,9 @@ struct pac_ctx {
     int forward_mode = 0;          // 0: automatic, 2: down-projections and head phase as two plain launches, 3: one-launch
                                    // forward whenever the shape allows, 4: chain-in-epilogue forward whenever the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
+    GemmPlan g_y{}, g_daL{};       // y = a_L W_up (+ h_L in the epilogue) and da_L = dy W_up^T on the tensor cores
     bool lm_tensor = false;
+    bool lm_skinny_tensor = false; // the three products around W_up also run on the tensor cores
     int sms = 0;                   // multiprocessors of the device
     bool lm_ce_stream = false;     // LM cross-entropy as a register-resident stream over the logits (V <= 32768, V % 4 == 0)
     HostCache hc;                  // out-of-core mode (pac_cache_register_host)
@@ -384,7 +389,19 @@ pac_status forward(pac_ctx* c, const int* d_ids, int B, bool train, float* d_log
         dim3 g1(cdiv(dm.d, SG_BN), cdiv(M, SG_BM), 1);
         MatA_RowMajor Aa{{aL, 0, dm.r}};
         MatB_RowMajor Bu{{W_up, 0, dm.d}};
-        if (c->lm_tensor) {
+        if (c->lm_tensor && c->lm_skinny_tensor) {
+            // bf16 copies of a_L and W_up, then y16 = bf16(a_L W_up + h_L) in one tensor-core GEMM whose epilogue adds
+            // the last cached layer's rows (y enters the LM head rounded to bf16 anyway)
+            to_bf16_kernel<<<cdiv((long long)M * dm.r / 4, 256), 256, 0, c->stream>>>(aL, (long long)M * dm.r, sc.aL16, ((uintptr_t)aL & 15) == 0);
+            LAUNCH_CHECK(c);
+            to_bf16_kernel<<<cdiv((long long)dm.r * dm.d / 4, 256), 256, 0, c->stream>>>(W_up, (long long)dm.r * dm.d, sc.wup16, ((uintptr_t)W_up & 15) == 0);
+            LAUNCH_CHECK(c);
+            GemmExtras ex;
+            ex.C16 = sc.y16; ex.ldc16 = dm.d;
+            ex.add_cache = (const bf16*)c->cache; ex.ids = d_ids; ex.n_cache = dm.N; ex.L = dm.L; ex.S = dm.S;
+            st = gemm_launch(c->g_y, c->stream, M, nullptr, 0, c->status, &c->launches, &ex);
+            if (st != PAC_OK) return fail(c, st, "tensor-core y GEMM launch failed: %s", tensor_last_error());
+        } else if (c->lm_tensor) {
             StorePlusLastLayerBf16<bf16> E{sc.y16, dm.d, CacheRows<bf16>{(const bf16*)c->cache, d_ids, dm.N, dm.L, dm.S, dm.d, dm.L - 1}};
             gemm_simt<<<g1, 256, 0, c->stream>>>(M, dm.d, dm.r, Aa, Bu, E);
         } else if (c->dtype == PAC_F32) {
@@ -460,7 +477,9 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
         // dy = dlogits W_lm   (the head is frozen: it receives no gradient)
         if (c->lm_tensor) {
             time_mark(c, 3, false);
-            pac_status gs = gemm_launch(c->g_dy, c->stream, M, sc.dy, dm.d, c->status, &c->launches);
+            GemmExtras ex;
+            if (c->lm_skinny_tensor) { ex.C16 = sc.dy16; ex.ldc16 = dm.d; }        // bf16 copy for the two products below
+            pac_status gs = gemm_launch(c->g_dy, c->stream, M, sc.dy, dm.d, c->status, &c->launches, c->lm_skinny_tensor ? &ex : nullptr);
             time_mark(c, 3, true);
             if (gs != PAC_OK) return fail(c, gs, "tensor-core dy GEMM launch failed: %s", tensor_last_error());
         } else {
@@ -497,7 +516,13 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
             gemm_simt<<<g2, 256, 0, c->stream>>>(dm.r, dm.d, M, At, Bd, Eu);
         }
         LAUNCH_CHECK(c);
-        // da_L = dy W_up^T
+        // da_L = dy W_up^T: on the tensor cores when the bf16 copy of dy exists (da_L only feeds du, which is
+        // rounded to bf16 anyway).  dW_up above stays in fp32 FMA: with a_L and dy rounded to bf16 its error,
+        // amplified by Adam, took the parameters after ten steps past the 1e-2 bound (1.1e-2 measured).
+        if (c->lm_tensor && c->lm_skinny_tensor) {
+            pac_status gs = gemm_launch(c->g_daL, c->stream, M, sc.daL, dm.r, c->status, &c->launches);
+            if (gs != PAC_OK) return fail(c, gs, "tensor-core da_L GEMM launch failed: %s", tensor_last_error());
+        } else {
         dim3 g3(cdiv(dm.r, SG_BN), cdiv(M, SG_BM), 1);
         MatA_RowMajor Ady{{sc.dy, 0, dm.d}};
         MatB_ColMajor But{{W_up, 0, dm.d}};
@@ -515,6 +540,7 @@ pac_status backward(pac_ctx* c, const int* d_ids, int B, float* d_loss) {
             gemm_simt<<<g3, 256, 0, c->stream>>>(M, dm.r, dm.d, Ady, But, Ea);
         }
         LAUNCH_CHECK(c);
+        }
         per_sample = 0;
     }
     const float* lam = c->params + c->lay.lam;
@@ -906,7 +932,7 @@ void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
-                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, c->tb.buf, c->params, c->grads,
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.aL16, s.wup16, s.dy16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, c->tb.buf, c->params, c->grads,
                     c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
@@ -1213,6 +1239,17 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             } else if (ts != PAC_ERR_UNSUPPORTED) {
                 st = fail(c, ts, "tensor path set-up failed: %s", tensor_last_error());
             }
+        }
+    }
+    c->lm_skinny_tensor = false;
+    if (st == PAC_OK && c->lm_tensor && c->tensor_ok && dm.r % 8 == 0 && dm.r <= 256 && (Mr % 4 == 0) && ((long long)dm.r * dm.d) % 4 == 0) {
+        A(dmalloc(c, &s.aL16, Mr)); A(dmalloc(c, &s.wup16, (long long)dm.r * dm.d)); A(dmalloc(c, &s.dy16, (long long)c->max_rows * dm.d));
+        if (st == PAC_OK) {
+            CU_OK(c, cudaMemsetAsync(s.aL16, 0, sizeof(bf16) * Mr, c->stream));
+            CU_OK(c, cudaMemsetAsync(s.dy16, 0, sizeof(bf16) * (size_t)c->max_rows * dm.d, c->stream));
+            pac_status g1 = gemm_plan_create(c->g_y, c->device, s.aL16, c->max_rows, s.wup16, dm.d, dm.r, 1);
+            pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_daL, c->device, s.dy16, c->max_rows, s.wup16, dm.r, dm.d, 0) : g1;
+            c->lm_skinny_tensor = g1 == PAC_OK && g2 == PAC_OK;
         }
     }
     if (st == PAC_OK && !use_tensor(c)) A(dmalloc(c, &s.du, Mr * dm.L));    // the plain path keeps du in fp32

@@ -19,7 +19,11 @@ struct GemmParams {
     int M, N, K;
     int m_tiles, n_tiles, k_chunks;
     int b_mn_major;            // 0: B stored [N][K] (K contiguous); 1: B stored [K][N] (N contiguous)
-    float* C; long long ldc;
+    float* C; long long ldc;   // fp32 output (may be null when only the bf16 output is wanted)
+    bf16* C16; long long ldc16; // optional second output: the same values rounded to bf16
+    // optional: add the last cached layer's row to every output row before storing, so that
+    // y = h_L + a_L W_up (Section IV-A) leaves the GEMM ready for the LM head; N == d then
+    const bf16* add_cache; const int* ids; long long n_cache; int L, S;
     unsigned* status;
 };
 
@@ -123,21 +127,65 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!mbar_wait_warp(accf0 + 8 * buf, aph, abort_flag, p.status)) break;
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
-            float* dst = p.C + (long long)row * p.ldc + n0;
+            float* dst = p.C ? p.C + (long long)row * p.ldc + n0 : nullptr;
+            bf16* dst16 = p.C16 ? p.C16 + (long long)row * p.ldc16 + n0 : nullptr;
+            const bf16* hrow = nullptr;
+            if (p.add_cache && row < p.M) {
+                const int b = row / p.S, sidx = row - b * p.S;
+                const long long id = safe_id(p.ids, b, p.n_cache, nullptr);
+                hrow = p.add_cache + (((id * p.L) + (p.L - 1)) * p.S + sidx) * (long long)p.N + n0;
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * GT_BN);
-            const bool vec_ok = (p.ldc & 3) == 0;
+            const bool vec_ok = (p.ldc & 3) == 0, vec16_ok = (p.ldc16 & 7) == 0 && (p.N & 7) == 0;
             for (int c0 = 0; c0 < GT_BN; c0 += 32) {
                 float v[32];
                 tmem_ld32(taddr + c0, v);
                 tmem_ld_wait();
                 if (row < p.M) {
-                    if (vec_ok && n0 + c0 + 32 <= p.N) {
+                    const bool full = n0 + c0 + 32 <= p.N;
+                    if (hrow) {
+                        if (full && vec16_ok) {
 #pragma unroll
-                        for (int c = 0; c < 32; c += 4) *reinterpret_cast<float4*>(dst + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                    } else {
+                            for (int c = 0; c < 32; c += 8) {
+                                const uint4 hv = *reinterpret_cast<const uint4*>(hrow + c0 + c);
+                                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&hv);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (n0 + c0 + c < p.N) dst[c0 + c] = v[c];
+                                for (int e = 0; e < 4; ++e) {
+                                    const float2 f2 = __bfloat1622float2(h2[e]);
+                                    v[c + 2 * e] += f2.x;
+                                    v[c + 2 * e + 1] += f2.y;
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (n0 + c0 + c < p.N) v[c] += __bfloat162float(hrow[c0 + c]);
+                        }
+                    }
+                    if (dst) {
+                        if (vec_ok && full) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) *reinterpret_cast<float4*>(dst + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (n0 + c0 + c < p.N) dst[c0 + c] = v[c];
+                        }
+                    }
+                    if (dst16) {
+                        if (vec16_ok && full) {
+#pragma unroll
+                            for (int c = 0; c < 32; c += 8) {
+                                __align__(16) __nv_bfloat162 o2[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) o2[e] = __floats2bfloat162_rn(v[c + 2 * e], v[c + 2 * e + 1]);
+                                *reinterpret_cast<uint4*>(dst16 + c0 + c) = *reinterpret_cast<const uint4*>(o2);
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (n0 + c0 + c < p.N) dst16[c0 + c] = __float2bfloat16(v[c]);
+                        }
                     }
                 }
             }
@@ -269,6 +317,20 @@ inline cudaError_t lm_ce_stream_launch(cudaStream_t stream, int sms, const float
     return cudaGetLastError();
 }
 
+// fp32 -> bf16 copies of GEMM operands (a_L, W_up), 4 elements per thread (n a multiple of 4).  W_up sits
+// behind lambda[L] in the flat parameter vector, so its address is 16-byte aligned only when L % 4 == 0:
+// src_vec says whether the source may be read as float4.
+__global__ void to_bf16_kernel(const float* __restrict__ x, long long n, bf16* __restrict__ out, int src_vec) {
+    const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= n) return;
+    const float4 v = src_vec ? *reinterpret_cast<const float4*>(x + i) : make_float4(x[i], x[i + 1], x[i + 2], x[i + 3]);
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<unsigned*>(&lo);
+    pk.y = *reinterpret_cast<unsigned*>(&hi);
+    *reinterpret_cast<uint2*>(out + i) = pk;
+}
+
 // Host side: tensor maps and launch for one GEMM shape.
 struct GemmPlan {
     bool ready = false;
@@ -312,9 +374,19 @@ inline pac_status gemm_plan_create(GemmPlan& gp, int device, const bf16* A, long
     return PAC_OK;
 }
 
+// Optional extras of a launch: a bf16 copy of the output and / or the residual rows of the last cached layer.
+struct GemmExtras {
+    bf16* C16 = nullptr; long long ldc16 = 0;
+    const bf16* add_cache = nullptr; const int* ids = nullptr; long long n_cache = 0; int L = 0, S = 0;
+};
+
 inline pac_status gemm_launch(const GemmPlan& gp, cudaStream_t stream, int M, float* C, long long ldc, unsigned* status,
-                              long long* launches) {
+                              long long* launches, const GemmExtras* ex = nullptr) {
     GemmParams p{};
+    if (ex) {
+        p.C16 = ex->C16; p.ldc16 = ex->ldc16;
+        p.add_cache = ex->add_cache; p.ids = ex->ids; p.n_cache = ex->n_cache; p.L = ex->L; p.S = ex->S;
+    }
     p.M = M; p.N = gp.N; p.K = gp.K;
     p.m_tiles = (M + GT_BM - 1) / GT_BM;
     p.n_tiles = (gp.N + GT_BN - 1) / GT_BN;
