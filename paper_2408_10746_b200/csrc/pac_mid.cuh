@@ -391,19 +391,21 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     for (int g = 0; g < GPT; ++g)
 #pragma unroll
         for (int e = 0; e < 4; ++e) daLr[g][e] = live[g] ? daL[j4[g] + e] : 0.f;
-    unsigned closed[GPT][4];                              // bit l set: the gate of layer l is closed
+    int top_closed[GPT][4];                               // highest layer whose gate is closed (-1: none): open from there up only
 #pragma unroll
     for (int g = 0; g < GPT; ++g)
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-            closed[g][e] = (ACT == PAC_ACT_RELU) ? (~mask[g][e] & (L >= 32 ? 0xffffffffu : ((1u << L) - 1u))) : 0u;
+        for (int e = 0; e < 4; ++e) {
+            const unsigned closed = (ACT == PAC_ACT_RELU) ? (~mask[g][e] & (L >= 32 ? 0xffffffffu : ((1u << L) - 1u))) : 0u;
+            top_closed[g][e] = 31 - __clz(closed);        // __clz(0) = 32
+        }
     // one layer of one group: du_l out, this thread's share of dlambda_l added to `part`
     auto reverse_step = [&](int l, int g, const float4& w4, float& part, float cp, float lm) {
         const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
         float dv[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const bool open = (closed[g][e] >> l) == 0u;       // gates l .. L all open
+            const bool open = l > top_closed[g][e];            // gates l .. L all open
             const float dz = open ? daLr[g][e] * cp : 0.f;
             part = fmaf(dz, wv[e], part);
             dv[e] = lm * dz;                                   // du_l
@@ -433,11 +435,19 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             cp_async_commit();
         };
         for (int i = 0; i < MID_RING; ++i) request(L - 1 - i);
+        // the launch geometry of this mode gives every group of a thread the same four columns, so the
+        // per-layer coefficients are formed once per thread and layer
+        DU* dst[GPT];
+#pragma unroll
+        for (int g = 0; g < GPT; ++g) dst[g] = du + (long long)(L - 1) * p.lstride + base[g];
 #pragma unroll 1
         for (int l = L - 1; l >= 0; --l) {
             cp_async_wait_group<MID_RING - 1>();
             float part = 0.f;
             const float cp = cprod[l], lm = lam_s[l];          // read once per layer (the stores below could alias them)
+            float dzc[4], duc[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { dzc[e] = daLr[0][e] * cp; duc[e] = lm * dzc[e]; }
             uint2 x[GPT];
 #pragma unroll
             for (int g = 0; g < GPT; ++g)
@@ -447,8 +457,21 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 if (live[g]) {
                     const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x[g].x));
                     const float2 c2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x[g].y));
-                    reverse_step(l, g, make_float4(a2.x, a2.y, c2.x, c2.y), part, cp, lm);
+                    const float wv[4] = {a2.x, a2.y, c2.x, c2.y};
+                    float dv[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const bool open = l > top_closed[g][e];
+                        part = fmaf(open ? dzc[e] : 0.f, wv[e], part);
+                        dv[e] = open ? duc[e] : 0.f;
+                    }
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<unsigned*>(&lo);
+                    pk.y = *reinterpret_cast<unsigned*>(&hi);
+                    *reinterpret_cast<uint2*>(dst[g]) = pk;
                 }
+                dst[g] -= p.lstride;
             }
             request(l - MID_RING);
             part = warp_sum(part);
@@ -774,8 +797,13 @@ inline MidPlan mid_plan_parked(const Dims& dm) {
         const long long need = (long long)Sg * (dm.r / 4);
         if (need > 4 * 512) continue;
         const int gpt = need <= 512 ? 1 : need <= 1024 ? 2 : 4;
-        int th = (int)(((need + gpt - 1) / gpt + 31) / 32 * 32);
-        if (th < 128) th = 128;
+        // every group of a thread must land on the same four columns: threads a multiple of the groups per token
+        const int gtok = dm.r / 4;
+        int unit = 32;
+        while (unit % gtok != 0) unit += 32;                    // lcm(32, r/4)
+        int th = (int)(((need + gpt - 1) / gpt + unit - 1) / unit * unit);
+        if (th < 128) th = (128 + unit - 1) / unit * unit;
+        if (th > 512) continue;
         int scratch;
         const size_t floats = mid_base_floats(dm, Sg, dg, th, &scratch, false) + (size_t)MID_RING * gpt * th * 2;    // + the state ring (8 bytes per slot)
         if (floats > 110 * 1024 / sizeof(float)) continue;                // two CTAs per SM
