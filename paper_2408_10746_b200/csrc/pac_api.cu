@@ -62,6 +62,7 @@ struct Scratch {
     float* dw_part = nullptr;      // split partials of dW_down
     unsigned* gates = nullptr;     // [M][r] ReLU gates of all layers, one word per element (chain-in-epilogue forward)
     float* pool_part = nullptr;    // [B][s_chunks * 4][r] token sums of a_L per 32-token group (chain-in-epilogue forward)
+    float* prodW = nullptr;        // [r][C] W_up W_head of the current parameters (stand-alone head kernels)
 };
 
 // Saved activations and work buffers of the transformer-body adapters (fp32, sized for max_batch).
@@ -160,6 +161,11 @@ struct pac_ctx {
     int chain_blocks_max = 0;
     Scratch sc;
     unsigned* status = nullptr;    // device status words
+    // counters that let the kernels of a step hand over to each other without waiting for whole grids to drain:
+    // [0] CTAs of forward halves done so far, [1 ...] row splits done so far per W_down tile (never reset)
+    unsigned* sync_words = nullptr;
+    unsigned fwd_target = 0, tile_target = 0;
+    bool step_handshake = false;   // the step being enqueued uses them
     // host staging (pinned)
     int* h_ids = nullptr;          // [STAGE_SLOTS][max_batch]
     cudaEvent_t slot_ev[STAGE_SLOTS] = {};
@@ -725,8 +731,11 @@ pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     pac_status st;
     time_mark(c, 2, false);
     if (use_tensor(c)) {
+        const bool hs = c->step_handshake && !reduce_splits;
+        if (hs) c->tile_target += (unsigned)tensor_splits(c->tplan, B);
         st = tensor_dw_down(c->tplan, c->stream, d_ids, B, c->sc.du16, c->grads + c->lay.w_down, c->sc.dw_part,
-                            reduce_splits, c->status, &c->launches, next_stamp(c, 1));
+                            reduce_splits, c->status, &c->launches, next_stamp(c, 1), hs ? c->sync_words : nullptr, c->fwd_target,
+                            hs ? c->sync_words + 1 : nullptr);
         if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
     } else {
         st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
@@ -751,11 +760,32 @@ MidParams mid_params(pac_ctx* c, const MidPlan& mp, const int* d_ids, int B, boo
     p.pooled_a = sc.pooled_a; p.dlogits = sc.dlogits;
     p.loss_b = sc.loss_b; p.lam_part = sc.lam_part; p.logits_out = train ? sc.logits : d_logits_out;
     p.status = c->status;
+    p.prodW = nullptr;
+    p.fwd_done = nullptr;
+    if (c->step_handshake && train) {
+        p.fwd_done = c->sync_words;
+        c->fwd_target += (unsigned)(B * mp.G);                // every CTA of this launch raises it once
+    }
     return p;
 }
 
+// W_up W_head for the stand-alone head kernels, once per forward (launched ahead of the down-projections so that
+// it overlaps the tail of the previous step's optimizer update).
+pac_status head_matrix_enqueue(pac_ctx* c) {
+    const Dims& dm = c->dm;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_launch_config(&cfg, attr, dim3(cdiv((long long)dm.r * dm.C, 8)), dim3(256), 0, c->stream);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, head_matrix_kernel, (const float*)(c->params + c->lay.w_up),
+                                       (const float*)(c->params + c->lay.w_head), dm.d, dm.r, dm.C, c->sc.prodW);
+    c->launches++;
+    if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "head matrix kernel launch failed: %s", cudaGetErrorString(e));
+    return PAC_OK;
+}
+
 pac_status mid_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, float* d_logits_out) {
-    const MidParams p = mid_params(c, c->mplan, d_ids, B, train, d_logits_out);
+    MidParams p = mid_params(c, c->mplan, d_ids, B, train, d_logits_out);
+    p.prodW = c->sc.prodW;
     cudaError_t e = mid_launch(c->mplan, p, c->cfg.act, use_tensor(c), c->stream);
     c->launches++;
     if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "fused head kernel launch failed: %s", cudaGetErrorString(e));
@@ -795,6 +825,8 @@ pac_status chain_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     cp.parked = c->sc.du16; cp.layer_stride = (long long)c->max_rows * dm.r;
     cp.gates = c->sc.gates; cp.pool_part = c->sc.pool_part;
     cp.status = c->status; cp.stamp = next_stamp(c, 0);
+    pac_status hs = head_matrix_enqueue(c);
+    if (hs != PAC_OK) return hs;
     time_mark(c, 0, false);
     cudaError_t e = chain_fwd_launch(c->tplan.map_cache_fwd, c->tplan.map_w, cp, c->tplan.smem_fwd, c->cfg.act, c->stream);
     c->launches++;
@@ -802,6 +834,7 @@ pac_status chain_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "chain-in-epilogue forward launch failed: %s", cudaGetErrorString(e));
     MidParams p = mid_params(c, c->pplan, d_ids, B, train, d_logits_out);
     p.gates = c->sc.gates; p.pool_part = c->sc.pool_part; p.n_pool_parts = cp.s_chunks * CF_POOL_PARTS;
+    p.prodW = c->sc.prodW;
     time_mark(c, 1, false);
     e = mid_launch_parked(c->pplan, p, c->cfg.act, c->stream);
     c->launches++;
@@ -820,6 +853,7 @@ pac_status cls_forward_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, 
         time_mark(c, 0, true);
         return st;
     }
+    if ((st = head_matrix_enqueue(c)) != PAC_OK) return st;
     if ((st = down_projection(c, d_ids, B)) != PAC_OK) return st;
     time_mark(c, 1, false);
     st = mid_enqueue(c, d_ids, B, train, d_logits_out);
@@ -864,6 +898,11 @@ pac_status finalize_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, 
         f.next_dev_tag = c->zc_dev_tag + (next_seq & 1u);
     }
     f.status = c->status;
+    if (c->step_handshake) {
+        f.fwd_done = c->sync_words; f.fwd_target = c->fwd_target;
+        if (f.splits > 1) { f.tile_done = c->sync_words + 1; f.tile_target = c->tile_target; }
+        f.tile_rows = 128 * c->tplan.bp.chunks; f.d_groups = c->tplan.bp.d_groups;
+    }
     const unsigned rest_blocks = cdiv(dm.d, FIN_KB);
     f.rest_blocks = (int)rest_blocks;
     const size_t fin_smem = sizeof(float) * ((size_t)2 * B * FIN_KB + (size_t)dm.r * FIN_KB + (size_t)FIN_KB * dm.C);
@@ -886,6 +925,9 @@ pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, con
         return hp ? adam_enqueue(c, hp) : PAC_OK;
     }
     if (use_fused_cls(c)) {
+        // on the tensor-core path the three or four kernels of a step hand over through counters
+        c->step_handshake = use_tensor(c) && c->sync_words && c->timing != 1;
+        struct Reset { pac_ctx* c; ~Reset() { c->step_handshake = false; } } reset{c};
         if ((st = cls_forward_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
         if (c->step_host_ids) d_ids = c->sc.ids;          // the forward kernel left a device copy for the later kernels
         if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
@@ -932,8 +974,8 @@ void free_all(pac_ctx* c) {
     Scratch& s = c->sc;
     if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
-                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.aL16, s.wup16, s.dy16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, c->tb.buf, c->params, c->grads,
-                    c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
+                    s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.aL16, s.wup16, s.dy16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, s.prodW, c->tb.buf, c->params, c->grads,
+                    c->m, c->v, c->status, c->sync_words, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (int k = 0; k < 2; ++k) {
@@ -1161,6 +1203,7 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
         A(dmalloc(c, &s.loss_b, cfg->max_batch));
         A(dmalloc(c, &s.gvec, (long long)cfg->max_batch * dm.d));
         A(dmalloc(c, &s.daL, (long long)cfg->max_batch * dm.r));
+        A(dmalloc(c, &s.prodW, (long long)dm.r * dm.C));
     } else {
         A(dmalloc(c, &s.loss_b, c->max_rows));
         A(dmalloc(c, &s.daL, Mr));
@@ -1232,6 +1275,12 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
                     }
                 }
                 c->tensor_ok = (st == PAC_OK);
+                if (c->tensor_ok && cls) {
+                    const long long words = 1 + (long long)dm.L * c->tplan.bp.d_groups;
+                    A(dmalloc(c, &c->sync_words, words));
+                    if (st == PAC_OK) CU_OK(c, cudaMemsetAsync(c->sync_words, 0, sizeof(unsigned) * words, c->stream));
+                    c->fwd_target = c->tile_target = 0;
+                }
                 if (c->tensor_ok && fwd_plan.ok) {
                     fwd_plan.max_clusters = fused_fwd_max_clusters(fwd_plan, cfg->act);
                     if (fwd_plan.max_clusters > 0) c->fplan = fwd_plan;

@@ -52,6 +52,8 @@ struct MidParams {
     float* lam_part;            // [L][B*G]
     float* logits_out;          // [B][C] (train: scratch copy; eval: caller's buffer)
     unsigned* status;
+    unsigned* fwd_done;         // optional: raised once per CTA when its du rows and per-sample outputs are written
+    const float* prodW;         // optional [r][C]: W_up W_head, formed once per step by head_matrix_kernel (else per CTA)
 };
 
 constexpr int MID_MAX_C = 32;
@@ -129,7 +131,8 @@ __device__ __forceinline__ void mid_prefetch_head(const MidParams& p, const MidS
 // index among them; none of it depends on u, so it can run while u is still being produced.
 __device__ __forceinline__ void mid_head_products(const MidParams& p, const MidShared& h, int q, int w, int nw, int lane) {
     const int k0 = q * p.dg, kn = max(0, min(p.dg, p.d - k0));
-    for (int j = w; j <= p.r; j += nw) {
+    // with the sample-independent rows already formed for the whole step only the hbar row is left
+    for (int j = p.prodW ? p.r + w : w; j <= p.r; j += nw) {
         for (int c0 = 0; c0 < p.C; c0 += 4) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
             for (int kk = lane; kk < kn; kk += 32) {
@@ -146,10 +149,27 @@ __device__ __forceinline__ void mid_head_products(const MidParams& p, const MidS
         }
     }
 }
+// prodW[j][c] = sum_k W_up[j][k] W_head[k][c], one warp per entry, k in lane order then a fixed shuffle tree.  The
+// product does not depend on the sample: the stand-alone head kernels take it from here instead of forming
+// it again in every CTA (the one-launch forward forms it on warps that would otherwise idle under the stream).
+__global__ void __launch_bounds__(256) head_matrix_kernel(const float* __restrict__ W_up, const float* __restrict__ W_head, int d, int r,
+                                                          int C, float* __restrict__ prodW) {
+    pdl_trigger();
+    pdl_wait();                      // the parameters come from the optimizer update before this kernel
+    const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (e >= r * C) return;
+    const int j = e / C, c = e - j * C;
+    float acc = 0.f;
+    for (int k = lane; k < d; k += 32) acc = fmaf(W_up[(long long)j * d + k], W_head[(long long)k * C + c], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) prodW[e] = acc;
+}
+
 // After a cluster-wide barrier behind mid_head_products: the sum over the cluster, in rank order.  The
 // last row also takes the classifier bias, so the head needs no global load of its own later on.
 __device__ __forceinline__ void mid_sum_products(const MidParams& p, const MidShared& h, cg::cluster_group& cluster, int t, int nthr) {
     for (int e = t; e < (p.r + 1) * p.C; e += nthr) {
+        if (p.prodW && e < p.r * p.C) { h.prod[e] = p.prodW[e]; continue; }
         float acc = 0.f;
         for (int g = 0; g < p.G; ++g) acc += cluster.map_shared_rank(h.prodq, g)[e];
         if (e >= p.r * p.C) acc = p.b_head[e - p.r * p.C] + acc;      // b_head + (mean_s h_L) W_head
@@ -516,6 +536,12 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int wv = 0; wv < nwarps; ++wv) acc += lred[wv * LT + t];
         p.lam_part[(long long)t * (p.B * p.G) + blockIdx.x] = acc;
     }
+    if (p.fwd_done) {
+        // everything the second pass and the finalisation need from this CTA is written: tell them, so that they
+        // need not wait for the whole grid to drain
+        __syncthreads();
+        if (t == 0) counter_signal(p.fwd_done);
+    }
     cluster.barrier_wait();                               // keep shared memory alive until every peer has read it
 }
 
@@ -564,6 +590,11 @@ struct FinalizeParams {
     // Device status words: when a bounded wait of this or an earlier step has run out, the gradients
     // are not trustworthy, so nothing is written to the gradients, parameters or moments.
     unsigned* status;
+    // Optional hand-shakes through counters (see BwdParams): fwd_done >= fwd_target: the forward half's outputs
+    // are written; tile_done[tile] >= tile_target: every row split of that W_down tile has written its partial.
+    const unsigned* fwd_done; unsigned fwd_target;
+    const unsigned* tile_done; unsigned tile_target;
+    int tile_rows, d_groups;                                 // rows of W_down^l per tile, tiles per layer
 };
 
 constexpr int FIN_KB = 4;       // hidden-width columns per head-side block of the finalisation kernel
@@ -603,6 +634,11 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     // Set by a wait that ran out in this step's forward half or in any earlier step since the last
     // pac_sync (the forward half has completed whenever this kernel runs); a wait that runs out in this
     // step's second pass is seen by the W_down blocks behind their own wait below.
+    if (f.fwd_done && blk < f.rest_blocks) {
+        // formal acquire of the forward half's outputs (the counter is complete by the time this kernel starts)
+        if (threadIdx.x == 0) counter_wait_ge(f.fwd_done, f.fwd_target, f.status);
+        __syncthreads();
+    }
     const bool dead = status_timed_out(f.status);
     if (blk < 0) {
         // dlambda_l (one warp per layer, lanes over the per-block partials, fixed
@@ -705,7 +741,19 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         }
         return;
     }
-    pdl_wait();
+    if (f.tile_done) {
+        // this block's elements lie in one or two tiles of the second pass: wait for exactly those tiles' row splits
+        if (threadIdx.x == 0) {
+            const long long dr = (long long)f.d * f.r, first = (long long)(blk - f.rest_blocks) * blockDim.x * 4;
+            const long long last = min(first + (long long)blockDim.x * 4, lay.lam) - 1;
+            const int t0 = (int)(first / dr) * f.d_groups + (int)(((first % dr) / f.r) / f.tile_rows);
+            const int t1 = (int)(last / dr) * f.d_groups + (int)(((last % dr) / f.r) / f.tile_rows);
+            for (int tt = t0; tt <= t1; ++tt) counter_wait_ge(f.tile_done + tt, f.tile_target, f.status);
+        }
+        __syncthreads();
+    } else {
+        pdl_wait();
+    }
     {
         // W_down block, four consecutive elements per thread
         const long long i = i_wd;
