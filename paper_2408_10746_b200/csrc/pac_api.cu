@@ -161,11 +161,6 @@ struct pac_ctx {
     int chain_blocks_max = 0;
     Scratch sc;
     unsigned* status = nullptr;    // device status words
-    // counters that let the kernels of a step hand over to each other without waiting for whole grids to drain:
-    // [0] CTAs of forward halves done so far, [1 ...] row splits done so far per W_down tile (never reset)
-    unsigned* sync_words = nullptr;
-    unsigned fwd_target = 0, tile_target = 0;
-    bool step_handshake = false;   // the step being enqueued uses them
     // host staging (pinned)
     int* h_ids = nullptr;          // [STAGE_SLOTS][max_batch]
     cudaEvent_t slot_ev[STAGE_SLOTS] = {};
@@ -731,11 +726,8 @@ pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     pac_status st;
     time_mark(c, 2, false);
     if (use_tensor(c)) {
-        const bool hs = c->step_handshake && !reduce_splits;
-        if (hs) c->tile_target += (unsigned)tensor_splits(c->tplan, B);
         st = tensor_dw_down(c->tplan, c->stream, d_ids, B, c->sc.du16, c->grads + c->lay.w_down, c->sc.dw_part,
-                            reduce_splits, c->status, &c->launches, next_stamp(c, 1), hs ? c->sync_words : nullptr, c->fwd_target,
-                            hs ? c->sync_words + 1 : nullptr);
+                            reduce_splits, c->status, &c->launches, next_stamp(c, 1));
         if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
     } else {
         st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);
@@ -761,11 +753,6 @@ MidParams mid_params(pac_ctx* c, const MidPlan& mp, const int* d_ids, int B, boo
     p.loss_b = sc.loss_b; p.lam_part = sc.lam_part; p.logits_out = train ? sc.logits : d_logits_out;
     p.status = c->status;
     p.prodW = nullptr;
-    p.fwd_done = nullptr;
-    if (c->step_handshake && train) {
-        p.fwd_done = c->sync_words;
-        c->fwd_target += (unsigned)(B * mp.G);                // every CTA of this launch raises it once
-    }
     return p;
 }
 
@@ -898,11 +885,6 @@ pac_status finalize_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, 
         f.next_dev_tag = c->zc_dev_tag + (next_seq & 1u);
     }
     f.status = c->status;
-    if (c->step_handshake) {
-        f.fwd_done = c->sync_words; f.fwd_target = c->fwd_target;
-        if (f.splits > 1) { f.tile_done = c->sync_words + 1; f.tile_target = c->tile_target; }
-        f.tile_rows = 128 * c->tplan.bp.chunks; f.d_groups = c->tplan.bp.d_groups;
-    }
     const unsigned rest_blocks = cdiv(dm.d, FIN_KB);
     f.rest_blocks = (int)rest_blocks;
     const size_t fin_smem = sizeof(float) * ((size_t)2 * B * FIN_KB + (size_t)dm.r * FIN_KB + (size_t)FIN_KB * dm.C);
@@ -925,9 +907,6 @@ pac_status train_enqueue(pac_ctx* c, const int* d_ids, int B, float* d_loss, con
         return hp ? adam_enqueue(c, hp) : PAC_OK;
     }
     if (use_fused_cls(c)) {
-        // on the tensor-core path the three or four kernels of a step hand over through counters
-        c->step_handshake = use_tensor(c) && c->sync_words && c->timing != 1;
-        struct Reset { pac_ctx* c; ~Reset() { c->step_handshake = false; } } reset{c};
         if ((st = cls_forward_enqueue(c, d_ids, B, true, nullptr)) != PAC_OK) return st;
         if (c->step_host_ids) d_ids = c->sc.ids;          // the forward kernel left a device copy for the later kernels
         if ((st = dw_down(c, d_ids, B, false)) != PAC_OK) return st;
@@ -975,7 +954,7 @@ void free_all(pac_ctx* c) {
     if (c->hc.on) s.hbar = nullptr;            // points into a staging slot, freed below
     void* ptrs[] = {s.ids, s.u, s.a, s.du, s.du16, s.lam_part, s.loss, s.hbar, s.pooled_a, s.pooled_y, s.logits,
                     s.dlogits, s.loss_b, s.gvec, s.daL, s.y, s.lm_logits, s.dy, s.y16, s.dlog16, s.aL16, s.wup16, s.dy16, s.wdT, s.lm_part, s.dw_part, s.gates, s.pool_part, s.prodW, c->tb.buf, c->params, c->grads,
-                    c->m, c->v, c->status, c->sync_words, c->d_perm, c->d_losses, c->d_stamps};
+                    c->m, c->v, c->status, c->d_perm, c->d_losses, c->d_stamps};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     for (int k = 0; k < 2; ++k) {
@@ -1275,12 +1254,6 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
                     }
                 }
                 c->tensor_ok = (st == PAC_OK);
-                if (c->tensor_ok && cls) {
-                    const long long words = 1 + (long long)dm.L * c->tplan.bp.d_groups;
-                    A(dmalloc(c, &c->sync_words, words));
-                    if (st == PAC_OK) CU_OK(c, cudaMemsetAsync(c->sync_words, 0, sizeof(unsigned) * words, c->stream));
-                    c->fwd_target = c->tile_target = 0;
-                }
                 if (c->tensor_ok && fwd_plan.ok) {
                     fwd_plan.max_clusters = fused_fwd_max_clusters(fwd_plan, cfg->act);
                     if (fwd_plan.max_clusters > 0) c->fplan = fwd_plan;

@@ -52,7 +52,6 @@ struct MidParams {
     float* lam_part;            // [L][B*G]
     float* logits_out;          // [B][C] (train: scratch copy; eval: caller's buffer)
     unsigned* status;
-    unsigned* fwd_done;         // optional: raised once per CTA when its du rows and per-sample outputs are written
     const float* prodW;         // optional [r][C]: W_up W_head, formed once per step by head_matrix_kernel (else per CTA)
 };
 
@@ -536,12 +535,6 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         for (int wv = 0; wv < nwarps; ++wv) acc += lred[wv * LT + t];
         p.lam_part[(long long)t * (p.B * p.G) + blockIdx.x] = acc;
     }
-    if (p.fwd_done) {
-        // everything the second pass and the finalisation need from this CTA is written: tell them, so that they
-        // need not wait for the whole grid to drain
-        __syncthreads();
-        if (t == 0) counter_signal(p.fwd_done);
-    }
     cluster.barrier_wait();                               // keep shared memory alive until every peer has read it
 }
 
@@ -590,11 +583,6 @@ struct FinalizeParams {
     // Device status words: when a bounded wait of this or an earlier step has run out, the gradients
     // are not trustworthy, so nothing is written to the gradients, parameters or moments.
     unsigned* status;
-    // Optional hand-shakes through counters (see BwdParams): fwd_done >= fwd_target: the forward half's outputs
-    // are written; tile_done[tile] >= tile_target: every row split of that W_down tile has written its partial.
-    const unsigned* fwd_done; unsigned fwd_target;
-    const unsigned* tile_done; unsigned tile_target;
-    int tile_rows, d_groups;                                 // rows of W_down^l per tile, tiles per layer
 };
 
 constexpr int FIN_KB = 4;       // hidden-width columns per head-side block of the finalisation kernel
@@ -634,11 +622,6 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
     // Set by a wait that ran out in this step's forward half or in any earlier step since the last
     // pac_sync (the forward half has completed whenever this kernel runs); a wait that runs out in this
     // step's second pass is seen by the W_down blocks behind their own wait below.
-    if (f.fwd_done && blk < f.rest_blocks) {
-        // formal acquire of the forward half's outputs (the counter is complete by the time this kernel starts)
-        if (threadIdx.x == 0) counter_wait_ge(f.fwd_done, f.fwd_target, f.status);
-        __syncthreads();
-    }
     const bool dead = status_timed_out(f.status);
     if (blk < 0) {
         // dlambda_l (one warp per layer, lanes over the per-block partials, fixed
@@ -741,19 +724,7 @@ __global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
         }
         return;
     }
-    if (f.tile_done) {
-        // this block's elements lie in one or two tiles of the second pass: wait for exactly those tiles' row splits
-        if (threadIdx.x == 0) {
-            const long long dr = (long long)f.d * f.r, first = (long long)(blk - f.rest_blocks) * blockDim.x * 4;
-            const long long last = min(first + (long long)blockDim.x * 4, lay.lam) - 1;
-            const int t0 = (int)(first / dr) * f.d_groups + (int)(((first % dr) / f.r) / f.tile_rows);
-            const int t1 = (int)(last / dr) * f.d_groups + (int)(((last % dr) / f.r) / f.tile_rows);
-            for (int tt = t0; tt <= t1; ++tt) counter_wait_ge(f.tile_done + tt, f.tile_target, f.status);
-        }
-        __syncthreads();
-    } else {
-        pdl_wait();
-    }
+    pdl_wait();
     {
         // W_down block, four consecutive elements per thread
         const long long i = i_wd;

@@ -78,32 +78,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, status, limit_ns);
 }
-// Bounded wait on a counter in global memory that other CTAs (of this or of an earlier kernel) raise with
-// a fence and an atomic add once their results are written: returns when the counter has reached `target`
-// (compared modulo 2^32, so counters never need a reset).  On expiry the status word is set.
-__device__ __forceinline__ unsigned ld_acquire_gpu_u32(const unsigned* p) {
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __noinline__ bool counter_wait_ge(const unsigned* ctr, unsigned target, unsigned* status) {
-    const unsigned long long t0 = global_ns();
-    for (uint32_t it = 0;; ++it) {
-        if ((int)(ld_acquire_gpu_u32(ctr) - target) >= 0) return true;
-        if ((it & 15u) == 15u) {
-            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
-            __nanosleep(40);
-        }
-    }
-    if (status) atomicAdd(&status[ST_TIMEOUT], 1u);
-    return false;
-}
-// Raises such a counter: call after a block barrier behind the block's last global stores.
-__device__ __forceinline__ void counter_signal(unsigned* ctr) {
-    __threadfence();
-    atomicAdd(ctr, 1u);
-}
-
 // The same for a whole warp: lane 0 waits, every lane gets the same answer.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
                                                unsigned long long limit_ns = WAIT_LIMIT_NS) {
@@ -451,12 +425,6 @@ struct BwdParams {
     float* out;                            // splits == 1: dW_down [L][d][r]; else partials [J][L][d][r]
     unsigned* status;
     unsigned long long* stamp;             // optional stream-phase timestamps (see stamp_begin)
-    // Optional hand-shakes through counters instead of whole-grid completion (both null: plain grid dependency).
-    // fwd_done: raised once by every CTA of the forward half when its du rows are written; this kernel starts
-    // streaming when it has reached fwd_target.  tile_done[layer * d_groups + group]: raised by each row split of
-    // a tile when its partial sums are written, for the finalisation blocks of that tile.
-    const unsigned* fwd_done; unsigned fwd_target;
-    unsigned* tile_done;
 };
 
 // ---------------------------------------------------------------------------
@@ -501,13 +469,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
-    if (p.fwd_done) {
-        // every CTA of the forward half has published its du rows: no need to wait for that grid to drain
-        if (threadIdx.x == 0 && !counter_wait_ge(p.fwd_done, p.fwd_target, p.status)) abort_sh = 1;
-        __syncthreads();
-    } else {
-        pdl_wait();
-    }
+    pdl_wait();
     // the successor may start only now: when it runs, the forward half of this step (and with it the
     // previous step's parameter update) is known to be complete
     pdl_trigger();
@@ -595,8 +557,6 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     }
     tc_fence_before();
     __syncthreads();
-    // this split's partial sums of its tile are written (or, after an abort, will never be: the status word says so)
-    if (threadIdx.x == 0 && p.tile_done) counter_signal(&p.tile_done[l * p.d_groups + g]);
     drain_after_abort(abort_flag);
     if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
 }
@@ -807,11 +767,9 @@ inline int tensor_splits(const TensorPlan& tp, int B) {
 // ([J][L][d][r]) for the caller's own reduction.
 inline pac_status tensor_dw_down(TensorPlan& tp, cudaStream_t stream, const int* d_ids, int B, const bf16* /*du16*/,
                                  float* dW, float* part, bool reduce_splits, unsigned* status, long long* launches,
-                                 unsigned long long* stamp = nullptr, const unsigned* fwd_done = nullptr, unsigned fwd_target = 0,
-                                 unsigned* tile_done = nullptr) {
+                                 unsigned long long* stamp = nullptr) {
     BwdParams p = tp.bp;
     p.ids = d_ids; p.B = B; p.status = status; p.stamp = stamp;
-    p.fwd_done = fwd_done; p.fwd_target = fwd_target; p.tile_done = tile_done;
     const int J = tensor_splits(tp, B);
     p.splits = J;
     p.out = J > 1 ? part : dW;
