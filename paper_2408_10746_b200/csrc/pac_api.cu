@@ -793,7 +793,7 @@ pac_status fused_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
         fp.mid.pref_seq = seq;
     }
     fp.mid.early_ids = c->step_early_ids ? 1 : 0;
-    fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset; fp.wide_n = pl.wide_n;
+    fp.k_chunks = pl.k_chunks; fp.stages = pl.stages; fp.mid_offset = pl.mid_offset; fp.state_offset = pl.state_offset; fp.n_land = pl.n_land; fp.wide_n = pl.wide_n;
     fp.stamp = next_stamp(c, 0);
     cudaError_t e = fused_fwd_launch(pl, c->tplan.map_cache_fwd, c->tplan.map_w, fp, c->cfg.act, c->stream);
     c->launches++;

@@ -73,6 +73,14 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// Shared-memory chain state, [layer][thread] 16-byte groups: group c4 of a CTA's token s_local sits at group
+// c4 ^ state_swizzle(s_local, groups per token) of the token's row, so that rows written one per lane (an
+// accumulator row per thread) and rows read one group per lane are both free of bank conflicts.
+__device__ __forceinline__ int state_swizzle(int s_local, int groups_per_tok) {
+    const int m = (groups_per_tok & (groups_per_tok - 1)) ? 0 : min(groups_per_tok, 8) - 1;
+    return s_local & m;
+}
+
 // Where the per-layer chain state (u_l on the way in, u_l - a_{l-1} for the reverse pass) lives.
 enum {
     STATE_SMEM = 0,      // this CTA's shared memory, prefetched from the global u buffer with cp.async
@@ -179,10 +187,13 @@ __device__ __forceinline__ void mid_sum_products(const MidParams& p, const MidSh
 // Everything after the down-projections for one sample, executed by one CTA (rank q) of the
 // sample's cluster.  GPT: 4-column groups per thread.  u_s: STATE_SMEM: [L][GPT][nt] float4 state;
 // products_ready: the caller has already prefetched the head
-// operands, run mid_head_products and passed a cluster barrier.
+// operands, run mid_head_products and passed a cluster barrier.  n_landed > 0 (STATE_SMEM): the state of the
+// top n_landed layers is not fetched from the u buffer: the cluster's CTAs write it into u_s directly and the
+// mbarrier land_bar (shared-memory address, phase 0) completes when all of it has arrived.
 template <int ACT, typename DU, int GPT, int STATE>
 __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& cluster, float4* u_s, const MidShared& h,
-                                         bool products_ready, long long known_id = -1) {
+                                         bool products_ready, long long known_id = -1, int n_landed = 0, uint32_t land_bar = 0,
+                                         volatile int* abort_flag = nullptr) {
     constexpr int LT = MID_MAX_L;
     const int q = (int)cluster.block_rank();
     const int b = blockIdx.x / p.G;
@@ -193,7 +204,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
           *lg = h.lg, *lam_s = h.lam_s, *lred = h.lred, *cprod = h.cprod, *daL = h.daL;
 
     const int groups_per_tok = r >> 2;
-    int s_local[GPT], j4[GPT];
+    int s_local[GPT], j4[GPT], ts[GPT];                   // ts: this thread's slot in a layer's plane of the shared-memory state
     bool live[GPT];
     long long base[GPT];
 #pragma unroll
@@ -204,16 +215,17 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         const int s = q * p.Sg + s_local[g];
         live[g] = s_local[g] < p.Sg && s < p.S;
         base[g] = ((long long)b * p.S + s) * r + j4[g];
+        ts[g] = t ^ state_swizzle(s_local[g], groups_per_tok);
     }
     DU* du = reinterpret_cast<DU*>(p.du);
     // layer l of group g: read u, park / fetch the reverse-pass state
     auto load_u = [&](int l, int g) -> float4 {
-        if constexpr (STATE == STATE_SMEM) return u_s[((size_t)l * GPT + g) * nt + t];
+        if constexpr (STATE == STATE_SMEM) return u_s[((size_t)l * GPT + g) * nt + ts[g]];
         else return *reinterpret_cast<const float4*>(p.u + (long long)l * p.lstride + base[g]);
     };
     auto store_w = [&](int l, int g, const float* wv) {
         if constexpr (STATE == STATE_SMEM) {
-            u_s[((size_t)l * GPT + g) * nt + t] = make_float4(wv[0], wv[1], wv[2], wv[3]);
+            u_s[((size_t)l * GPT + g) * nt + ts[g]] = make_float4(wv[0], wv[1], wv[2], wv[3]);
         } else if constexpr (sizeof(DU) == 2) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]), hi = __floats2bfloat162_rn(wv[2], wv[3]);
             uint2 pk;
@@ -226,7 +238,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     };
     auto load_w = [&](int l, int g) -> float4 {
         if constexpr (STATE == STATE_SMEM) {
-            return u_s[((size_t)l * GPT + g) * nt + t];
+            return u_s[((size_t)l * GPT + g) * nt + ts[g]];
         } else if constexpr (sizeof(DU) == 2) {
             const uint2 pk = *reinterpret_cast<const uint2*>(du + (long long)l * p.lstride + base[g]);
             const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
@@ -243,7 +255,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
 #pragma unroll
         for (int g = 0; g < GPT; ++g)
             if (live[g])
-                for (int l = 0; l < L; ++l) cp_async_16(u_s + ((size_t)l * GPT + g) * nt + t, p.u + (long long)l * p.lstride + base[g]);
+                for (int l = 0; l < L - n_landed; ++l) cp_async_16(u_s + ((size_t)l * GPT + g) * nt + ts[g], p.u + (long long)l * p.lstride + base[g]);
     }
     cp_async_commit();                                                          // group: u
     const int label = p.train ? p.labels[id] : 0;                               // fetched long before the head needs it
@@ -263,6 +275,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     // code once, so small code beats unrolled code).
     unsigned mask[GPT][4];
     float ap[GPT][4];
+    bool landed = false;
 #pragma unroll
     for (int g = 0; g < GPT; ++g) {
 #pragma unroll
@@ -278,6 +291,10 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         if (live[g]) {
 #pragma unroll 1
             for (int l0 = 0; l0 < L; l0 += 4) {
+                if (n_landed > 0 && !landed && l0 + 4 > L - n_landed) {
+                    mbar_wait(land_bar, 0, abort_flag, p.status);      // the handed-over layers have arrived
+                    landed = true;
+                }
                 float4 uq[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
