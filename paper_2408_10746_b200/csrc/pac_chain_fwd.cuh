@@ -73,31 +73,39 @@ down_chain_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid
     }
     const int id = (int)safe_id(p.ids, b, p.N, (threadIdx.x == 0 && sc == 0) ? p.status : nullptr);
 
+    // Both pipeline loops carry ring positions, parities, addresses and descriptors from step to step: their own
+    // instruction streams are on the critical path of a K step.
     if (warp == 0) {
         const uint64_t pol = l2_policy_evict_first();
-        uint32_t it = 0;
+        uint32_t s = 0, eph = 1;                                   // eph: parity of the "stage free" phase to wait for
+        const uint32_t ring0 = smem_u32(smem);
+        uint32_t dst = ring0;
         bool ok = true;
         if (lane == 0) stamp_begin(p.stamp);
         for (int l = 0; l < p.L && ok; ++l) {
-            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+            for (int kc = 0; kc < p.k_chunks; ++kc) {
+                if (!mbar_wait_uniform(empty0 + 8 * s, eph, abort_flag, p.status)) { ok = false; break; }
                 if (elect_one()) {
-                    mbar_expect_tx(full0 + 8 * s, stage_bytes);
-                    tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, sc * FWD_ROWS, l, id, pol);
+                    const uint32_t full = full0 + 8 * s;
+                    mbar_expect_tx(full, stage_bytes);
+                    tma_load_4d_hint(dst, &map_cache, full, kc * KC, sc * FWD_ROWS, l, id, pol);
                     for (int rb = 0; rb < r_blocks; ++rb)
-                        tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full0 + 8 * s, rb * 64, kc * KC, 0, l);
+                        tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full, rb * 64, kc * KC, 0, l);
                 }
                 __syncwarp();
+                dst += stage_bytes;
+                if (++s == (uint32_t)p.stages) { s = 0; eph ^= 1u; dst = ring0; }
             }
         }
     } else if (warp == 1) {
         // hi and lo blocks lie side by side along N ([r block][hi|lo], 64 columns each): one MMA of
         // N = 128 * r_blocks per K step leaves u_hi | u_lo next to each other in TMEM
         const uint32_t idesc = instr_desc_bf16(FWD_ROWS, 128 * r_blocks, 0, 1);
-        uint32_t it = 0;
+        // descriptors hold addresses in units of 16 bytes
+        const uint64_t a_desc0 = smem_desc_sw128(smem_u32(smem), 16, 1024), w_desc0 = smem_desc_sw128(smem_u32(smem) + b_off, b_box, 1024);
+        const uint64_t desc_step = (uint64_t)(stage_bytes >> 4);
+        uint64_t ad0 = a_desc0, bw0 = w_desc0;
+        uint32_t s = 0, ph = 0;
         bool ok = true;
         for (int l = 0; l < p.L && ok; ++l) {
             const int buf = l & 1;
@@ -105,13 +113,9 @@ down_chain_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid
             if (!mbar_wait_uniform(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_stride;
-            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
+            for (int kc = 0; kc < p.k_chunks; ++kc) {
                 if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + b_off;
-                const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024), bw0 = smem_desc_sw128(b0, b_box, 1024);
                 if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < KC / 16; ++k)
@@ -119,6 +123,8 @@ down_chain_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid
                     umma_commit(empty0 + 8 * s);
                 }
                 __syncwarp();
+                ad0 += desc_step; bw0 += desc_step;
+                if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; ad0 = a_desc0; bw0 = w_desc0; }
             }
             if (!ok) break;
             if (elect_one()) umma_commit(accf0 + 8 * buf);

@@ -313,35 +313,46 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
 
     // The two pipeline loops are run by whole converged warps with one elected lane issuing, so that
     // addresses, coordinates and descriptors stay warp-uniform values.
+    // Both pipeline loops carry ring positions, parities, addresses and descriptors from step to step: their own
+    // instruction streams are on the critical path of a K step.
     if (warp == 0) {
-        uint32_t it = 0;
         // cache tiles are read once per pass: evict them first, so that u, du, the weight shadow and
         // the optimizer state stay L2-resident
         const uint64_t pol = l2_policy_evict_first();
+        uint32_t s = 0, eph = 1;                                   // eph: parity of the "stage free" phase to wait for
+        const uint32_t ring0 = smem_u32(smem);
+        uint32_t dst = ring0;
         bool ok = true;
         if (lane == 0) stamp_begin(p.stamp);
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
             const int sc = t % p.s_chunks, b = (t / p.s_chunks) % p.B, l = t / (p.s_chunks * p.B);
             const int id = (int)safe_id(p.ids, b, p.N, nullptr);
-            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+            for (int kc = 0; kc < p.k_chunks; ++kc) {
+                if (!mbar_wait_uniform(empty0 + 8 * s, eph, abort_flag, p.status)) { ok = false; break; }
                 if (elect_one()) {
-                    mbar_expect_tx(full0 + 8 * s, a_bytes + b_bytes);
-                    tma_load_4d_hint(dst, &map_cache, full0 + 8 * s, kc * KC, sc * FWD_ROWS, l, id, pol);
+                    const uint32_t full = full0 + 8 * s;
+                    mbar_expect_tx(full, a_bytes + b_bytes);
+                    tma_load_4d_hint(dst, &map_cache, full, kc * KC, sc * FWD_ROWS, l, id, pol);
                     for (int rb = 0; rb < r_blocks; ++rb)
-                        tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full0 + 8 * s, rb * 64, kc * KC, 0, l);
+                        tma_load_4d(dst + b_off + rb * 2 * b_box, &map_w, full, rb * 64, kc * KC, 0, l);
                 }
                 __syncwarp();
+                dst += stage_bytes;
+                if (++s == (uint32_t)p.stages) { s = 0; eph ^= 1u; dst = ring0; }
             }
         }
     } else if (warp == 1) {
         // wide_n: the hi and lo blocks lie next to each other along N ([r block][hi|lo] in 64-column
         // blocks), so one MMA of N = 128 * r_blocks yields u_hi | u_lo side by side in TMEM
         const uint32_t idesc = p.wide_n ? instr_desc_bf16(FWD_ROWS, 128 * r_blocks, 0, 1) : instr_desc_bf16(FWD_ROWS, r_pad, 0, 1);
-        uint32_t it = 0, tile_n = 0;
+        // descriptors of a stage's first 16-wide K step (start-address field in 16-byte units); later steps
+        // only move the start address: +32 B per step in the K-major A tile, +2048 B (16 rows) in B
+        const uint32_t ring0 = smem_u32(smem);
+        const uint64_t a_desc0 = smem_desc_sw128(ring0, 16, 1024), bw_desc0 = smem_desc_sw128(ring0 + b_off, b_box, 1024);
+        const uint64_t bh_desc0 = smem_desc_sw128(ring0 + b_off, 2 * b_box, 1024), bl_desc0 = smem_desc_sw128(ring0 + b_off + b_box, 2 * b_box, 1024);
+        const uint64_t desc_step = (uint64_t)(stage_bytes >> 4);
+        uint64_t doff = 0;
+        uint32_t s = 0, ph = 0, tile_n = 0;
         for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_n) {
             const int buf = tile_n & 1;
             const uint32_t aph = (tile_n >> 1) & 1;
@@ -349,19 +360,13 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_stride);
             bool ok = true;
-            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                const int s = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
+            for (int kc = 0; kc < p.k_chunks; ++kc) {
                 if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + b_off;
-                // descriptors of the first 16-wide K step; later steps only move the start address
-                // (field in 16-byte units): +32 B per step in the K-major A tile, +2048 B (16 rows) in B
-                const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
-                const uint64_t bh0 = smem_desc_sw128(b0, 2 * b_box, 1024), bl0 = smem_desc_sw128(b0 + b_box, 2 * b_box, 1024);
+                const uint64_t ad0 = a_desc0 + doff, bh0 = bh_desc0 + doff, bl0 = bl_desc0 + doff;
                 if (elect_one()) {
                     if (p.wide_n) {
-                        const uint64_t bw0 = smem_desc_sw128(b0, b_box, 1024);
+                        const uint64_t bw0 = bw_desc0 + doff;
 #pragma unroll
                         for (int k = 0; k < KC / 16; ++k)
                             umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bw0 + (uint64_t)(k * 128), idesc, (kc | k) ? 1u : 0u);
@@ -375,6 +380,8 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     umma_commit(empty0 + 8 * s);          // frees the smem slot once these MMAs are done
                 }
                 __syncwarp();
+                doff += desc_step;
+                if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; doff = 0; }
             }
             if (!ok) break;
             if (elect_one()) umma_commit(accf0 + 8 * buf);    // accumulator complete
@@ -488,48 +495,60 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     // previous step's parameter update) is known to be complete
     pdl_trigger();
 
+    // Both pipeline loops carry ring positions, parities, addresses and descriptors from step to step.
     if (warp == 0) {
-        uint32_t it = 0;
         const uint64_t pol = l2_policy_evict_first();
         if (lane == 0 && rt1 > rt0) stamp_begin(p.stamp);
-        for (int rt = rt0; rt < rt1; ++rt, ++it) {
-            const int sc = rt % p.s_chunks, b = rt / p.s_chunks;
-            const int id = (int)safe_id(p.ids, b, p.N, nullptr);
-            const int s = it % p.stages;
-            const uint32_t ph = (it / p.stages) & 1;
-            if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-            const uint32_t dst = smem_u32(smem + (size_t)s * stage_bytes);
+        uint32_t s = 0, eph = 1;                                   // eph: parity of the "stage free" phase to wait for
+        const uint32_t ring0 = smem_u32(smem);
+        uint32_t dst = ring0;
+        int sc = rt0 % p.s_chunks, b = rt0 / p.s_chunks;
+        int id = rt1 > rt0 ? (int)safe_id(p.ids, b, p.N, nullptr) : 0;
+        for (int rt = rt0; rt < rt1; ++rt) {
+            if (!mbar_wait_uniform(empty0 + 8 * s, eph, abort_flag, p.status)) break;
             if (elect_one()) {
-                mbar_expect_tx(full0 + 8 * s, stage_bytes);
+                const uint32_t full = full0 + 8 * s;
+                mbar_expect_tx(full, stage_bytes);
                 for (int q = 0; q < 2 * p.chunks; ++q)
-                    tma_load_4d_hint(dst + q * box_bytes, &map_cache, full0 + 8 * s, col0 + q * 64, sc * BWD_KR, l, id, pol);
+                    tma_load_4d_hint(dst + q * box_bytes, &map_cache, full, col0 + q * 64, sc * BWD_KR, l, id, pol);
                 for (int q = 0; q < p.r_blocks; ++q)
-                    tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full0 + 8 * s, q * 64, b * p.S + sc * BWD_KR, l);
+                    tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full, q * 64, b * p.S + sc * BWD_KR, l);
             }
             __syncwarp();
+            dst += stage_bytes;
+            if (++s == (uint32_t)p.stages) { s = 0; eph ^= 1u; dst = ring0; }
+            if (++sc == p.s_chunks) {
+                sc = 0; ++b;
+                if (rt + 1 < rt1) id = (int)safe_id(p.ids, b, p.N, nullptr);
+            }
         }
     } else if (warp == 1) {
         const uint32_t idesc = instr_desc_bf16(128, r_pad, 1, 1);
-        uint32_t it = 0;
+        // descriptors of a stage's first K step (start-address field in 16-byte units)
+        const uint32_t ring0 = smem_u32(smem);
+        const uint64_t a_desc0 = smem_desc_sw128(ring0, box_bytes, 1024), b_desc0 = smem_desc_sw128(ring0 + a_bytes, box_bytes, 1024);
+        const uint64_t desc_step = (uint64_t)(stage_bytes >> 4), a_chunk = (uint64_t)((2 * box_bytes) >> 4);
+        uint64_t doff = 0;
+        uint32_t s = 0, ph = 0, first = 0;                         // first: 0 until the first K step has been issued
         bool ok = true;
-        for (int rt = rt0; rt < rt1 && ok; ++rt, ++it) {
-            const int s = it % p.stages;
-            const uint32_t ph = (it / p.stages) & 1;
+        for (int rt = rt0; rt < rt1 && ok; ++rt) {
             if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t a0 = smem_u32(smem + (size_t)s * stage_bytes), b0 = a0 + a_bytes;
-            const uint64_t bd0 = smem_desc_sw128(b0, box_bytes, 1024);
             if (elect_one()) {
+                const uint64_t ad0 = a_desc0 + doff, bd0 = b_desc0 + doff;
                 // consecutive MMAs alternate between the column blocks' accumulators: an MMA that adds to
                 // the result of the one before it would have to wait for that one to finish
 #pragma unroll
                 for (int k = 0; k < BWD_KR / 16; ++k)          // 16 tokens = 2048 B further along K in both operands
                     for (int c = 0; c < p.chunks; ++c)
-                        umma_bf16(tmem_base + (uint32_t)(c * r_pad), smem_desc_sw128(a0 + c * 2 * box_bytes, box_bytes, 1024) + (uint64_t)(k * 128),
-                                  bd0 + (uint64_t)(k * 128), idesc, (it | (uint32_t)k) ? 1u : 0u);
+                        umma_bf16(tmem_base + (uint32_t)(c * r_pad), ad0 + (uint64_t)c * a_chunk + (uint64_t)(k * 128),
+                                  bd0 + (uint64_t)(k * 128), idesc, (first | (uint32_t)k) ? 1u : 0u);
                 umma_commit(empty0 + 8 * s);
             }
             __syncwarp();
+            first = 1;
+            doff += desc_step;
+            if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; doff = 0; }
         }
         if (ok) {
             if (elect_one()) umma_commit(accf);
