@@ -727,7 +727,8 @@ pac_status dw_down(pac_ctx* c, const int* d_ids, int B, bool reduce_splits) {
     time_mark(c, 2, false);
     if (use_tensor(c)) {
         st = tensor_dw_down(c->tplan, c->stream, d_ids, B, c->sc.du16, c->grads + c->lay.w_down, c->sc.dw_part,
-                            reduce_splits, c->status, &c->launches, next_stamp(c, 1));
+                            reduce_splits, c->status, &c->launches, next_stamp(c, 1),
+                            c->step_early_ids && !c->step_host_ids);       // ids no kernel in flight writes
         if (st != PAC_OK) return fail(c, st, "tensor-core dW_down launch failed: %s", tensor_last_error());
     } else {
         st = c->dtype == PAC_F32 ? dw_down_simt<float>(c, d_ids, B) : dw_down_simt<bf16>(c, d_ids, B);

@@ -249,6 +249,7 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, int a_mn_ma
 }
 
 constexpr int TC_THREADS = 192;            // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int DW_THREADS = 320;            // dW_down: two epilogue warps per TMEM lane quadrant (warps 2-9)
 constexpr int KC = 64;                     // bf16 elements per 128-byte swizzled row
 constexpr int FWD_ROWS = 128;              // token rows per forward tile (MMA M)
 constexpr int BWD_KR = 64;                 // token rows per backward stage (MMA K extent per stage)
@@ -443,6 +444,7 @@ struct BwdParams {
     int r_blocks;                          // ceil(r / 64)
     int stages;
     int tmem_cols;
+    int early_ids;                         // 1: no kernel ahead of this one in the stream writes the ids
     float* out;                            // splits == 1: dW_down [L][d][r]; else partials [J][L][d][r]
     unsigned* status;
     unsigned long long* stamp;             // optional stream-phase timestamps (see stamp_begin)
@@ -454,7 +456,7 @@ struct BwdParams {
 // du_l (MN-major B: N = r), accumulates [128 x r] blocks in TMEM over all its rows and writes
 // them once.  With splits > 1 the partial sums are added afterwards in split order.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(DW_THREADS, 1)
 dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_constant__ CUtensorMap map_du, BwdParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -490,6 +492,24 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
+    // The cache never changes: with ids that were final before this launch the h tiles of the first ring are
+    // requested while the predecessor still runs; only du (its result) has to wait.
+    uint32_t pre = 0;
+    if (p.early_ids && warp == 0 && rt1 > rt0) {
+        pre = (uint32_t)min(rt1 - rt0, p.stages);
+        if (elect_one()) {
+            const uint64_t pol = l2_policy_evict_first();
+            for (uint32_t i = 0; i < pre; ++i) {
+                const int rt = rt0 + (int)i, sc = rt % p.s_chunks, b = rt / p.s_chunks;
+                const int id = (int)safe_id(p.ids, b, p.N, nullptr);
+                const uint32_t dst = smem_u32(smem + (size_t)i * stage_bytes);
+                mbar_expect_tx(full0 + 8 * i, stage_bytes);
+                for (int q = 0; q < 2 * p.chunks; ++q)
+                    tma_load_4d_hint(dst + q * box_bytes, &map_cache, full0 + 8 * i, col0 + q * 64, sc * BWD_KR, l, id, pol);
+            }
+        }
+        __syncwarp();
+    }
     pdl_wait();
     // the successor may start only now: when it runs, the forward half of this step (and with it the
     // previous step's parameter update) is known to be complete
@@ -505,14 +525,22 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
         int sc = rt0 % p.s_chunks, b = rt0 / p.s_chunks;
         int id = rt1 > rt0 ? (int)safe_id(p.ids, b, p.N, nullptr) : 0;
         for (int rt = rt0; rt < rt1; ++rt) {
-            if (!mbar_wait_uniform(empty0 + 8 * s, eph, abort_flag, p.status)) break;
-            if (elect_one()) {
-                const uint32_t full = full0 + 8 * s;
-                mbar_expect_tx(full, stage_bytes);
-                for (int q = 0; q < 2 * p.chunks; ++q)
-                    tma_load_4d_hint(dst + q * box_bytes, &map_cache, full, col0 + q * 64, sc * BWD_KR, l, id, pol);
-                for (int q = 0; q < p.r_blocks; ++q)
-                    tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full, q * 64, b * p.S + sc * BWD_KR, l);
+            const uint32_t full = full0 + 8 * s;
+            if (pre > 0) {
+                // first ring: the h tiles are already on their way
+                --pre;
+                if (elect_one())
+                    for (int q = 0; q < p.r_blocks; ++q)
+                        tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full, q * 64, b * p.S + sc * BWD_KR, l);
+            } else {
+                if (!mbar_wait_uniform(empty0 + 8 * s, eph, abort_flag, p.status)) break;
+                if (elect_one()) {
+                    mbar_expect_tx(full, stage_bytes);
+                    for (int q = 0; q < 2 * p.chunks; ++q)
+                        tma_load_4d_hint(dst + q * box_bytes, &map_cache, full, col0 + q * 64, sc * BWD_KR, l, id, pol);
+                    for (int q = 0; q < p.r_blocks; ++q)
+                        tma_load_3d(dst + a_bytes + q * box_bytes, &map_du, full, q * 64, b * p.S + sc * BWD_KR, l);
+                }
             }
             __syncwarp();
             dst += stage_bytes;
@@ -555,7 +583,8 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
             __syncwarp();
         }
     } else {
-        const int q = warp & 3;
+        const int q = warp & 3;                                   // TMEM lane quadrant this warp may read
+        const int ne = ((int)(blockDim.x >> 5) - 2) >> 2, e16 = ((warp - 2) >> 2) * 16;      // warps per quadrant; this warp's first 16 columns
         if (rt1 > rt0) {
             if (mbar_wait_warp(accf, 0, abort_flag, p.status)) {
                 tc_fence_after();
@@ -564,7 +593,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
                     const int k = col0 + c * 128 + q * 32 + lane;             // column of h = row of dW_down
                     float* dst = p.out + (((long long)j * p.L + l) * p.d + k) * p.r;
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * r_pad);
-                    for (int c0 = 0; c0 < p.r; c0 += 16) {
+                    for (int c0 = e16; c0 < p.r; c0 += 16 * ne) {              // the quadrant's warps share its columns
                         float v[16];
                         tmem_ld16(taddr + c0, v);
                         tmem_ld_wait();
@@ -581,7 +610,7 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
             // no rows in this split: the partial is zero
             for (int c = 0; c < p.chunks; ++c) {
                 const int k = col0 + c * 128 + q * 32 + lane;
-                if (k < p.d) {
+                if (k < p.d && e16 == 0) {
                     float* dst = p.out + (((long long)j * p.L + l) * p.d + k) * p.r;
                     for (int c0 = 0; c0 < p.r; ++c0) dst[c0] = 0.f;
                 }
@@ -800,16 +829,16 @@ inline int tensor_splits(const TensorPlan& tp, int B) {
 // ([J][L][d][r]) for the caller's own reduction.
 inline pac_status tensor_dw_down(TensorPlan& tp, cudaStream_t stream, const int* d_ids, int B, const bf16* /*du16*/,
                                  float* dW, float* part, bool reduce_splits, unsigned* status, long long* launches,
-                                 unsigned long long* stamp = nullptr) {
+                                 unsigned long long* stamp = nullptr, bool early_ids = false) {
     BwdParams p = tp.bp;
-    p.ids = d_ids; p.B = B; p.status = status; p.stamp = stamp;
+    p.ids = d_ids; p.B = B; p.status = status; p.stamp = stamp; p.early_ids = early_ids ? 1 : 0;
     const int J = tensor_splits(tp, B);
     p.splits = J;
     p.out = J > 1 ? part : dW;
     const int grid = p.L * p.d_groups * J;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    pdl_launch_config(&cfg, attr, dim3((unsigned)grid), dim3(TC_THREADS), tp.smem_bwd, stream);
+    pdl_launch_config(&cfg, attr, dim3((unsigned)grid), dim3(DW_THREADS), tp.smem_bwd, stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, dw_down_tc_kernel, tp.map_cache_bwd, tp.map_du, p);
     (*launches)++;
     if (e != cudaSuccess) { tensor_err() = cudaGetErrorString(e); return PAC_ERR_CUDA; }
