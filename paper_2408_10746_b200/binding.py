@@ -16,6 +16,7 @@ import numpy as np
 PAC_F32, PAC_BF16 = 0, 1
 PAC_ACT_RELU, PAC_ACT_IDENTITY = 0, 1
 PAC_HEAD_MEANPOOL_CLS, PAC_HEAD_FROZEN_LM = 0, 1
+PAC_BODY_POINTWISE, PAC_BODY_TRANSFORMER = 0, 1
 PAC_OPT_KERNEL_PATH = 0
 PAC_OPT_KERNEL_TIMING = 1
 STATUS_NAMES = ["PAC_OK", "PAC_ERR_INVALID_ARG", "PAC_ERR_BAD_STATE", "PAC_ERR_SAMPLE_ID_RANGE",
