@@ -95,7 +95,10 @@ typedef enum {
                                  1 = force the plain fp32-FMA kernels,
                                  2 = tensor-core path, forward half always as two plain launches,
                                  3 = tensor-core path, one-launch forward whenever the shape allows it,
-                                 4 = tensor-core path, chain-in-epilogue forward whenever the shape allows it;
+                                 4 = tensor-core path, chain-in-epilogue forward whenever the shape allows it (with
+                                     r > 64 and an even number of 128-token tiles its CTAs work in pairs that share
+                                     each weight tile),
+                                 5 = as 4, but never in CTA pairs;
                                  set before adapter_init */
     PAC_OPT_KERNEL_TIMING = 1 /* 0 = off (default), 1 = bracket the cache-stream kernels with events
                                  (pac_kernel_times), 2 = device-side timestamps of the two passes' stream

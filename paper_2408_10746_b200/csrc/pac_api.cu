@@ -185,6 +185,7 @@ struct pac_ctx {
     FusedFwdPlan fplan{};          // down-projections + classifier-head kernel in one launch (short sequences)
     MidPlan pplan{};               // head / reverse-chain kernel behind the chain-in-epilogue forward
     bool chain_ok = false;         // the chain-in-epilogue forward can take this shape
+    int chain_pair_stages = 0;     // > 0: its CTA-pair form can too, with this many stages
     int forward_mode = 0;          // 0: automatic, 2: down-projections and head phase as two plain launches, 3: one-launch
                                    // forward whenever the shape allows, 4: chain-in-epilogue forward whenever the shape allows
     GemmPlan g_logits{}, g_dy{};   // tensor-core GEMMs of the frozen LM head
@@ -693,14 +694,14 @@ bool use_fused_cls(const pac_ctx* c) { return c->cfg.head == PAC_HEAD_MEANPOOL_C
 // and chain phases do not overlap across waves); larger batches keep the two separate kernels.
 bool use_fused_fwd(const pac_ctx* c, int B) {
     if (!use_fused_cls(c) || !use_tensor(c) || !c->fplan.ok) return false;
-    if (c->forward_mode == 4 && c->chain_ok) return false;
+    if ((c->forward_mode == 4 || c->forward_mode == 5) && c->chain_ok) return false;
     return c->forward_mode == 3 || B <= c->fplan.max_clusters;
 }
 // Chain-in-epilogue forward: one CTA per 128-token tile walks all layers, so it needs enough tiles to fill
 // the device (long sequences or large batches); the one-launch cluster forward keeps the short shapes.
 bool use_chain_fwd(const pac_ctx* c, int B) {
     if (!use_fused_cls(c) || !use_tensor(c) || !c->chain_ok || c->forward_mode == 2 || c->forward_mode == 3) return false;
-    if (c->forward_mode == 4) return true;
+    if (c->forward_mode == 4 || c->forward_mode == 5) return true;
     if (use_fused_fwd(c, B)) return false;
     return 2 * B * c->tplan.fp.s_chunks >= c->sms;
 }
@@ -816,7 +817,10 @@ pac_status chain_fwd_enqueue(pac_ctx* c, const int* d_ids, int B, bool train, fl
     pac_status hs = head_matrix_enqueue(c);
     if (hs != PAC_OK) return hs;
     time_mark(c, 0, false);
-    cudaError_t e = chain_fwd_launch(c->tplan.map_cache_fwd, c->tplan.map_w, cp, c->tplan.smem_fwd, c->cfg.act, c->stream);
+    const bool pair = c->chain_pair_stages > 0 && c->forward_mode != 5 && ((B * cp.s_chunks) & 1) == 0;
+    if (pair) cp.stages = c->chain_pair_stages;
+    cudaError_t e = pair ? chain_pair_launch(c->tplan.map_cache_fwd, c->tplan.map_w, cp, chain_pair_smem(cp.stages), c->cfg.act, c->stream)
+                         : chain_fwd_launch(c->tplan.map_cache_fwd, c->tplan.map_w, cp, c->tplan.smem_fwd, c->cfg.act, c->stream);
     c->launches++;
     time_mark(c, 0, true);
     if (e != cudaSuccess) return fail(c, PAC_ERR_CUDA, "chain-in-epilogue forward launch failed: %s", cudaGetErrorString(e));
@@ -1252,6 +1256,12 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
                         A(dmalloc(c, &s.gates, Mr));
                         A(dmalloc(c, &s.pool_part, (long long)cfg->max_batch * c->tplan.fp.s_chunks * CF_POOL_PARTS * dm.r));
                         c->chain_ok = (st == PAC_OK);
+                        int max_smem = 0;
+                        if (c->chain_ok && chain_pair_supported(dm) &&
+                            cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) == cudaSuccess) {
+                            const int ps = chain_pair_stages(max_smem);
+                            c->chain_pair_stages = ps >= 3 ? ps : 0;
+                        }
                     }
                 }
                 c->tensor_ok = (st == PAC_OK);
@@ -1644,7 +1654,7 @@ pac_status pac_params_changed(pac_ctx* c) {
 pac_status pac_set_option(pac_ctx* c, int option, int value) {
     NEED_CTX(c);
     if (option == PAC_OPT_KERNEL_PATH) {
-        if (value < 0 || value > 4) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0, 1, 2, 3 or 4");
+        if (value < 0 || value > 5) return fail(c, PAC_ERR_INVALID_ARG, "pac_set_option: kernel path must be 0 ... 5");
         if (c->inited) return fail(c, PAC_ERR_BAD_STATE, "pac_set_option: set the kernel path before pac_adapter_init");
         c->force_simt = value == 1;
         c->forward_mode = value >= 2 ? value : 0;

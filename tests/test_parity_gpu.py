@@ -299,7 +299,7 @@ def tc_check(spec, max_batch, act, ids=None, loss_tol=2e-2, chain_tol=1e-2, head
         assert ctx.kernel_path() in ("tensor+fused_forward", "tensor", "tensor+chain_forward")
         assert ctx.kernel_path() == "tensor+fused_forward" or not can_fuse or max_batch > 8
         assert ctx.kernel_path() != "tensor+chain_forward" or (can_chain and 2 * max_batch * ((spec.S + 127) // 128) >= 100)
-    elif kernel_path == 4:
+    elif kernel_path in (4, 5):
         assert ctx.kernel_path() == ("tensor+chain_forward" if can_chain else "tensor")
     else:
         assert ctx.kernel_path() == ("tensor+fused_forward" if can_fuse and kernel_path == 3 else "tensor")
@@ -350,6 +350,17 @@ def test_tensor_path_chain_in_epilogue_forward(spec, max_batch, act):
     ctx.sync()
     ref = po.eval_logits(case.oracle_params(flat), case.H(ids), act)
     assert rel_l2(out.cpu().numpy(), ref) < 1e-3
+
+
+TC_CHAIN_WIDE = [s for s in TC_CHAIN_FORWARD if s[0].r > 64]
+
+
+@pytest.mark.parametrize("spec,max_batch,act", TC_CHAIN_WIDE, ids=[s[0].name for s in TC_CHAIN_WIDE])
+def test_tensor_path_chain_forward_without_cta_pairs(spec, max_batch, act):
+    """Adapters wider than 64 run the chain-in-epilogue forward in CTA pairs that share each weight tile
+    (kernel path 4, above); the single-CTA form of the same kernel, which odd tile counts fall back to, is
+    exercised here."""
+    tc_check(spec, max_batch, act, kernel_path=5)
 
 
 def test_chain_in_epilogue_forward_ten_steps():
