@@ -83,10 +83,8 @@ __device__ __forceinline__ void chain_epilogue(const ChainFwdParams& p, const fl
                     a[c][e] = z;
                 }
             }
-            if (p.train && row_ok) {
-                *reinterpret_cast<uint4*>(pk + c0) = *reinterpret_cast<const uint4*>(park);
-                *reinterpret_cast<uint4*>(pk + c0 + 8) = *reinterpret_cast<const uint4*>(park + 8);
-            }
+            if (p.train && row_ok)          // 16 bf16 = one whole 32-byte sector
+                st_global_32(pk + c0, *reinterpret_cast<const uint4*>(park), *reinterpret_cast<const uint4*>(park + 8));
         }
         tc_fence_before();
         __syncwarp();
@@ -101,8 +99,9 @@ __device__ __forceinline__ void chain_epilogue(const ChainFwdParams& p, const fl
 #pragma unroll
             for (int c = 0; c < CH; ++c)
 #pragma unroll
-                for (int e = 0; e < 16; e += 4)
-                    *reinterpret_cast<uint4*>(g + col_base + c * 16 + e) = make_uint4(gate[c][e], gate[c][e + 1], gate[c][e + 2], gate[c][e + 3]);
+                for (int e = 0; e < 16; e += 8)
+                    st_global_32(g + col_base + c * 16 + e, make_uint4(gate[c][e], gate[c][e + 1], gate[c][e + 2], gate[c][e + 3]),
+                                 make_uint4(gate[c][e + 4], gate[c][e + 5], gate[c][e + 6], gate[c][e + 7]));
         }
         // token sums of a_L over this warp's 32 rows (fixed shuffle order); lane e of chunk c keeps column e
         float* pp = p.pool_part + ((long long)b * (p.s_chunks * CF_POOL_PARTS) + sc * CF_POOL_PARTS + quad) * p.r;

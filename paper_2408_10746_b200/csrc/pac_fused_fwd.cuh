@@ -235,9 +235,17 @@ fwd_cluster_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                         tmem_ld_wait();
                     }
                     if (row < p.S) {
+                        if (handed) {
 #pragma unroll
-                        for (int c = 0; c < 16; c += 4)
-                            *reinterpret_cast<float4*>(dst + ((((c0 + c) >> 2) ^ sw) << 2)) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                            for (int c = 0; c < 16; c += 4)
+                                *reinterpret_cast<float4*>(dst + ((((c0 + c) >> 2) ^ sw) << 2)) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                        } else {
+                            // whole 32-byte sectors
+#pragma unroll
+                            for (int c = 0; c < 16; c += 8)
+                                st_global_32(dst + c0 + c, make_uint4(__float_as_uint(v[c]), __float_as_uint(v[c + 1]), __float_as_uint(v[c + 2]), __float_as_uint(v[c + 3])),
+                                             make_uint4(__float_as_uint(v[c + 4]), __float_as_uint(v[c + 5]), __float_as_uint(v[c + 6]), __float_as_uint(v[c + 7])));
+                        }
                     }
                 }
             }

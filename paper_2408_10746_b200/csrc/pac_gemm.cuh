@@ -137,6 +137,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * GT_BN);
             const bool vec_ok = (p.ldc & 3) == 0, vec16_ok = (p.ldc16 & 7) == 0 && (p.N & 7) == 0;
+            const bool vec32_ok = (p.ldc & 7) == 0 && (reinterpret_cast<uintptr_t>(p.C) & 31) == 0;
             for (int c0 = 0; c0 < GT_BN; c0 += 32) {
                 float v[32];
                 tmem_ld32(taddr + c0, v);
@@ -163,7 +164,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     }
                     if (dst) {
-                        if (vec_ok && full) {
+                        if (vec32_ok && full) {
+                            // whole 32-byte sectors
+#pragma unroll
+                            for (int c = 0; c < 32; c += 8)
+                                st_global_32(dst + c0 + c, make_uint4(__float_as_uint(v[c]), __float_as_uint(v[c + 1]), __float_as_uint(v[c + 2]), __float_as_uint(v[c + 3])),
+                                             make_uint4(__float_as_uint(v[c + 4]), __float_as_uint(v[c + 5]), __float_as_uint(v[c + 6]), __float_as_uint(v[c + 7])));
+                        } else if (vec_ok && full) {
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) *reinterpret_cast<float4*>(dst + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
                         } else {

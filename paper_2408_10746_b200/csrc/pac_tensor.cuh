@@ -24,6 +24,11 @@ namespace pac {
 // ---------------------------------------------------------------------------
 // PTX wrappers
 // ---------------------------------------------------------------------------
+// One 32-byte store (a whole L2 sector) from two 16-byte halves; p must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32(void* p, uint4 a, uint4 b) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
 // Programmatic dependent launch: a kernel launched with the programmatic-serialization
 // attribute may start while its predecessor in the stream is still running; pdl_wait() blocks
 // until the predecessor grid has completed and its writes are visible, pdl_trigger() lets the
@@ -459,9 +464,11 @@ down_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_c
                     tmem_ld_wait();
                 }
                 if (srow < p.S) {
+                    // r is a multiple of 16: the chunk is whole; two 32-byte sectors
 #pragma unroll
-                    for (int c = 0; c < 16; c += 4)
-                        if (c0 + c < p.r) *reinterpret_cast<float4*>(dst + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                    for (int c = 0; c < 16; c += 8)
+                        st_global_32(dst + c0 + c, make_uint4(__float_as_uint(v[c]), __float_as_uint(v[c + 1]), __float_as_uint(v[c + 2]), __float_as_uint(v[c + 3])),
+                                     make_uint4(__float_as_uint(v[c + 4]), __float_as_uint(v[c + 5]), __float_as_uint(v[c + 6]), __float_as_uint(v[c + 7])));
                 }
             }
             tc_fence_before();
@@ -639,10 +646,10 @@ dw_down_tc_kernel(const __grid_constant__ CUtensorMap map_cache, const __grid_co
                         tmem_ld16(taddr + c0, v);
                         tmem_ld_wait();
                         if (k < p.d) {
+                            // (16-byte stores: with 32-byte ones here the step measured 0.4 us slower)
 #pragma unroll
                             for (int cc = 0; cc < 16; cc += 4)
-                                if (c0 + cc < p.r)
-                                    *reinterpret_cast<float4*>(dst + c0 + cc) = make_float4(v[cc], v[cc + 1], v[cc + 2], v[cc + 3]);
+                                *reinterpret_cast<float4*>(dst + c0 + cc) = make_float4(v[cc], v[cc + 1], v[cc + 2], v[cc + 3]);
                         }
                     }
                 }
