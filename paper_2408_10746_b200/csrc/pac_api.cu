@@ -1200,8 +1200,8 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
             A(dmalloc(c, &s.y16, (long long)c->max_rows * dm.d));
             A(dmalloc(c, &s.dlog16, (long long)c->max_rows * dm.C));
             if (st == PAC_OK) {
-                pac_status g1 = gemm_plan_create(c->g_logits, c->device, s.y16, c->max_rows, (const bf16*)cfg->lm_head, dm.C, dm.d, 0);
-                pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_dy, c->device, s.dlog16, c->max_rows, (const bf16*)cfg->lm_head, dm.d, dm.C, 1) : g1;
+                pac_status g1 = gemm_plan_create(c->g_logits, c->device, s.y16, c->max_rows, (const bf16*)cfg->lm_head, dm.C, dm.d, 0, c->forward_mode != 5);
+                pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_dy, c->device, s.dlog16, c->max_rows, (const bf16*)cfg->lm_head, dm.d, dm.C, 1, c->forward_mode != 5) : g1;
                 if (g1 == PAC_OK && g2 == PAC_OK) {
                     c->lm_tensor = true;
                     int max_smem = 0;
@@ -1280,8 +1280,8 @@ pac_status pac_adapter_init(pac_ctx* c, const pac_adapter_cfg* cfg, unsigned lon
         if (st == PAC_OK) {
             CU_OK(c, cudaMemsetAsync(s.aL16, 0, sizeof(bf16) * Mr, c->stream));
             CU_OK(c, cudaMemsetAsync(s.dy16, 0, sizeof(bf16) * (size_t)c->max_rows * dm.d, c->stream));
-            pac_status g1 = gemm_plan_create(c->g_y, c->device, s.aL16, c->max_rows, s.wup16, dm.d, dm.r, 1);
-            pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_daL, c->device, s.dy16, c->max_rows, s.wup16, dm.r, dm.d, 0) : g1;
+            pac_status g1 = gemm_plan_create(c->g_y, c->device, s.aL16, c->max_rows, s.wup16, dm.d, dm.r, 1, c->forward_mode != 5);
+            pac_status g2 = g1 == PAC_OK ? gemm_plan_create(c->g_daL, c->device, s.dy16, c->max_rows, s.wup16, dm.r, dm.d, 0, c->forward_mode != 5) : g1;
             c->lm_skinny_tensor = g1 == PAC_OK && g2 == PAC_OK;
         }
     }

@@ -6,7 +6,15 @@
 // TMA-fed shared-memory ring, accumulators double-buffered in TMEM (2 x 256 columns) so the
 // epilogue of one tile overlaps the MMAs of the next.  Persistent CTAs walk tiles with the M
 // index fastest, so the CTAs running at the same time share B tiles through L2.
+//
+// PAIR: the CTAs work as 2-CTA clusters on 256 x 256 tiles (tcgen05.mma.cta_group::2): each CTA loads
+// its own 128 rows of A and HALF of the B tile (128 of the 256 columns), the CTA of rank 0 counts the
+// bytes of both on its barriers and issues the MMAs.  A single CTA takes in 48 KB per K step for 512
+// clocks of tensor work, more than the 64 bytes per clock an SM receives from L2; a CTA of a pair
+// takes in 32 KB, and its ring is six stages deep instead of four.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "pac_tensor.cuh"
 
 namespace pac {
@@ -14,6 +22,9 @@ namespace pac {
 constexpr int GT_BM = 128, GT_BN = 256, GT_BK = 64, GT_STAGES = 4;
 constexpr uint32_t GT_A_BYTES = GT_BM * GT_BK * 2, GT_B_BYTES = GT_BN * GT_BK * 2, GT_STAGE = GT_A_BYTES + GT_B_BYTES;
 constexpr size_t GT_SMEM = (size_t)GT_STAGES * GT_STAGE + 1024;
+constexpr int GT_STAGES_PAIR = 6;
+constexpr uint32_t GT_STAGE_PAIR = GT_A_BYTES + GT_B_BYTES / 2;
+constexpr size_t GT_SMEM_PAIR = (size_t)GT_STAGES_PAIR * GT_STAGE_PAIR + 1024;
 
 struct GemmParams {
     int M, N, K;
@@ -33,29 +44,48 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+
+// map_b: PAIR and K-major B: boxes of 128 rows; otherwise as in the single-CTA form.
+template <bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) unsigned long long bars[2 * GT_STAGES + 4];
+    constexpr int STAGES = PAIR ? GT_STAGES_PAIR : GT_STAGES;
+    constexpr uint32_t STAGE = PAIR ? GT_STAGE_PAIR : GT_STAGE;
+    __shared__ __align__(8) unsigned long long bars[2 * GT_STAGES_PAIR + 4];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
-    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[GT_STAGES]);
-    const uint32_t accf0 = smem_u32(&bars[2 * GT_STAGES]), acce0 = smem_u32(&bars[2 * GT_STAGES + 2]);
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
+    const uint32_t accf0 = smem_u32(&bars[2 * STAGES]), acce0 = smem_u32(&bars[2 * STAGES + 2]);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = p.m_tiles * p.n_tiles;
+    uint32_t rank = 0;                                         // in the pair; 0 issues the MMAs
+    if constexpr (PAIR) rank = cooperative_groups::this_cluster().block_rank();
+    // a unit of work: one tile, or the two tiles of a pair (M indices 2i and 2i + 1, one N index)
+    const int m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    const int n_units = m_units * p.n_tiles;
+    const int unit0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, unit_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         abort_sh = 0;
-        for (int s = 0; s < GT_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 4); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, PAIR ? 8 : 4); }
         fence_mbar_init();
         tma_prefetch_desc(&map_a);
         tma_prefetch_desc(&map_b);
     }
-    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_sh), 512u); tmem_relinquish(); }
+    if (warp == 1) {
+        if constexpr (PAIR) { tmem_alloc_pair(smem_u32(&tmem_base_sh), 512u); tmem_relinquish_pair(); }
+        else { tmem_alloc(smem_u32(&tmem_base_sh), 512u); tmem_relinquish(); }
+    }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cooperative_groups::this_cluster().sync();     // the peer's barriers exist before anything arrives at them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
@@ -63,65 +93,93 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // Both pipeline loops are run by whole converged warps with one elected lane issuing, so that
     // addresses, coordinates and descriptors stay warp-uniform values.
     if (warp == 0) {
-        uint32_t it = 0;
+        uint32_t s = 0, eph = 1;                               // eph: parity of the "stage free" phase to wait for
+        const uint32_t ring0 = smem_u32(smem);
+        uint32_t dst = ring0;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-            const int m0 = (t % p.m_tiles) * GT_BM, n0 = (t / p.m_tiles) * GT_BN;
-            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                const int s = it % GT_STAGES;
-                const uint32_t ph = (it / GT_STAGES) & 1;
-                if (!mbar_wait_uniform(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-                const uint32_t dst = smem_u32(smem + (size_t)s * GT_STAGE);
+        for (int t = unit0; t < n_units && ok; t += unit_step) {
+            const int m0 = ((t % m_units) * (PAIR ? 2 : 1) + (int)rank) * GT_BM, n0 = (t / m_units) * GT_BN;
+            for (int kc = 0; kc < p.k_chunks; ++kc) {
+                if (!mbar_wait_uniform(empty0 + 8 * s, eph, abort_flag, p.status)) { ok = false; break; }
                 if (elect_one()) {
-                    mbar_expect_tx(full0 + 8 * s, GT_STAGE);
-                    tma_load_2d(dst, &map_a, full0 + 8 * s, kc * GT_BK, m0);
-                    if (p.b_mn_major) {
-                        for (int q = 0; q < GT_BN / 64; ++q)       // [64 k][64 n] boxes, one per 64 columns of N
-                            tma_load_2d(dst + GT_A_BYTES + q * 8192, &map_b, full0 + 8 * s, n0 + q * 64, kc * GT_BK);
+                    if constexpr (PAIR) {
+                        // both CTAs: own rows of A, own half of B's columns, counted on the barrier of CTA 0
+                        const uint32_t full = mapa_shared(full0 + 8 * s, 0u);
+                        if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * STAGE);
+                        tma_load_2d_pair(dst, &map_a, full, kc * GT_BK, m0);
+                        if (p.b_mn_major) {
+                            for (int q = 0; q < GT_BN / 128; ++q)  // [64 k][64 n] boxes, one per 64 columns of N
+                                tma_load_2d_pair(dst + GT_A_BYTES + q * 8192, &map_b, full, n0 + ((int)rank * 2 + q) * 64, kc * GT_BK);
+                        } else {
+                            tma_load_2d_pair(dst + GT_A_BYTES, &map_b, full, kc * GT_BK, n0 + (int)rank * (GT_BN / 2));
+                        }
                     } else {
-                        tma_load_2d(dst + GT_A_BYTES, &map_b, full0 + 8 * s, kc * GT_BK, n0);
+                        const uint32_t full = full0 + 8 * s;
+                        mbar_expect_tx(full, STAGE);
+                        tma_load_2d(dst, &map_a, full, kc * GT_BK, m0);
+                        if (p.b_mn_major) {
+                            for (int q = 0; q < GT_BN / 64; ++q)   // [64 k][64 n] boxes, one per 64 columns of N
+                                tma_load_2d(dst + GT_A_BYTES + q * 8192, &map_b, full, n0 + q * 64, kc * GT_BK);
+                        } else {
+                            tma_load_2d(dst + GT_A_BYTES, &map_b, full, kc * GT_BK, n0);
+                        }
                     }
                 }
                 __syncwarp();
+                dst += STAGE;
+                if (++s == (uint32_t)STAGES) { s = 0; eph ^= 1u; dst = ring0; }
             }
         }
     } else if (warp == 1) {
-        const uint32_t idesc = instr_desc_bf16(GT_BM, GT_BN, 0, p.b_mn_major);
-        uint32_t it = 0, tile_n = 0;
-        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_n) {
-            const int buf = tile_n & 1;
-            const uint32_t aph = (tile_n >> 1) & 1;
-            if (!mbar_wait_uniform(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GT_BN);
-            bool ok = true;
-            for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-                const int s = it % GT_STAGES;
-                const uint32_t ph = (it / GT_STAGES) & 1;
-                if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+        if (!PAIR || rank == 0) {
+            const uint32_t idesc = instr_desc_bf16(PAIR ? 2 * GT_BM : GT_BM, GT_BN, 0, p.b_mn_major);
+            // descriptors of a stage's first K step (start-address field in 16-byte units).  K-major B: rows of
+            // 128 B; MN-major B: [64 k][128 B] blocks 8192 B apart
+            const uint32_t ring0 = smem_u32(smem);
+            const uint64_t a_desc0 = smem_desc_sw128(ring0, 16, 1024);
+            const uint64_t b_desc0 = p.b_mn_major ? smem_desc_sw128(ring0 + GT_A_BYTES, 8192, 1024) : smem_desc_sw128(ring0 + GT_A_BYTES, 16, 1024);
+            const uint64_t bstep = p.b_mn_major ? 128u : 2u;     // 16 K elements further, in 16-byte units
+            const uint64_t desc_step = (uint64_t)(STAGE >> 4);
+            uint64_t doff = 0;
+            uint32_t s = 0, ph = 0, tile_n = 0;
+            for (int t = unit0; t < n_units; t += unit_step, ++tile_n) {
+                const int buf = tile_n & 1;
+                const uint32_t aph = (tile_n >> 1) & 1;
+                if (!mbar_wait_uniform(acce0 + 8 * buf, aph ^ 1, abort_flag, p.status)) break;
                 tc_fence_after();
-                const uint32_t a0 = smem_u32(smem + (size_t)s * GT_STAGE), b0 = a0 + GT_A_BYTES;
-                const uint64_t ad0 = smem_desc_sw128(a0, 16, 1024);
-                // K-major B: 256 rows of 128 B; MN-major B: four [64 k][128 B] blocks 8192 B apart
-                const uint64_t bd0 = p.b_mn_major ? smem_desc_sw128(b0, 8192, 1024) : smem_desc_sw128(b0, 16, 1024);
-                const uint64_t bstep = p.b_mn_major ? 128u : 2u;     // 16 K elements further, in 16-byte units
-                if (elect_one()) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GT_BN);
+                bool ok = true;
+                for (int kc = 0; kc < p.k_chunks; ++kc) {
+                    if (!mbar_wait_uniform(full0 + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t ad0 = a_desc0 + doff, bd0 = b_desc0 + doff;
+                    if (elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < GT_BK / 16; ++k)
-                        umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bd0 + bstep * k, idesc, (kc | k) ? 1u : 0u);
-                    umma_commit(empty0 + 8 * s);
+                        for (int k = 0; k < GT_BK / 16; ++k) {
+                            if constexpr (PAIR) umma_bf16_pair(d_tmem, ad0 + (uint64_t)(k * 2), bd0 + bstep * k, idesc, (kc | k) ? 1u : 0u);
+                            else umma_bf16(d_tmem, ad0 + (uint64_t)(k * 2), bd0 + bstep * k, idesc, (kc | k) ? 1u : 0u);
+                        }
+                        if constexpr (PAIR) umma_commit_pair(empty0 + 8 * s, (uint16_t)3);
+                        else umma_commit(empty0 + 8 * s);
+                    }
+                    __syncwarp();
+                    doff += desc_step;
+                    if (++s == (uint32_t)STAGES) { s = 0; ph ^= 1u; doff = 0; }
+                }
+                if (!ok) break;
+                if (elect_one()) {
+                    if constexpr (PAIR) umma_commit_pair(accf0 + 8 * buf, (uint16_t)3);
+                    else umma_commit(accf0 + 8 * buf);
                 }
                 __syncwarp();
             }
-            if (!ok) break;
-            if (elect_one()) umma_commit(accf0 + 8 * buf);
-            __syncwarp();
         }
     } else {
         const int q = warp & 3;
+        const uint32_t acce_arrive0 = PAIR ? mapa_shared(acce0, 0u) : acce0;     // the "drained" barriers of the CTA that issues the MMAs
         uint32_t tile_n = 0;
-        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_n) {
-            const int m0 = (t % p.m_tiles) * GT_BM, n0 = (t / p.m_tiles) * GT_BN;
+        for (int t = unit0; t < n_units; t += unit_step, ++tile_n) {
+            const int m0 = ((t % m_units) * (PAIR ? 2 : 1) + (int)rank) * GT_BM, n0 = (t / m_units) * GT_BN;
             const int buf = tile_n & 1;
             const uint32_t aph = (tile_n >> 1) & 1;
             if (!mbar_wait_warp(accf0 + 8 * buf, aph, abort_flag, p.status)) break;
@@ -198,13 +256,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_cluster(acce_arrive0 + 8 * buf);
+                else mbar_arrive(acce0 + 8 * buf);
+            }
         }
     }
     tc_fence_before();
     __syncthreads();
     drain_after_abort(abort_flag);
-    if (warp == 1) tmem_dealloc(tmem_base, 512u);
+    if constexpr (PAIR) {
+        cooperative_groups::this_cluster().sync();     // neither CTA frees TMEM or leaves while the pair's MMAs or arrivals may still touch it
+        if (warp == 1) tmem_dealloc_pair(tmem_base, 512u);
+    } else {
+        if (warp == 1) tmem_dealloc(tmem_base, 512u);
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -342,12 +408,14 @@ __global__ void to_bf16_kernel(const float* __restrict__ x, long long n, bf16* _
 struct GemmPlan {
     bool ready = false;
     CUtensorMap map_a, map_b;
+    CUtensorMap map_b_pair;        // K-major B in boxes of 128 rows, for CTA pairs (MN-major B: the same boxes as map_b)
+    bool pair = false;             // run as 2-CTA clusters on 256 x 256 tiles
     int b_mn_major = 0, N = 0, K = 0, sms = 0;
 };
 
 // A: [rows_a][K] bf16 row-major.  B: K-major [N][K], or MN-major [K][N].
 inline pac_status gemm_plan_create(GemmPlan& gp, int device, const bf16* A, long long rows_a, const bf16* B, int N, int K,
-                                   int b_mn_major) {
+                                   int b_mn_major, bool pair = true) {
     gp.ready = false;
     if (N % 8 != 0 || K % 8 != 0) { tensor_err() = "GEMM operand rows are not 16-byte multiples"; return PAC_ERR_UNSUPPORTED; }
     cudaDeviceProp prop;
@@ -365,13 +433,17 @@ inline pac_status gemm_plan_create(GemmPlan& gp, int device, const bf16* A, long
         cuuint64_t str[1] = {(cuuint64_t)N * 2};
         cuuint32_t box[2] = {64, GT_BK};
         if (!make_map(&gp.map_b, B, 2, dims, str, box)) return PAC_ERR_UNSUPPORTED;
+        gp.map_b_pair = gp.map_b;
     } else {
         cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N};
         cuuint64_t str[1] = {(cuuint64_t)K * 2};
-        cuuint32_t box[2] = {GT_BK, GT_BN};
+        cuuint32_t box[2] = {GT_BK, GT_BN}, box_pair[2] = {GT_BK, GT_BN / 2};
         if (!make_map(&gp.map_b, B, 2, dims, str, box)) return PAC_ERR_UNSUPPORTED;
+        if (!make_map(&gp.map_b_pair, B, 2, dims, str, box_pair)) return PAC_ERR_UNSUPPORTED;
     }
-    if (smem_opt_in((const void*)gemm_tc_kernel, GT_SMEM) != cudaSuccess) {
+    gp.pair = pair && gp.sms >= 2;
+    if (smem_opt_in((const void*)gemm_tc_kernel<false>, GT_SMEM) != cudaSuccess ||
+        smem_opt_in((const void*)gemm_tc_kernel<true>, GT_SMEM_PAIR) != cudaSuccess) {
         tensor_err() = "cudaFuncSetAttribute(MaxDynamicSharedMemorySize) failed";
         cudaGetLastError();
         return PAC_ERR_CUDA;
@@ -400,11 +472,29 @@ inline pac_status gemm_launch(const GemmPlan& gp, cudaStream_t stream, int M, fl
     p.k_chunks = (gp.K + GT_BK - 1) / GT_BK;
     p.b_mn_major = gp.b_mn_major;
     p.C = C; p.ldc = ldc; p.status = status;
-    const int tiles = p.m_tiles * p.n_tiles;
-    const int grid = tiles < gp.sms ? tiles : gp.sms;
-    gemm_tc_kernel<<<grid, TC_THREADS, GT_SMEM, stream>>>(gp.map_a, gp.map_b, p);
+    cudaError_t e;
+    if (gp.pair) {
+        const int units = ((p.m_tiles + 1) / 2) * p.n_tiles, clusters = units < gp.sms / 2 ? units : gp.sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * clusters), 1, 1);
+        cfg.blockDim = dim3(TC_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = GT_SMEM_PAIR;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, gp.map_a, gp.map_b_pair, p);
+    } else {
+        const int tiles = p.m_tiles * p.n_tiles;
+        const int grid = tiles < gp.sms ? tiles : gp.sms;
+        gemm_tc_kernel<false><<<grid, TC_THREADS, GT_SMEM, stream>>>(gp.map_a, gp.map_b, p);
+        e = cudaGetLastError();
+    }
     (*launches)++;
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tensor_err() = cudaGetErrorString(e); return PAC_ERR_CUDA; }
     return PAC_OK;
 }

@@ -544,6 +544,13 @@ def test_lm_head_tensor_path_loss_and_gradients(spec):
     tc_check(spec, spec.B, 0, ids=[spec.N - 1, 0, 2, 2][:spec.B], head_tol=5e-3)
 
 
+@pytest.mark.parametrize("spec", LM_TC_SPECS, ids=lambda s: s.name)
+def test_lm_head_tensor_path_single_cta_gemms(spec):
+    """The LM head's GEMMs run as CTA pairs on 256 x 256 tiles by default (above); kernel path 5 keeps
+    their single-CTA form, 128 x 256 tiles, in use."""
+    tc_check(spec, spec.B, 0, ids=[spec.N - 1, 0, 2, 2][:spec.B], head_tol=5e-3, kernel_path=5)
+
+
 def test_lm_head_tensor_path_eval_logits():
     spec = LM_TC_SPECS[1]
     case = Case(spec)
