@@ -615,7 +615,8 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
     return v;
 }
 
-__global__ void __launch_bounds__(256) finalize_cls_kernel(FinalizeParams f) {
+// (five blocks per SM: 48 registers, no spills; T5-Base step 51.0 -> 50.3 us against the 63 registers of an open bound)
+__global__ void __launch_bounds__(256, 5) finalize_cls_kernel(FinalizeParams f) {
     pdl_trigger();
     const ParamLayout& lay = f.lay;
     // W_down blocks fetch the old parameter and moments while the predecessor still runs: nothing since the
