@@ -276,6 +276,8 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     unsigned mask[GPT][4];
     float ap[GPT][4];
     bool landed = false;
+    // column sums of a_L straight from registers when a warp holds whole tokens (one group per thread, 4, 8 or 16 groups per token)
+    const bool shuffle_sums = GPT == 1 && STATE != STATE_PARKED && groups_per_tok <= 32 && (32 % groups_per_tok) == 0;
 #pragma unroll
     for (int g = 0; g < GPT; ++g) {
 #pragma unroll
@@ -323,17 +325,32 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 }
             }
         }
-        if (s_local[g] < p.Sg) {
+        if (!shuffle_sums && s_local[g] < p.Sg) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) aL[(size_t)s_local[g] * r + j4[g] + e] = live[g] ? ap[g][e] : 0.f;
         }
+    }
+    if (shuffle_sums) {
+        // the lanes of a warp that hold the same four columns (one per token of the warp) add up by shuffles, in a
+        // fixed order; one partial sum per warp and column goes to shared memory
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = live[0] ? ap[0][e] : 0.f;
+        for (int off = groups_per_tok; off < 32; off <<= 1)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[e] += __shfl_xor_sync(0xffffffffu, v[e], off);
+        if (lane < groups_per_tok)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) lred[warp * r + (lane << 2) + e] = v[e];
     }
     __syncthreads();
     // column sums over this CTA's tokens: `parts` partial sums per column over contiguous token
     // ranges, then added in range order
     {
         int parts = 1;
-        if constexpr (STATE == STATE_PARKED) {
+        if (shuffle_sums) {
+            parts = nwarps;
+        } else if constexpr (STATE == STATE_PARKED) {
             // token-group sums from the down-projection kernel; CTA q of the cluster takes groups q, q + G, ...
             if (t < r) {
                 float acc = 0.f;
@@ -350,7 +367,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 lred[part * r + j] = acc;
             }
         }
-        __syncthreads();
+        if (!shuffle_sums) __syncthreads();
         if (t < r) {
             float acc = 0.f;
             for (int part = 0; part < parts; ++part) acc += lred[part * r + t];
@@ -782,6 +799,7 @@ inline size_t mid_base_floats(const Dims& dm, int Sg, int dg, int th, int* scrat
     int scratch = nw * MID_MAX_L;
     const int parts = th / dm.r > 0 ? th / dm.r : 1;
     if (parts * dm.r > scratch) scratch = parts * dm.r;
+    if (nw * dm.r > scratch) scratch = nw * dm.r;              // one partial column sum per warp
     *scratch_out = scratch;
     return (with_aL ? (size_t)Sg * dm.r : 0) + 2 * (size_t)dm.r + MID_MAX_C + 2 * (size_t)(dm.r + 1) * dm.C + (size_t)dg + MID_MAX_C + MID_MAX_L + scratch +
            (size_t)dg * dm.C + MID_MAX_L + 4;
