@@ -335,6 +335,7 @@ def test_tensor_path_separate_forward_kernels(spec, max_batch, act):
 TC_CHAIN_FORWARD = [s for s in TC_SPECS if s[0].r % 32 == 0 and s[0].r <= 128] + [
     (TC_BASE.scaled(name="tc_chain_r96", S=200, d=264, r=96, L=5, B=3), 3, 0),        # three 16-column chunks per warp, ragged S
     (TC_BASE.scaled(name="tc_chain_L32", S=130, d=128, r=32, L=32, B=2, N=6), 2, 0),  # every gate bit in use
+    (TC_BASE.scaled(name="tc_chain_odd_tiles", S=120, d=128, r=128, L=3, B=3, N=6), 3, 0),  # wide adapter, odd tile count: no CTA pairs
 ]
 
 
