@@ -479,20 +479,27 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
         // ring of MID_RING layers in shared memory (cp.async, each thread reads back only what it requested),
         // so that GPT * MID_RING loads per thread are in flight without holding registers.
         uint2* ring = reinterpret_cast<uint2*>(u_s);
-        auto request = [&](int l) {
-            if (l >= 0) {
+        // Running pointers instead of per-layer index arithmetic: src[g] walks the parked rows MID_RING layers
+        // ahead of dst[g] (the same slots of the du buffer), slot walks the ring.
+        DU* dst[GPT];
+        const DU* src[GPT];
 #pragma unroll
-                for (int g = 0; g < GPT; ++g)
-                    if (live[g]) cp_async_8(ring + ((size_t)(l % MID_RING) * GPT + g) * nt + t, du + (long long)l * p.lstride + base[g]);
+        for (int g = 0; g < GPT; ++g) { dst[g] = du + (long long)(L - 1) * p.lstride + base[g]; src[g] = dst[g]; }
+        uint2* const ring_t = ring + t;
+        const size_t slot_stride = (size_t)GPT * nt;
+        int slot = 0;                                            // ring slot of the layer consumed next
+        for (int i = 0; i < MID_RING; ++i) {
+            if (L - 1 - i >= 0) {
+#pragma unroll
+                for (int g = 0; g < GPT; ++g) {
+                    if (live[g]) cp_async_8(ring_t + (size_t)i * slot_stride + (size_t)g * nt, src[g]);
+                    src[g] -= p.lstride;
+                }
             }
             cp_async_commit();
-        };
-        for (int i = 0; i < MID_RING; ++i) request(L - 1 - i);
+        }
         // the launch geometry of this mode gives every group of a thread the same four columns, so the
         // per-layer coefficients are formed once per thread and layer
-        DU* dst[GPT];
-#pragma unroll
-        for (int g = 0; g < GPT; ++g) dst[g] = du + (long long)(L - 1) * p.lstride + base[g];
 #pragma unroll 1
         for (int l = L - 1; l >= 0; --l) {
             cp_async_wait_group<MID_RING - 1>();
@@ -501,10 +508,11 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             float dzc[4], duc[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) { dzc[e] = daLr[0][e] * cp; duc[e] = lm * dzc[e]; }
+            uint2* const rp = ring_t + (size_t)slot * slot_stride;
             uint2 x[GPT];
 #pragma unroll
             for (int g = 0; g < GPT; ++g)
-                if (live[g]) x[g] = ring[((size_t)(l % MID_RING) * GPT + g) * nt + t];
+                if (live[g]) x[g] = rp[(size_t)g * nt];
 #pragma unroll
             for (int g = 0; g < GPT; ++g) {
                 if (live[g]) {
@@ -526,7 +534,16 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 }
                 dst[g] -= p.lstride;
             }
-            request(l - MID_RING);
+            // the slot just consumed takes the layer MID_RING further down
+            if (l - MID_RING >= 0) {
+#pragma unroll
+                for (int g = 0; g < GPT; ++g) {
+                    if (live[g]) cp_async_8(rp + (size_t)g * nt, src[g]);
+                    src[g] -= p.lstride;
+                }
+            }
+            cp_async_commit();
+            if (++slot == MID_RING) slot = 0;
             part = warp_sum(part);
             if (lane == 0) lred[warp * LT + l] = part;
         }
