@@ -453,7 +453,7 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             top_closed[g][e] = 31 - __clz(closed);        // __clz(0) = 32
         }
     // one layer of one group: du_l out, this thread's share of dlambda_l added to `part`
-    auto reverse_step = [&](int l, int g, const float4& w4, float& part, float cp, float lm) {
+    auto reverse_step = [&](int l, int g, const float4& w4, float& part, float cp, float lm, DU* dst) {
         const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
         float dv[4];
 #pragma unroll
@@ -463,7 +463,6 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
             part = fmaf(dz, wv[e], part);
             dv[e] = lm * dz;                                   // du_l
         }
-        DU* dst = du + (long long)l * p.lstride + base[g];
         if constexpr (sizeof(DU) == 2) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(dv[0], dv[1]), hi = __floats2bfloat162_rn(dv[2], dv[3]);
             uint2 pk;
@@ -550,6 +549,9 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
     } else {
         // layers per batch: about four state loads in flight per thread whatever the number of groups it owns
         constexpr int LB = GPT >= 4 ? 1 : 4 / GPT;
+        DU* dstp[GPT];                                        // running pointers into du, one layer down per step
+#pragma unroll
+        for (int g = 0; g < GPT; ++g) dstp[g] = du + (long long)(L - 1) * p.lstride + base[g];
 #pragma unroll 1
         for (int l0 = L - 1; l0 >= 0; l0 -= LB) {
             float4 wq[LB][GPT];
@@ -565,8 +567,10 @@ __device__ __forceinline__ void mid_body(const MidParams& p, cg::cluster_group& 
                 if (l0 - i >= 0) {
                     const float cp = cprod[l0 - i], lm = lam_s[l0 - i];
 #pragma unroll
-                    for (int g = 0; g < GPT; ++g)
-                        if (live[g]) reverse_step(l0 - i, g, wq[i][g], part[i], cp, lm);
+                    for (int g = 0; g < GPT; ++g) {
+                        if (live[g]) reverse_step(l0 - i, g, wq[i][g], part[i], cp, lm, dstp[g]);
+                        dstp[g] -= p.lstride;
+                    }
                 }
             }
             // this warp's shares of dlambda of the batch's layers: independent shuffle trees
